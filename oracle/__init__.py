@@ -1,0 +1,169 @@
+"""ctypes front end of the CPU oracle (``moe_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: the tests, the smoke check and the benchmark's CPU-baseline leg may
+import this; the CUDA package never does.  Every function takes and returns host numpy arrays.
+bf16 tensors are ``uint16`` arrays of bit patterns; ``dtype`` is 0 for fp32, 1 for bf16.
+
+The steps are those of Section II-A of the paper (routing, dispatch, expert computation,
+combine, scaling); the dispatch layout is the dense per-expert packing of Section IV-B.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "moe_oracle.c")
+_SO = os.path.join(_HERE, "libmoe_oracle.so")
+_lib = None
+
+FP32, BF16 = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (no CUDA involved). Returns the path of the shared object."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fopenmp", "-shared", "-fPIC",
+               _SRC, "-o", _SO, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _SO
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().oracle_num_threads())
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _storage(a: np.ndarray, dtype: int) -> np.ndarray:
+    want = np.float32 if dtype == FP32 else np.uint16
+    assert a.dtype == want, f"expected {want}, got {a.dtype}"
+    return np.ascontiguousarray(a)
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise RuntimeError(f"{what} failed with code {rc}")
+
+
+def logits(x, wr, bias, dtype):
+    T, H = x.shape
+    E = wr.shape[0]
+    x, wr = _storage(x, dtype), _storage(wr, dtype)
+    b = None if bias is None else np.ascontiguousarray(bias, np.float32)
+    out = np.empty((T, E), np.float32)
+    _check(lib().oracle_logits(T, H, E, dtype, _p(x), _p(wr), _p(b), _p(out)), "oracle_logits")
+    return out
+
+
+def topk(lg, K, renormalize=0):
+    lg = np.ascontiguousarray(lg, np.float32)
+    T, E = lg.shape
+    idx = np.empty((T, K), np.int32)
+    w = np.empty((T, K), np.float32)
+    _check(lib().oracle_topk(T, E, K, int(renormalize), _p(lg), _p(idx), _p(w)), "oracle_topk")
+    return idx, w
+
+
+def route(x, wr, bias, K, dtype, renormalize=0):
+    """Returns (topk_idx[T,K] int32, topk_w[T,K] fp32, logits[T,E] fp32)."""
+    T, H = x.shape
+    E = wr.shape[0]
+    x, wr = _storage(x, dtype), _storage(wr, dtype)
+    b = None if bias is None else np.ascontiguousarray(bias, np.float32)
+    idx = np.empty((T, K), np.int32)
+    w = np.empty((T, K), np.float32)
+    lg = np.empty((T, E), np.float32)
+    _check(lib().oracle_route(T, H, E, K, dtype, int(renormalize), _p(x), _p(wr), _p(b), _p(idx), _p(w),
+                              _p(lg)), "oracle_route")
+    return idx, w, lg
+
+
+def dispatch(x, topk_idx, E, R, dtype, want_rows=True):
+    """Returns dict(count[E], offset[E+1], rank_count[R], recv[T*K,H] or None, src[T*K], slot_of[T,K])."""
+    T, H = x.shape
+    K = topk_idx.shape[1]
+    x = _storage(x, dtype)
+    idx = np.ascontiguousarray(topk_idx, np.int32)
+    count = np.empty(E, np.int32)
+    offset = np.empty(E + 1, np.int32)
+    rank_count = np.empty(R, np.int32)
+    recv = np.empty((T * K, H), x.dtype) if want_rows else None
+    src = np.empty(T * K, np.int32)
+    slot_of = np.empty((T, K), np.int32)
+    _check(lib().oracle_dispatch(T, H, E, R, K, dtype, _p(x), _p(idx), _p(count), _p(offset), _p(rank_count),
+                                 _p(recv), _p(src), _p(slot_of)), "oracle_dispatch")
+    return dict(count=count, offset=offset, rank_count=rank_count, recv=recv, src=src, slot_of=slot_of)
+
+
+def expert_ffn(recv, offset, wg, wu, wd, dtype):
+    """wg/wu/wd: sequences of E per-expert arrays ([F,H],[F,H],[H,F]); None allowed for empty experts.
+
+    Returns out[rows,H] fp64."""
+    rows, H = recv.shape
+    E = len(wg)
+    recv = _storage(recv, dtype)
+    offset = np.ascontiguousarray(offset, np.int32)
+    F = next(a.shape[0] for a in wg if a is not None)
+    keep = []
+
+    def ptrs(ws):
+        arr = (ctypes.c_void_p * E)()
+        for e, a in enumerate(ws):
+            if a is None:
+                arr[e] = None
+            else:
+                a = _storage(a, dtype)
+                keep.append(a)
+                arr[e] = a.ctypes.data
+        return arr
+
+    out = np.empty((rows, H), np.float64)
+    _check(lib().oracle_expert_ffn(H, F, E, dtype, _p(recv), _p(offset), ptrs(wg), ptrs(wu), ptrs(wd),
+                                   _p(out)), "oracle_expert_ffn")
+    return out
+
+
+def identity_ffn(recv, dtype):
+    rows, H = recv.shape
+    recv = _storage(recv, dtype)
+    out = np.empty((rows, H), np.float64)
+    lib().oracle_identity_ffn.argtypes = [ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+                                          ctypes.c_void_p]
+    _check(lib().oracle_identity_ffn(rows, H, dtype, _p(recv), _p(out)), "oracle_identity_ffn")
+    return out
+
+
+def combine(rows, slot_of, topk_w):
+    rows = np.ascontiguousarray(rows, np.float64)
+    T, K = slot_of.shape
+    H = rows.shape[1]
+    slot_of = np.ascontiguousarray(slot_of, np.int32)
+    topk_w = np.ascontiguousarray(topk_w, np.float32)
+    y = np.empty((T, H), np.float64)
+    _check(lib().oracle_combine(T, H, K, _p(rows), _p(slot_of), _p(topk_w), _p(y)), "oracle_combine")
+    return y
+
+
+def layer(x, wr, bias, wg, wu, wd, E, R, K, dtype, renormalize=0, identity_experts=False):
+    """The whole layer: route -> dispatch -> experts -> combine. Returns dict with every stage's output."""
+    idx, w, lg = route(x, wr, bias, K, dtype, renormalize)
+    d = dispatch(x, idx, E, R, dtype)
+    if identity_experts:
+        rows = identity_ffn(d["recv"], dtype)
+    else:
+        rows = expert_ffn(d["recv"], d["offset"], wg, wu, wd, dtype)
+    y = combine(rows, d["slot_of"], w)
+    return dict(topk_idx=idx, topk_w=w, logits=lg, out_rows=rows, y=y, **d)
