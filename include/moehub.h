@@ -1,0 +1,162 @@
+/*
+ * moehub.h — C ABI of the B200 (sm_100a) MoE-layer hot path.
+ *
+ * The path is the five-step MoE layer of Section II-A of the paper "MoE-Hub" (routing,
+ * all-to-all dispatch, expert computation, all-to-all combine, scaling) on ONE GPU, where the
+ * E experts are partitioned over R logical expert-parallel ranks that are buffer partitions
+ * only (expert e lives on rank e / (E/R)).  The paper's destination-agnostic dispatch
+ * (Section IV-A/IV-B: a producer sends a row as soon as its expert id is known and the consumer
+ * side hands out the next free row of that expert's region, address =
+ * BaseAddr + LocalRowID*RowSize + RowOffset) is realised in software: slot allocation by
+ * aggregated atomics on per-expert row pointers.  The conventional "software mediation"
+ * (Section III-A: counts -> scan -> offsets -> shuffle) is kept as dispatch mode 0, the
+ * baseline it is shown against.
+ *
+ * General rules
+ *  - Every pointer named d_* is DEVICE memory owned by the caller; h_* is HOST memory.  The
+ *    library allocates no device memory: its scratch is the caller's workspace (see
+ *    moe_workspace_bytes / moe_plan_create).  A plan owns host-side metadata only.
+ *  - dtype 0: fp32, dtype 1: bf16.  It is the type of x, the router weight, the expert
+ *    weights, the receive buffers, the expert outputs and y.  Routing weights are fp32,
+ *    indices int32.  All matrices are row-major and dense.
+ *  - Alignment: H*elem and F*elem must be multiples of 16 bytes; device pointers must be
+ *    16-byte aligned (cudaMalloc / torch allocations are).
+ *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default
+ *    stream).  Return value: 0 = MOE_OK, negative = error found on the host before anything
+ *    was launched.  Errors found on the device (region overflow, a bounded wait that ran out)
+ *    are left in a device status word: read it with moe_last_status.
+ *  - A plan is used by one host thread / one stream at a time.  No global state.
+ *  - Receive-buffer geometry: rows live in a pool of P tiles of 128 rows
+ *    (moe_pool_tiles).  tile_expert[p] names the expert that owns tile p (-1: unused).  An
+ *    expert's rows are dense inside its tiles (only its last tile may be partly filled).
+ *    Physical row = tile*128 + row-in-tile.  Within one expert the order of rows is
+ *    unspecified in the atomic modes (arrival order, Section IV-B) and is (token, k) order in
+ *    mode 0.
+ */
+#ifndef MOEHUB_H_
+#define MOEHUB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MOE_OK 0
+#define MOE_ERR_ARG (-1)         /* null pointer, non-positive size, K > E, E % R != 0, ... */
+#define MOE_ERR_ALIGN (-2)       /* H or F row pitch not a multiple of 16 bytes, misaligned pointer */
+#define MOE_ERR_UNSUPPORTED (-3) /* outside what the kernels cover (E > 256, K > 32, ...) */
+#define MOE_ERR_CUDA (-4)        /* a CUDA runtime/driver call failed */
+#define MOE_ERR_OVERFLOW (-5)    /* device status: an expert's region (mode 1) or the pool is full */
+#define MOE_ERR_TIMEOUT (-6)     /* device status: a bounded device-side wait ran out */
+#define MOE_ERR_WORKSPACE (-7)   /* workspace too small or misaligned */
+
+#define MOE_DTYPE_FP32 0
+#define MOE_DTYPE_BF16 1
+
+#define MOE_DISPATCH_SCAN 0          /* baseline: histogram -> exclusive scan -> stable scatter */
+#define MOE_DISPATCH_ATOMIC_STATIC 1 /* row-pointer atomics, one static region per expert   */
+#define MOE_DISPATCH_ATOMIC_PAGED 2  /* row-pointer atomics, 128-row tiles paged on demand  */
+
+#define MOE_TILE_ROWS 128
+
+typedef struct moe_plan moe_plan_t; /* opaque */
+
+typedef struct {
+  int32_t T, H, E, R, K, F;     /* tokens, hidden, experts, logical ranks, top-K, FFN width   */
+  int32_t dtype;                /* MOE_DTYPE_*                                               */
+  int32_t renormalize;          /* 0: w = softmax prob. of the picked experts; 1: / their sum */
+  int32_t dispatch_mode;        /* MOE_DISPATCH_*                                            */
+  int32_t identity_experts;     /* 1: moe_layer skips the FFN (expert output = expert input)  */
+  int32_t ffn_kernel;           /* 0: tensor-core (tcgen05) kernel for bf16, SIMT for fp32;
+                                   1: SIMT fp32-FMA kernel for either dtype (check path)      */
+  int32_t reserved;
+  int64_t capacity_rows;        /* mode 1: rows per expert region, multiple of 128, 0 = T
+                                   rounded up (overflow-free); modes 0/2: ignored            */
+  uint64_t spin_limit;          /* bound on every device-side wait, 0 = default (1<<22)      */
+} moe_config_t;
+
+/* Number P of 128-row tiles in the receive pool for this configuration:
+ * modes 0/2: floor(T*K/128) + E;  mode 1: E * capacity_rows/128. */
+int moe_pool_tiles(const moe_config_t* cfg, int64_t* out_tiles);
+
+/* Bytes of device workspace moe_plan_create needs (scratch counters, tile tables, the SwiGLU
+ * intermediate, and the internal buffers moe_layer uses between its stages). */
+int moe_workspace_bytes(const moe_config_t* cfg, size_t* out_bytes);
+
+/* Analogue of the paper's rowspMalloc (Section IV-A, runtime API): registers the receive
+ * regions (base, row size, tile pool) once.  d_workspace: device memory, 256-byte aligned,
+ * at least moe_workspace_bytes() long, owned by the caller, must outlive the plan's queued
+ * work.  Runs on the current CUDA device.  *out is freed by moe_plan_destroy. */
+int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, moe_plan_t** out);
+int moe_plan_destroy(moe_plan_t* plan);
+
+/* Step 1 (Section II-A, routing): logits l[t,e] = sum_h x[t,h]*Wr[e,h] (+bias[e]) as one
+ * ascending fp32 FMA chain, softmax over the E experts, the K largest logits (lowest index
+ * wins ties), in descending order.
+ * d_x [T,H], d_wr [E,H] (dtype); d_bias [E] fp32 or NULL;
+ * out: d_topk_idx [T,K] int32, d_topk_w [T,K] fp32. */
+int moe_route(moe_plan_t* plan, const void* d_x, const void* d_wr, const float* d_bias,
+              int32_t* d_topk_idx, float* d_topk_w, void* stream);
+
+/* Step 2 (Section II-A dispatch; address resolution per Section III-A in mode 0, per
+ * Section IV-B in modes 1/2): copies x[t,:] to one slot of each of its K experts.
+ * in: d_x [T,H], d_topk_idx [T,K].
+ * out: d_recv [P*128,H] (dtype; rows of unused slots are left untouched),
+ *      d_expert_count [E] rows per expert, d_tile_expert [P] owner of each tile or -1,
+ *      d_src_info [P*128] = t*K+k of the row in that slot, -1 for an empty slot (the source
+ *      information of Section IV-B, combine), d_slot_of [T,K] physical row of assignment
+ *      (t,k), or -1 if it was dropped by an overflow (status MOE_ERR_OVERFLOW). */
+int moe_dispatch(moe_plan_t* plan, const void* d_x, const int32_t* d_topk_idx, void* d_recv,
+                 int32_t* d_expert_count, int32_t* d_tile_expert, int32_t* d_src_info,
+                 int32_t* d_slot_of, void* stream);
+
+/* Step 3 (Section II-A, expert computation; "two GEMMs with an activation between", here
+ * SwiGLU): for every used tile p of expert e = tile_expert[p]:
+ *   S = silu(A*Wg[e]^T) .* (A*Wu[e]^T),  O = S*Wd[e]^T,  A = the tile's 128 rows of d_recv.
+ * Unused tiles are skipped and their experts' weights never read (Section IV-D: thread
+ * blocks whose counters stay zero are never scheduled).
+ * in: d_recv [P*128,H], d_tile_expert [P], d_wg/d_wu [E,F,H], d_wd [E,H,F] (dtype).
+ * out: d_out_rows [P*128,H] (dtype); rows of empty slots hold unspecified values. */
+int moe_expert_ffn(moe_plan_t* plan, const void* d_recv, const int32_t* d_tile_expert,
+                   const void* d_wg, const void* d_wu, const void* d_wd, void* d_out_rows,
+                   void* stream);
+
+/* Steps 4+5 (Section II-A, combine and scaling): y[t,:] = sum_k w[t,k]*rows[slot_of[t,k],:],
+ * k ascending, fp32 accumulation, rounded once to dtype.  Assignments with slot -1 add 0.
+ * in: d_rows [P*128,H] (dtype), d_slot_of [T,K], d_topk_w [T,K].  out: d_y [T,H] (dtype). */
+int moe_combine(moe_plan_t* plan, const void* d_rows, const int32_t* d_slot_of,
+                const float* d_topk_w, void* d_y, void* stream);
+
+/* The whole layer, steps 1-5, on device buffers: route -> dispatch -> experts -> combine,
+ * intermediate buffers in the plan's workspace. */
+int moe_layer(moe_plan_t* plan, const void* d_x, const void* d_wr, const float* d_bias,
+              const void* d_wg, const void* d_wu, const void* d_wd, void* d_y, void* stream);
+
+/* The whole layer with the activations in HOST memory: copies h_x [T,H] to the device,
+ * runs moe_layer, copies y back to h_y [T,H] and synchronises the stream.  Weights stay
+ * device-resident (they are parameters, not per-step inputs).  Pinned host memory makes the
+ * copies asynchronous to the host but the call still returns only when h_y is complete. */
+int moe_layer_host(moe_plan_t* plan, const void* h_x, const void* d_wr, const float* d_bias,
+                   const void* d_wg, const void* d_wu, const void* d_wd, void* h_y, void* stream);
+
+/* Device pointers of moe_layer's intermediate results inside the workspace (valid after a
+ * moe_layer call completes): which = 0 topk_idx, 1 topk_w, 2 recv, 3 expert_count,
+ * 4 tile_expert, 5 src_info, 6 slot_of, 7 out_rows. */
+int moe_layer_buffer(moe_plan_t* plan, int which, void** out_ptr);
+
+/* Number of kernels the last stage call (or moe_layer) launched. */
+int moe_last_launch_count(moe_plan_t* plan, int32_t* out);
+
+/* Synchronises `stream` and reads the device status word: *code is MOE_OK, MOE_ERR_OVERFLOW
+ * or MOE_ERR_TIMEOUT; *detail says where (expert id for an overflow, wait site for a
+ * timeout). */
+int moe_last_status(moe_plan_t* plan, void* stream, int32_t* code, int32_t* detail);
+
+const char* moe_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOEHUB_H_ */

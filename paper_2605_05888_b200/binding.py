@@ -1,0 +1,197 @@
+"""Thin ctypes binding of libmoehub.so (the C ABI in include/moehub.h).
+
+Argument marshalling only: every step of the path runs in the CUDA kernels behind the C ABI.
+torch is used for device memory and streams.  There is no CPU fallback: if the library is
+missing or no CUDA device is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libmoehub.so")
+_lib = None
+
+MOE_OK = 0
+DTYPE_FP32, DTYPE_BF16 = 0, 1
+DISPATCH_SCAN, DISPATCH_ATOMIC_STATIC, DISPATCH_ATOMIC_PAGED = 0, 1, 2
+TILE_ROWS = 128
+
+EXPORTS = ["moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
+           "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host", "moe_layer_buffer",
+           "moe_last_launch_count", "moe_last_status", "moe_strerror"]
+
+
+class MoeConfig(ctypes.Structure):
+    _fields_ = [("T", ctypes.c_int32), ("H", ctypes.c_int32), ("E", ctypes.c_int32), ("R", ctypes.c_int32),
+                ("K", ctypes.c_int32), ("F", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("renormalize", ctypes.c_int32), ("dispatch_mode", ctypes.c_int32),
+                ("identity_experts", ctypes.c_int32), ("ffn_kernel", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("capacity_rows", ctypes.c_int64), ("spin_limit", ctypes.c_uint64)]
+
+
+class MoeError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {strerror(code)} ({code})")
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libmoehub.so (built in-tree by build.py). Raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_SO):
+            raise RuntimeError(f"{_SO} not found: build it with paper_2605_05888_b200/build.py (needs nvcc)")
+        L = ctypes.CDLL(_SO)
+        vp, i32p, fp = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p
+        cfgp = ctypes.POINTER(MoeConfig)
+        L.moe_pool_tiles.argtypes = [cfgp, ctypes.POINTER(ctypes.c_int64)]
+        L.moe_workspace_bytes.argtypes = [cfgp, ctypes.POINTER(ctypes.c_size_t)]
+        L.moe_plan_create.argtypes = [cfgp, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
+        L.moe_plan_destroy.argtypes = [vp]
+        L.moe_route.argtypes = [vp, vp, vp, fp, i32p, fp, vp]
+        L.moe_dispatch.argtypes = [vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp]
+        L.moe_expert_ffn.argtypes = [vp, vp, i32p, vp, vp, vp, vp, vp]
+        L.moe_combine.argtypes = [vp, vp, i32p, fp, vp, vp]
+        L.moe_layer.argtypes = [vp] * 9
+        L.moe_layer_host.argtypes = [vp] * 9
+        L.moe_layer_buffer.argtypes = [vp, ctypes.c_int, ctypes.POINTER(vp)]
+        L.moe_last_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
+        L.moe_last_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+        L.moe_strerror.argtypes = [ctypes.c_int]
+        L.moe_strerror.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            if name != "moe_strerror":
+                getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def strerror(code: int) -> str:
+    return lib().moe_strerror(code).decode()
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != MOE_OK:
+        raise MoeError(rc, where)
+
+
+def _ptr(t) -> int | None:
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    assert t.is_contiguous()
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def make_config(T, H, E, R, K, F, dtype, renormalize=0, dispatch_mode=DISPATCH_ATOMIC_PAGED, identity_experts=0,
+                ffn_kernel=0, capacity_rows=0, spin_limit=0) -> MoeConfig:
+    return MoeConfig(T, H, E, R, K, F, dtype, int(renormalize), dispatch_mode, int(identity_experts), ffn_kernel, 0,
+                     capacity_rows, spin_limit)
+
+
+def moe_pool_tiles(cfg: MoeConfig) -> int:
+    out = ctypes.c_int64()
+    _check(lib().moe_pool_tiles(ctypes.byref(cfg), ctypes.byref(out)), "moe_pool_tiles")
+    return out.value
+
+
+def moe_workspace_bytes(cfg: MoeConfig) -> int:
+    out = ctypes.c_size_t()
+    _check(lib().moe_workspace_bytes(ctypes.byref(cfg), ctypes.byref(out)), "moe_workspace_bytes")
+    return out.value
+
+
+class Plan:
+    """Owns a moe_plan_t and the torch-allocated workspace it points into."""
+
+    def __init__(self, cfg: MoeConfig, device="cuda"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("moehub needs a CUDA device; there is no CPU path")
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.P = moe_pool_tiles(cfg)
+        nbytes = moe_workspace_bytes(cfg)
+        with torch.cuda.device(self.device):
+            self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=self.device)
+            base = (self.workspace.data_ptr() + 255) // 256 * 256
+            h = ctypes.c_void_p()
+            _check(lib().moe_plan_create(ctypes.byref(cfg), base, nbytes, ctypes.byref(h)), "moe_plan_create")
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None) and _lib is not None:
+            _lib.moe_plan_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+    # ---- the C ABI, same names -------------------------------------------------------------
+    def moe_route(self, x, wr, bias, topk_idx, topk_w, stream=None):
+        _check(lib().moe_route(self.handle, _ptr(x), _ptr(wr), _ptr(bias), _ptr(topk_idx), _ptr(topk_w),
+                               _stream(stream)), "moe_route")
+
+    def moe_dispatch(self, x, topk_idx, recv, expert_count, tile_expert, src_info, slot_of, stream=None):
+        _check(lib().moe_dispatch(self.handle, _ptr(x), _ptr(topk_idx), _ptr(recv), _ptr(expert_count),
+                                  _ptr(tile_expert), _ptr(src_info), _ptr(slot_of), _stream(stream)), "moe_dispatch")
+
+    def moe_expert_ffn(self, recv, tile_expert, wg, wu, wd, out_rows, stream=None):
+        _check(lib().moe_expert_ffn(self.handle, _ptr(recv), _ptr(tile_expert), _ptr(wg), _ptr(wu), _ptr(wd),
+                                    _ptr(out_rows), _stream(stream)), "moe_expert_ffn")
+
+    def moe_combine(self, rows, slot_of, topk_w, y, stream=None):
+        _check(lib().moe_combine(self.handle, _ptr(rows), _ptr(slot_of), _ptr(topk_w), _ptr(y), _stream(stream)),
+               "moe_combine")
+
+    def moe_layer(self, x, wr, bias, wg, wu, wd, y, stream=None):
+        _check(lib().moe_layer(self.handle, _ptr(x), _ptr(wr), _ptr(bias), _ptr(wg), _ptr(wu), _ptr(wd), _ptr(y),
+                               _stream(stream)), "moe_layer")
+
+    def moe_layer_host(self, h_x, wr, bias, wg, wu, wd, h_y, stream=None):
+        """h_x, h_y: HOST tensors (pinned for asynchronous copies); weights: device tensors."""
+        assert not h_x.is_cuda and not h_y.is_cuda
+        _check(lib().moe_layer_host(self.handle, _ptr(h_x), _ptr(wr), _ptr(bias), _ptr(wg), _ptr(wu), _ptr(wd),
+                                    _ptr(h_y), _stream(stream)), "moe_layer_host")
+
+    def moe_layer_buffer(self, which: int) -> int:
+        out = ctypes.c_void_p()
+        _check(lib().moe_layer_buffer(self.handle, which, ctypes.byref(out)), "moe_layer_buffer")
+        return out.value
+
+    def moe_last_launch_count(self) -> int:
+        out = ctypes.c_int32()
+        _check(lib().moe_last_launch_count(self.handle, ctypes.byref(out)), "moe_last_launch_count")
+        return out.value
+
+    def moe_last_status(self, stream=None) -> tuple[int, int]:
+        code, detail = ctypes.c_int32(), ctypes.c_int32()
+        _check(lib().moe_last_status(self.handle, _stream(stream), ctypes.byref(code), ctypes.byref(detail)),
+               "moe_last_status")
+        return code.value, detail.value
+
+    # ---- convenience: read one of moe_layer's internal buffers back as a torch tensor ----------
+    def layer_tensor(self, which: int) -> torch.Tensor:
+        c = self.cfg
+        rows = self.P * TILE_ROWS
+        el = torch.bfloat16 if c.dtype == DTYPE_BF16 else torch.float32
+        shapes = {0: ((c.T, c.K), torch.int32), 1: ((c.T, c.K), torch.float32), 2: ((rows, c.H), el),
+                  3: ((c.E,), torch.int32), 4: ((self.P,), torch.int32), 5: ((rows,), torch.int32),
+                  6: ((c.T, c.K), torch.int32), 7: ((rows, c.H), el)}
+        shape, dt = shapes[which]
+        ptr = self.moe_layer_buffer(which)
+        off = ptr - self.workspace.data_ptr()
+        n = 1
+        for s in shape:
+            n *= s
+        nbytes = n * torch.empty(0, dtype=dt).element_size()
+        return self.workspace[off: off + nbytes].view(dt).view(shape)

@@ -1,0 +1,278 @@
+// The C ABI declared in include/moehub.h: argument checks, workspace carving, stage launches.
+// No device memory is allocated here; every buffer is the caller's.
+#include <new>
+#include <string.h>
+
+#include "common.cuh"
+
+using namespace moehub;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct Geometry {
+  int64_t P, cap_rows;
+  int tiles_per_expert, dispatch_tokens, nblk, eb;
+};
+
+int check_config(const moe_config_t* c, Geometry* g) {
+  if (!c) return MOE_ERR_ARG;
+  if (c->T < 0 || c->H <= 0 || c->E <= 0 || c->R <= 0 || c->K <= 0) return MOE_ERR_ARG;
+  if (c->K > c->E || c->E % c->R != 0) return MOE_ERR_ARG;
+  if (c->dtype != MOE_DTYPE_FP32 && c->dtype != MOE_DTYPE_BF16) return MOE_ERR_ARG;
+  if (c->dispatch_mode < 0 || c->dispatch_mode > 2) return MOE_ERR_ARG;
+  if (!c->identity_experts && c->F <= 0) return MOE_ERR_ARG;
+  if (c->E > 256 || c->K > 32) return MOE_ERR_UNSUPPORTED;
+  const int eb = c->dtype == MOE_DTYPE_BF16 ? 2 : 4;
+  if (((int64_t)c->H * eb) % 16 != 0) return MOE_ERR_ALIGN;
+  if (!c->identity_experts && ((int64_t)c->F * eb) % 16 != 0) return MOE_ERR_ALIGN;
+  if ((int64_t)c->T * c->K >= (1ll << 31) / 2) return MOE_ERR_UNSUPPORTED;
+  g->eb = eb;
+  const int64_t rows = (int64_t)c->T * c->K;
+  if (c->dispatch_mode == MOE_DISPATCH_ATOMIC_STATIC) {
+    int64_t cap = c->capacity_rows > 0 ? c->capacity_rows : (c->T + kTileRows - 1) / kTileRows * kTileRows;
+    if (cap % kTileRows != 0) return MOE_ERR_ARG;
+    if (cap == 0) cap = kTileRows;
+    g->cap_rows = cap;
+    g->P = (int64_t)c->E * (cap / kTileRows);
+  } else {
+    g->cap_rows = 0;
+    g->P = rows / kTileRows + c->E;
+  }
+  if (g->P * kTileRows >= (1ll << 31)) return MOE_ERR_UNSUPPORTED;
+  g->tiles_per_expert = (c->T + kTileRows - 1) / kTileRows;
+  if (g->tiles_per_expert == 0) g->tiles_per_expert = 1;
+  int tpb = 256 / c->K;  // at most 256 assignments per dispatch CTA
+  if (tpb > 16) tpb = 16;
+  if (tpb < 1) tpb = 1;
+  g->dispatch_tokens = tpb;
+  g->nblk = (c->T + tpb - 1) / tpb;
+  return MOE_OK;
+}
+
+// Lays the scratch out in the workspace; with base == nullptr only measures it.
+size_t carve(const moe_config_t& c, const Geometry& g, char* base, Scratch* s, size_t* counters_bytes) {
+  size_t off = 0;
+  auto take = [&](size_t bytes) -> char* {
+    char* ptr = base ? base + off : nullptr;
+    off += align_up(bytes);
+    return ptr;
+  };
+  Scratch t;
+  memset(&t, 0, sizeof t);
+  // leading block, cleared by every dispatch: status, pool_next, scan_ticket
+  t.status = (int*)take(sizeof(int) * 4);
+  t.pool_next = (int*)take(sizeof(int));
+  t.scan_ticket = (int*)take(sizeof(int));
+  if (counters_bytes) *counters_bytes = off;
+  t.tile_table = (int*)take(sizeof(int) * (size_t)c.E * g.tiles_per_expert);
+  t.cta_count = (int*)take(sizeof(int) * (size_t)(g.nblk > 0 ? g.nblk : 1) * c.E);
+  t.cta_base = (int*)take(sizeof(int) * (size_t)(g.nblk > 0 ? g.nblk : 1) * c.E);
+  t.tile_base = (int*)take(sizeof(int) * (size_t)(c.E + 1));
+  t.tile_list = (int*)take(sizeof(int) * (size_t)(g.P > 0 ? g.P : 1));
+  t.expert_start = (int*)take(sizeof(int) * (size_t)(c.E + 1));
+  const size_t pool_rows = (size_t)g.P * kTileRows;
+  if (!c.identity_experts) t.inter = take(pool_rows * c.F * g.eb);
+  t.topk_idx = (int*)take(sizeof(int) * (size_t)c.T * c.K);
+  t.topk_w = (float*)take(sizeof(float) * (size_t)c.T * c.K);
+  t.recv = take(pool_rows * c.H * g.eb);
+  t.out_rows = c.identity_experts ? t.recv : take(pool_rows * c.H * g.eb);
+  t.expert_count = (int*)take(sizeof(int) * (size_t)c.E);
+  t.tile_expert = (int*)take(sizeof(int) * (size_t)g.P);
+  t.src_info = (int*)take(sizeof(int) * pool_rows);
+  t.slot_of = (int*)take(sizeof(int) * (size_t)c.T * c.K);
+  t.x_stage = take((size_t)c.T * c.H * g.eb);
+  t.y_stage = take((size_t)c.T * c.H * g.eb);
+  if (s) *s = t;
+  return off;
+}
+
+inline bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) != 0; }
+
+}  // namespace
+
+extern "C" {
+
+int moe_pool_tiles(const moe_config_t* cfg, int64_t* out_tiles) {
+  Geometry g;
+  if (!out_tiles) return MOE_ERR_ARG;
+  int rc = check_config(cfg, &g);
+  if (rc != MOE_OK) return rc;
+  *out_tiles = g.P;
+  return MOE_OK;
+}
+
+int moe_workspace_bytes(const moe_config_t* cfg, size_t* out_bytes) {
+  Geometry g;
+  if (!out_bytes) return MOE_ERR_ARG;
+  int rc = check_config(cfg, &g);
+  if (rc != MOE_OK) return rc;
+  *out_bytes = carve(*cfg, g, nullptr, nullptr, nullptr);
+  return MOE_OK;
+}
+
+int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, moe_plan_t** out) {
+  Geometry g;
+  if (!out) return MOE_ERR_ARG;
+  *out = nullptr;
+  int rc = check_config(cfg, &g);
+  if (rc != MOE_OK) return rc;
+  if (!d_workspace) return MOE_ERR_ARG;
+  if (reinterpret_cast<uintptr_t>(d_workspace) % kAlign != 0) return MOE_ERR_WORKSPACE;
+  if (bytes < carve(*cfg, g, nullptr, nullptr, nullptr)) return MOE_ERR_WORKSPACE;
+  moe_plan* p = new (std::nothrow) moe_plan();
+  if (!p) return MOE_ERR_ARG;
+  p->cfg = *cfg;
+  p->P = g.P;
+  p->cap_rows = g.cap_rows;
+  p->tiles_per_expert = g.tiles_per_expert;
+  p->dispatch_tokens = g.dispatch_tokens;
+  p->nblk = g.nblk;
+  p->launches = 0;
+  p->encode_tiled = nullptr;
+  carve(*cfg, g, (char*)d_workspace, &p->s, &p->counters_bytes);
+  if (cudaGetDevice(&p->device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device) != cudaSuccess) {
+    delete p;
+    return MOE_ERR_CUDA;
+  }
+  // The status word must start clean even if a stage other than dispatch is called first.
+  if (cudaMemset(p->s.status, 0, p->counters_bytes) != cudaSuccess) {
+    delete p;
+    return MOE_ERR_CUDA;
+  }
+  *out = p;
+  return MOE_OK;
+}
+
+int moe_plan_destroy(moe_plan_t* plan) {
+  delete plan;
+  return MOE_OK;
+}
+
+int moe_route(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_bias, int32_t* d_topk_idx,
+              float* d_topk_w, void* stream) {
+  if (!p || !d_wr || !d_topk_idx || !d_topk_w || (!d_x && p->cfg.T > 0)) return MOE_ERR_ARG;
+  if (misaligned(d_x) || misaligned(d_wr)) return MOE_ERR_ALIGN;
+  p->launches = 0;
+  return launch_route(p, d_x, d_wr, d_bias, d_topk_idx, d_topk_w, (cudaStream_t)stream) ? MOE_ERR_CUDA : MOE_OK;
+}
+
+int moe_dispatch(moe_plan_t* p, const void* d_x, const int32_t* d_topk_idx, void* d_recv,
+                 int32_t* d_expert_count, int32_t* d_tile_expert, int32_t* d_src_info, int32_t* d_slot_of,
+                 void* stream) {
+  if (!p || !d_recv || !d_expert_count || !d_tile_expert || !d_src_info) return MOE_ERR_ARG;
+  if (p->cfg.T > 0 && (!d_x || !d_topk_idx || !d_slot_of)) return MOE_ERR_ARG;
+  if (misaligned(d_x) || misaligned(d_recv)) return MOE_ERR_ALIGN;
+  p->launches = 0;
+  return launch_dispatch(p, d_x, d_topk_idx, d_recv, d_expert_count, d_tile_expert, d_src_info, d_slot_of,
+                         (cudaStream_t)stream) ? MOE_ERR_CUDA : MOE_OK;
+}
+
+static int ffn_dispatch(moe_plan* p, const void* recv, const int* tile_expert, const void* wg, const void* wu,
+                        const void* wd, void* out_rows, cudaStream_t st) {
+  if (p->cfg.dtype == MOE_DTYPE_BF16 && p->cfg.ffn_kernel == 0)
+    return launch_ffn_tc(p, recv, tile_expert, wg, wu, wd, out_rows, st);
+  return launch_ffn_simt(p, recv, tile_expert, wg, wu, wd, out_rows, st);
+}
+
+int moe_expert_ffn(moe_plan_t* p, const void* d_recv, const int32_t* d_tile_expert, const void* d_wg,
+                   const void* d_wu, const void* d_wd, void* d_out_rows, void* stream) {
+  if (!p || !d_recv || !d_tile_expert || !d_wg || !d_wu || !d_wd || !d_out_rows) return MOE_ERR_ARG;
+  if (p->cfg.identity_experts) return MOE_ERR_ARG;
+  if (misaligned(d_recv) || misaligned(d_wg) || misaligned(d_wu) || misaligned(d_wd) || misaligned(d_out_rows))
+    return MOE_ERR_ALIGN;
+  p->launches = 0;
+  int rc = ffn_dispatch(p, d_recv, d_tile_expert, d_wg, d_wu, d_wd, d_out_rows, (cudaStream_t)stream);
+  return rc == 0 ? MOE_OK : (rc < 0 ? rc : MOE_ERR_CUDA);
+}
+
+int moe_combine(moe_plan_t* p, const void* d_rows, const int32_t* d_slot_of, const float* d_topk_w, void* d_y,
+                void* stream) {
+  if (!p) return MOE_ERR_ARG;
+  if (p->cfg.T > 0 && (!d_rows || !d_slot_of || !d_topk_w || !d_y)) return MOE_ERR_ARG;
+  if (misaligned(d_rows) || misaligned(d_y)) return MOE_ERR_ALIGN;
+  p->launches = 0;
+  return launch_combine(p, d_rows, d_slot_of, d_topk_w, d_y, (cudaStream_t)stream) ? MOE_ERR_CUDA : MOE_OK;
+}
+
+int moe_layer(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_bias, const void* d_wg,
+              const void* d_wu, const void* d_wd, void* d_y, void* stream) {
+  if (!p || !d_wr) return MOE_ERR_ARG;
+  if (p->cfg.T > 0 && (!d_x || !d_y)) return MOE_ERR_ARG;
+  if (!p->cfg.identity_experts && (!d_wg || !d_wu || !d_wd)) return MOE_ERR_ARG;
+  if (misaligned(d_x) || misaligned(d_wr) || misaligned(d_wg) || misaligned(d_wu) || misaligned(d_wd) ||
+      misaligned(d_y))
+    return MOE_ERR_ALIGN;
+  cudaStream_t st = (cudaStream_t)stream;
+  Scratch& s = p->s;
+  p->launches = 0;
+  if (launch_route(p, d_x, d_wr, d_bias, s.topk_idx, s.topk_w, st)) return MOE_ERR_CUDA;
+  if (launch_dispatch(p, d_x, s.topk_idx, s.recv, s.expert_count, s.tile_expert, s.src_info, s.slot_of, st))
+    return MOE_ERR_CUDA;
+  if (!p->cfg.identity_experts) {
+    int rc = ffn_dispatch(p, s.recv, s.tile_expert, d_wg, d_wu, d_wd, s.out_rows, st);
+    if (rc != 0) return rc < 0 ? rc : MOE_ERR_CUDA;
+  }
+  if (launch_combine(p, s.out_rows, s.slot_of, s.topk_w, d_y, st)) return MOE_ERR_CUDA;
+  return MOE_OK;
+}
+
+int moe_layer_host(moe_plan_t* p, const void* h_x, const void* d_wr, const float* d_bias, const void* d_wg,
+                   const void* d_wu, const void* d_wd, void* h_y, void* stream) {
+  if (!p) return MOE_ERR_ARG;
+  if (p->cfg.T > 0 && (!h_x || !h_y)) return MOE_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t bytes = (size_t)p->cfg.T * p->cfg.H * (p->cfg.dtype == MOE_DTYPE_BF16 ? 2 : 4);
+  if (bytes && cudaMemcpyAsync(p->s.x_stage, h_x, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  int rc = moe_layer(p, p->s.x_stage, d_wr, d_bias, d_wg, d_wu, d_wd, p->s.y_stage, stream);
+  if (rc != MOE_OK) return rc;
+  if (bytes && cudaMemcpyAsync(h_y, p->s.y_stage, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  return cudaStreamSynchronize(st) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+int moe_layer_buffer(moe_plan_t* p, int which, void** out_ptr) {
+  if (!p || !out_ptr) return MOE_ERR_ARG;
+  Scratch& s = p->s;
+  void* tab[8] = {s.topk_idx, s.topk_w, s.recv, s.expert_count, s.tile_expert, s.src_info, s.slot_of, s.out_rows};
+  if (which < 0 || which >= 8) return MOE_ERR_ARG;
+  *out_ptr = tab[which];
+  return MOE_OK;
+}
+
+int moe_last_launch_count(moe_plan_t* p, int32_t* out) {
+  if (!p || !out) return MOE_ERR_ARG;
+  *out = p->launches;
+  return MOE_OK;
+}
+
+int moe_last_status(moe_plan_t* p, void* stream, int32_t* code, int32_t* detail) {
+  if (!p || !code) return MOE_ERR_ARG;
+  int host[2] = {0, 0};
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemcpyAsync(host, p->s.status, sizeof host, cudaMemcpyDeviceToHost, st) != cudaSuccess) return MOE_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ERR_CUDA;
+  *code = host[0];
+  if (detail) *detail = host[1];
+  return MOE_OK;
+}
+
+const char* moe_strerror(int code) {
+  switch (code) {
+    case MOE_OK: return "ok";
+    case MOE_ERR_ARG: return "bad argument";
+    case MOE_ERR_ALIGN: return "row pitch or pointer not 16-byte aligned";
+    case MOE_ERR_UNSUPPORTED: return "configuration outside what the kernels cover";
+    case MOE_ERR_CUDA: return "CUDA call failed";
+    case MOE_ERR_OVERFLOW: return "receive region overflow";
+    case MOE_ERR_TIMEOUT: return "bounded device-side wait ran out";
+    case MOE_ERR_WORKSPACE: return "workspace too small or misaligned";
+    default: return "unknown error";
+  }
+}
+
+}  // extern "C"

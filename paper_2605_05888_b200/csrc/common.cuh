@@ -1,0 +1,136 @@
+// Shared declarations of the sm_100a MoE hot path: the plan, the launchers each .cu file
+// exports to api.cu, and small device helpers.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/moehub.h"
+
+namespace moehub {
+
+constexpr int kTileRows = MOE_TILE_ROWS;
+
+// Device status word: [0] code, [1] detail.  First error wins.
+struct Status {
+  int code;
+  int detail;
+  int pad[2];
+};
+
+__device__ __forceinline__ void set_status(int* status, int code, int detail) {
+  if (atomicCAS(status, 0, code) == 0) status[1] = detail;
+}
+
+// Wait sites reported in the detail word of MOE_ERR_TIMEOUT.
+enum WaitSite { kWaitTileTable = 1, kWaitScanTicket = 2, kWaitMbarTma = 3, kWaitMbarMma = 4,
+                kWaitMbarEpi = 5, kWaitMbarTmemFree = 6 };
+
+struct Scratch {          // device pointers carved out of the caller's workspace
+  int* status;            // [4]
+  int* pool_next;         // [1]   paged mode: next free tile
+  int* scan_ticket;       // [1]   mode 0: CTAs of the scan kernel that finished
+  int* tile_table;        // [E * tiles_per_expert] paged mode: expert-local tile -> pool tile
+  int* cta_count;         // [nblk * E] mode 0: per token-block histogram
+  int* cta_base;          // [nblk * E] mode 0: exclusive prefix inside the expert
+  int* tile_base;         // [E + 1]    mode 0: first pool tile of each expert
+  int* tile_list;         // [P]   used tiles grouped by expert (FFN work list)
+  int* expert_start;      // [E + 1] first work-list index of each expert
+  void* inter;            // [P*128, F] SwiGLU intermediate
+  // moe_layer's internal buffers
+  int* topk_idx;
+  float* topk_w;
+  void* recv;
+  void* out_rows;
+  int* expert_count;
+  int* tile_expert;
+  int* src_info;
+  int* slot_of;
+  void* x_stage;          // [T,H] device copy of host x (moe_layer_host)
+  void* y_stage;          // [T,H]
+};
+
+}  // namespace moehub
+
+struct moe_plan {
+  moe_config_t cfg;
+  int64_t P;                 // pool tiles
+  int64_t cap_rows;          // mode 1: rows per expert
+  int tiles_per_expert;      // paged tile-table width
+  int dispatch_tokens;       // tokens per dispatch CTA
+  int nblk;                  // dispatch CTAs
+  int device;
+  int sm_count;
+  int launches;
+  size_t counters_bytes;     // leading part of the workspace cleared by dispatch
+  moehub::Scratch s;
+  void* encode_tiled;        // cuTensorMapEncodeTiled entry point (driver API), looked up once
+};
+
+namespace moehub {
+
+// ---- launchers (defined in the other .cu files); each returns a cudaError_t as int ------------
+int launch_route(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
+                 float* topk_w, cudaStream_t st);
+int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv, int* expert_count,
+                    int* tile_expert, int* src_info, int* slot_of, cudaStream_t st);
+int launch_combine(moe_plan* p, const void* rows, const int* slot_of, const float* topk_w, void* y,
+                   cudaStream_t st);
+int launch_ffn_simt(moe_plan* p, const void* recv, const int* tile_expert, const void* wg,
+                    const void* wu, const void* wd, void* out_rows, cudaStream_t st);
+int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const void* wg,
+                  const void* wu, const void* wd, void* out_rows, cudaStream_t st);
+
+// ---- element helpers ---------------------------------------------------------------------------
+__device__ __forceinline__ float to_float(float v) { return v; }
+__device__ __forceinline__ float to_float(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_float(float v);
+template <> __device__ __forceinline__ float from_float<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float v) {
+  return __float2bfloat16_rn(v);
+}
+
+// Unpack one 16-byte vector of T into floats (4 for fp32, 8 for bf16).
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+  static constexpr int N = 4;
+  __device__ static __forceinline__ void unpack(const uint4& v, float* f) {
+    f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+    f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+  }
+  __device__ static __forceinline__ uint4 pack(const float* f) {
+    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]),
+                      __float_as_uint(f[3]));
+  }
+};
+template <> struct Vec16<__nv_bfloat16> {
+  static constexpr int N = 8;
+  __device__ static __forceinline__ void unpack(const uint4& v, float* f) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      f[2 * i] = __uint_as_float(w[i] << 16);
+      f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+  __device__ static __forceinline__ uint4 pack(const float* f) {
+    uint32_t w[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      __nv_bfloat162 h = __floats2bfloat162_rn(f[2 * i], f[2 * i + 1]);
+      w[i] = *reinterpret_cast<uint32_t*>(&h);
+    }
+    return make_uint4(w[0], w[1], w[2], w[3]);
+  }
+};
+
+__device__ __forceinline__ int ld_acquire(const int* p) {
+  int v;
+  asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(int* p, int v) {
+  asm volatile("st.release.gpu.global.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+}  // namespace moehub

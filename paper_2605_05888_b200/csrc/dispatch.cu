@@ -1,0 +1,307 @@
+// Step 2 of the MoE layer (paper Section II-A, dispatch) with both address-resolution schemes.
+//
+// Mode 0, the conventional software mediation (Section III-A): per token-block histogram ->
+// exclusive scan over (expert, block) and over experts (tile-padded) -> stable scatter.  Three
+// kernels, and no row moves before every count is known.  The layout is the canonical one: an
+// expert's rows are in (token, k) order.
+//
+// Modes 1/2, destination-agnostic (Section IV-A/IV-B): one kernel.  As soon as a token block
+// knows its expert ids it takes rows from the experts' row pointers with one aggregated atomicAdd
+// per touched expert (the software stand-in of the allocation pointer table's self-incrementing
+// RowPointer) and stores each row at Base + LocalRowID*RowSize.  Mode 1 gives every expert a
+// static region (the paper's conservative pre-allocation); mode 2 pages 128-row tiles out of one
+// pool on demand (the paging-style manager the paper allows behind rowspMalloc): the block whose
+// rows open a new tile takes it from the pool and publishes it in the expert's tile table, the
+// others look it up with a bounded wait.
+//
+// Row movement is the same in every mode: one warp per token reads the row once with 16-byte
+// vectors (several in flight per lane) and stores it to its K slots; the slot indices are staged
+// in shared memory first so the copy loop has no dependent index loads.
+#include "common.cuh"
+
+namespace moehub {
+
+constexpr int kDispThreads = 256;
+constexpr int kMaxAssign = 256;  // assignments (token,k pairs) per CTA
+
+// ------------------------------------------------------------------------------------------------
+// Row copy: warp `warp` of the CTA copies token rows tl = warp, warp+8, ... to their K slots.
+template <int UNROLL>
+__device__ __forceinline__ void copy_rows(const uint4* __restrict__ x, uint4* __restrict__ recv,
+                                          const int* s_slot, int t0, int ntok, int K, int vec_per_row) {
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  for (int tl = warp; tl < ntok; tl += kDispThreads / 32) {
+    const uint4* src = x + (size_t)(t0 + tl) * vec_per_row;
+    const int* slots = s_slot + tl * K;
+    for (int v0 = 0; v0 < vec_per_row; v0 += 32 * UNROLL) {
+      uint4 r[UNROLL];
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        const int v = v0 + u * 32 + lane;
+        if (v < vec_per_row) r[u] = __ldg(src + v);
+      }
+      for (int k = 0; k < K; ++k) {
+        const int slot = slots[k];
+        if (slot < 0) continue;
+        uint4* dst = recv + (size_t)slot * vec_per_row;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+          const int v = v0 + u * 32 + lane;
+          if (v < vec_per_row) __stcs(dst + v, r[u]);
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Mode 0, kernel 1: histogram of one token block.  cta_count[blk][e].
+__global__ void __launch_bounds__(kDispThreads)
+hist_kernel(const int* __restrict__ topk_idx, int T, int E, int K, int tok_per_blk,
+            int* __restrict__ cta_count) {
+  extern __shared__ int s_cnt[];  // [E]
+  for (int e = threadIdx.x; e < E; e += kDispThreads) s_cnt[e] = 0;
+  __syncthreads();
+  const int t0 = blockIdx.x * tok_per_blk;
+  const int na = min(tok_per_blk, T - t0) * K;
+  for (int a = threadIdx.x; a < na; a += kDispThreads) atomicAdd(&s_cnt[topk_idx[(size_t)t0 * K + a]], 1);
+  __syncthreads();
+  for (int e = threadIdx.x; e < E; e += kDispThreads) cta_count[(size_t)blockIdx.x * E + e] = s_cnt[e];
+}
+
+// Mode 0, kernel 2: CTA e scans expert e's per-block counts (exclusive) -> cta_base[blk][e] and
+// expert_count[e]; the last CTA to finish scans ceil(count/128) over the experts -> tile_base,
+// tile_expert.
+__global__ void __launch_bounds__(kDispThreads)
+scan_kernel(const int* __restrict__ cta_count, int nblk, int E, int P, int* __restrict__ cta_base,
+            int* __restrict__ expert_count, int* __restrict__ tile_base, int* __restrict__ tile_expert,
+            int* __restrict__ ticket) {
+  __shared__ int s_warp[kDispThreads / 32];
+  __shared__ int s_carry;
+  __shared__ int s_last;
+  const int e = blockIdx.x;
+  const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+  if (threadIdx.x == 0) s_carry = 0;
+  __syncthreads();
+  for (int b0 = 0; b0 < nblk; b0 += kDispThreads) {
+    const int b = b0 + threadIdx.x;
+    const int c = (b < nblk) ? cta_count[(size_t)b * E + e] : 0;
+    int incl = c;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += n;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    int wbase = 0;
+    for (int w = 0; w < warp; ++w) wbase += s_warp[w];
+    const int carry = s_carry;
+    if (b < nblk) cta_base[(size_t)b * E + e] = carry + wbase + incl - c;
+    __syncthreads();
+    if (threadIdx.x == kDispThreads - 1) s_carry = carry + wbase + incl;
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) {
+    expert_count[e] = s_carry;
+    __threadfence();
+    s_last = (atomicAdd(ticket, 1) == E - 1);
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  // Exclusive scan of tiles-per-expert over the experts (E <= 256: one element per thread).
+  int tiles = 0;
+  if (threadIdx.x < E) tiles = (ld_acquire(&expert_count[threadIdx.x]) + kTileRows - 1) / kTileRows;
+  int incl = tiles;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += n;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  int wbase = 0;
+  for (int w = 0; w < warp; ++w) wbase += s_warp[w];
+  const int first = wbase + incl - tiles;
+  if (threadIdx.x < E) {
+    tile_base[threadIdx.x] = first;
+    for (int i = 0; i < tiles; ++i)
+      if (first + i < P) tile_expert[first + i] = threadIdx.x;
+  }
+  if (threadIdx.x == E - 1) tile_base[E] = first + tiles;
+}
+
+// Mode 0, kernel 3: stable scatter.  The rank of an assignment inside its block is the number of
+// earlier assignments (in (token,k) order) of the same expert.
+__global__ void __launch_bounds__(kDispThreads)
+scatter_kernel(const uint4* __restrict__ x, const int* __restrict__ topk_idx, int T, int E, int K,
+               int tok_per_blk, int vec_per_row, const int* __restrict__ cta_base,
+               const int* __restrict__ tile_base, uint4* __restrict__ recv, int* __restrict__ src_info,
+               int* __restrict__ slot_of) {
+  extern __shared__ int smem_i[];
+  int* s_wcnt = smem_i;                          // [8][E] per-warp counts
+  int* s_slot = smem_i + (kDispThreads / 32) * E;  // [kMaxAssign]
+  const int t0 = blockIdx.x * tok_per_blk;
+  const int ntok = min(tok_per_blk, T - t0);
+  const int na = ntok * K;
+  const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+  for (int i = threadIdx.x; i < (kDispThreads / 32) * E; i += kDispThreads) s_wcnt[i] = 0;
+  __syncthreads();
+  const int a = threadIdx.x;  // one assignment per thread, na <= 256
+  int e = -1, wrank = 0;
+  if (a < na) e = topk_idx[(size_t)t0 * K + a];
+  {
+    const unsigned peers = __match_any_sync(0xffffffffu, e);
+    wrank = __popc(peers & ((1u << lane) - 1u));
+    if (e >= 0 && wrank == 0) s_wcnt[warp * E + e] = __popc(peers);
+  }
+  __syncthreads();
+  if (a < na) {
+    int before = 0;
+    for (int w = 0; w < warp; ++w) before += s_wcnt[w * E + e];
+    const int slot = tile_base[e] * kTileRows + cta_base[(size_t)blockIdx.x * E + e] + before + wrank;
+    s_slot[a] = slot;
+    slot_of[(size_t)t0 * K + a] = slot;
+    src_info[slot] = t0 * K + a;
+  }
+  __syncthreads();
+  copy_rows<4>(x, recv, s_slot, t0, ntok, K, vec_per_row);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Modes 1/2: destination-agnostic dispatch in one kernel.
+template <bool PAGED>
+__global__ void __launch_bounds__(kDispThreads)
+dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk_idx, int T, int E, int K,
+                       int tok_per_blk, int vec_per_row, int cap_rows, int P, int tiles_per_expert,
+                       unsigned long long spin_limit, int* __restrict__ row_pointer,
+                       int* __restrict__ tile_table, int* __restrict__ pool_next,
+                       int* __restrict__ tile_expert, uint4* __restrict__ recv, int* __restrict__ src_info,
+                       int* __restrict__ slot_of, int* __restrict__ status) {
+  extern __shared__ int smem_i[];
+  int* s_cnt = smem_i;        // [E] rows this block sends to expert e
+  int* s_base = smem_i + E;   // [E] first LocalRowID this block got from expert e's row pointer
+  int* s_slot = smem_i + 2 * E;  // [kMaxAssign] physical row per assignment
+  const int t0 = blockIdx.x * tok_per_blk;
+  const int ntok = min(tok_per_blk, T - t0);
+  const int na = ntok * K;
+  const int lane = threadIdx.x % 32;
+  for (int e = threadIdx.x; e < E; e += kDispThreads) s_cnt[e] = 0;
+  __syncthreads();
+
+  // (a) rank inside the block: warp-aggregated shared-memory atomics
+  const int a = threadIdx.x;
+  int e = -1, lrank = 0;
+  if (a < na) e = topk_idx[(size_t)t0 * K + a];
+  {
+    const unsigned peers = __match_any_sync(0xffffffffu, e);
+    const int leader = __ffs(peers) - 1;
+    int base = 0;
+    if (e >= 0 && lane == leader) base = atomicAdd(&s_cnt[e], __popc(peers));
+    base = __shfl_sync(0xffffffffu, base, leader);
+    lrank = base + __popc(peers & ((1u << lane) - 1u));
+  }
+  __syncthreads();
+
+  // (b) one global atomicAdd per touched expert: the block's rows get LocalRowIDs
+  //     [base, base+n).  The block whose range opens a tile (a multiple of 128) claims it.
+  for (int ee = threadIdx.x; ee < E; ee += kDispThreads) {
+    const int n = s_cnt[ee];
+    if (n == 0) continue;
+    const int base = atomicAdd(&row_pointer[ee], n);
+    s_base[ee] = base;
+    const int first_tile = (base + kTileRows - 1) / kTileRows;  // tiles whose row 0 lies in [base, base+n)
+    const int last_tile = (base + n - 1) / kTileRows;
+    for (int lt = first_tile; lt <= last_tile; ++lt) {
+      if (PAGED) {
+        if (lt >= tiles_per_expert) { set_status(status, MOE_ERR_OVERFLOW, ee); continue; }
+        const int tile = atomicAdd(pool_next, 1);
+        if (tile >= P) { set_status(status, MOE_ERR_OVERFLOW, ee); continue; }
+        tile_expert[tile] = ee;
+        st_release(&tile_table[(size_t)ee * tiles_per_expert + lt], tile);
+      } else {
+        if ((lt + 1) * kTileRows <= cap_rows) tile_expert[ee * (cap_rows / kTileRows) + lt] = ee;
+      }
+    }
+  }
+  __syncthreads();
+
+  // (c) LocalRowID -> physical row (address = Base + LocalRowID*RowSize), staged in shared memory
+  if (a < na) {
+    const int local_row = s_base[e] + lrank;
+    int slot = -1;
+    if (PAGED) {
+      const int lt = local_row / kTileRows;
+      if (lt < tiles_per_expert) {
+        const int* entry = &tile_table[(size_t)e * tiles_per_expert + lt];
+        int tile = ld_acquire(entry);
+        unsigned long long spins = 0;
+        while (tile < 0) {  // bounded wait for the block that opened this tile
+          if (ld_acquire(status) != 0 || ++spins > spin_limit) {
+            set_status(status, MOE_ERR_TIMEOUT, kWaitTileTable);
+            break;
+          }
+          __nanosleep(32);
+          tile = ld_acquire(entry);
+        }
+        if (tile >= 0) slot = tile * kTileRows + local_row % kTileRows;
+      }
+    } else {
+      if (local_row < cap_rows) slot = e * cap_rows + local_row;
+      else set_status(status, MOE_ERR_OVERFLOW, e);
+    }
+    s_slot[a] = slot;
+    slot_of[(size_t)t0 * K + a] = slot;
+    if (slot >= 0) src_info[slot] = t0 * K + a;  // the row's source information
+  }
+  __syncthreads();
+  copy_rows<4>(x, recv, s_slot, t0, ntok, K, vec_per_row);
+}
+
+// ------------------------------------------------------------------------------------------------
+int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv, int* expert_count,
+                    int* tile_expert, int* src_info, int* slot_of, cudaStream_t st) {
+  const moe_config_t& c = p->cfg;
+  const int eb = c.dtype == MOE_DTYPE_BF16 ? 2 : 4;
+  const int vec_per_row = c.H * eb / 16;
+  cudaError_t err;
+  // Per-call reset: scratch counters and tables, the caller's counters, owner and source arrays.
+  if ((err = cudaMemsetAsync(p->s.status, 0, p->counters_bytes, st)) != cudaSuccess) return (int)err;
+  if (c.dispatch_mode == MOE_DISPATCH_ATOMIC_PAGED) {
+    if ((err = cudaMemsetAsync(p->s.tile_table, 0xff, sizeof(int) * (size_t)c.E * p->tiles_per_expert, st)) != cudaSuccess)
+      return (int)err;
+  }
+  if ((err = cudaMemsetAsync(expert_count, 0, sizeof(int) * c.E, st)) != cudaSuccess) return (int)err;
+  if ((err = cudaMemsetAsync(tile_expert, 0xff, sizeof(int) * p->P, st)) != cudaSuccess) return (int)err;
+  if ((err = cudaMemsetAsync(src_info, 0xff, sizeof(int) * p->P * kTileRows, st)) != cudaSuccess) return (int)err;
+  if (c.T == 0) return 0;
+  const int nblk = p->nblk, tpb = p->dispatch_tokens;
+  if (c.dispatch_mode == MOE_DISPATCH_SCAN) {
+    hist_kernel<<<nblk, kDispThreads, sizeof(int) * c.E, st>>>(topk_idx, c.T, c.E, c.K, tpb, p->s.cta_count);
+    scan_kernel<<<c.E, kDispThreads, 0, st>>>(p->s.cta_count, nblk, c.E, (int)p->P, p->s.cta_base, expert_count,
+                                              p->s.tile_base, tile_expert, p->s.scan_ticket);
+    const size_t smem = sizeof(int) * ((kDispThreads / 32) * c.E + kMaxAssign);
+    scatter_kernel<<<nblk, kDispThreads, smem, st>>>((const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row,
+                                                     p->s.cta_base, p->s.tile_base, (uint4*)recv, src_info,
+                                                     slot_of);
+    p->launches += 3;
+  } else {
+    const size_t smem = sizeof(int) * (2 * c.E + kMaxAssign);
+    const unsigned long long spin = c.spin_limit ? c.spin_limit : (1ull << 22);
+    if (c.dispatch_mode == MOE_DISPATCH_ATOMIC_PAGED)
+      dispatch_atomic_kernel<true><<<nblk, kDispThreads, smem, st>>>(
+          (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row, (int)p->cap_rows, (int)p->P,
+          p->tiles_per_expert, spin, expert_count, p->s.tile_table, p->s.pool_next, tile_expert, (uint4*)recv,
+          src_info, slot_of, p->s.status);
+    else
+      dispatch_atomic_kernel<false><<<nblk, kDispThreads, smem, st>>>(
+          (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row, (int)p->cap_rows, (int)p->P,
+          p->tiles_per_expert, spin, expert_count, p->s.tile_table, p->s.pool_next, tile_expert, (uint4*)recv,
+          src_info, slot_of, p->s.status);
+    p->launches += 1;
+  }
+  return (int)cudaGetLastError();
+}
+
+}  // namespace moehub

@@ -1,0 +1,436 @@
+// Step 3 of the MoE layer (paper Section II-A, expert computation: two GEMMs with an activation
+// between) for bf16 on the 5th-generation tensor cores: a persistent, warp-specialised grouped
+// GEMM.  Operands are staged in shared memory by TMA (128-byte swizzle), tcgen05.mma accumulates
+// 128 x 256 fp32 tiles in tensor memory, and the epilogue warps read them back with tcgen05.ld.
+//
+// The unit of work is what the paper's dependency table calls a thread-block group: one 128-row
+// tile of one expert's receive region times one block of output columns (Section IV-D, static
+// tiling).  Tiles nobody wrote to are not in the work list, so their experts' weights are never
+// touched (the "counters that stay zero are never scheduled" rule of Section IV-D).
+//
+//   GEMM1 (SWIGLU): D[128, 256] = A[128, H] * [Wg[e, f0:f0+128, :] ; Wu[e, f0:f0+128, :]]^T
+//                   inter[:, f0:f0+128] = bf16( silu(D[:, 0:128]) * D[:, 128:256] )
+//   GEMM2         : D[128, 256] = inter[128, F] * Wd[e, h0:h0+256, :]^T ; out = bf16(D)
+//
+// Work order is expert-major, then column block, then tile, so that CTAs running at the same time
+// share the weight block through L2 and an expert's rows stay L2-resident across its column blocks.
+//
+// Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (owns the TMEM allocation),
+// warps 2-5 = epilogue (TMEM lane quarter = warp % 4).  Every mbarrier wait is bounded in time;
+// on expiry the CTA records MOE_ERR_TIMEOUT, drains its outstanding TMA copies (bounded), frees
+// its TMEM and returns.
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace moehub {
+
+constexpr int kTcThreads = 192;
+constexpr int kStages = 4;
+constexpr int kBK = 64;                       // k elements per stage (128 bytes of bf16)
+constexpr int kUmmaN = 256;
+constexpr int kABytes = kTileRows * kBK * 2;  // 16 KB
+constexpr int kBBytes = kUmmaN * kBK * 2;     // 32 KB
+constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kTcSmem = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr unsigned long long kWaitNs = 2000000000ull;  // 2 s bound on any single wait
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the time limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer();
+  for (unsigned it = 1;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 31u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer() - t0 > kWaitNs) return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) in the
+// 128-byte swizzle: 8-row groups are 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr >> 4) & 0x3fff);   // start address, 16-byte units
+  d |= (uint64_t)1 << 16;                  // leading byte offset (unused with swizzle, K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;        // stride byte offset between 8-row groups
+  d |= (uint64_t)1 << 46;                  // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                  // 128-byte swizzle
+  return d;
+}
+// Instruction descriptor: bf16 x bf16 -> fp32, A and B K-major, M = 128, N = 256.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kUmmaN >> 3) << 17) |
+                            ((uint32_t)(kTileRows >> 4) << 24);
+
+// ---- work list ------------------------------------------------------------------------------
+// tile_list: the used tiles grouped by expert; expert_start[e]: first index of expert e's tiles,
+// expert_start[E] = number of used tiles.
+__global__ void __launch_bounds__(256)
+worklist_kernel(const int* __restrict__ tile_expert, int P, int E, int* __restrict__ tile_list,
+                int* __restrict__ expert_start) {
+  __shared__ int s_cnt[256];
+  __shared__ int s_cur[256];
+  __shared__ int s_warp[8];
+  const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+  s_cnt[threadIdx.x] = 0;
+  __syncthreads();
+  for (int p = threadIdx.x; p < P; p += 256) {
+    const int e = tile_expert[p];
+    if (e >= 0 && e < E) atomicAdd(&s_cnt[e], 1);
+  }
+  __syncthreads();
+  const int c = s_cnt[threadIdx.x];
+  int incl = c;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int n = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += n;
+  }
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  int wbase = 0;
+  for (int w = 0; w < warp; ++w) wbase += s_warp[w];
+  const int first = wbase + incl - c;
+  s_cur[threadIdx.x] = first;
+  if (threadIdx.x < E) expert_start[threadIdx.x] = first;
+  if (threadIdx.x == E - 1) expert_start[E] = first + c;
+  __syncthreads();
+  for (int p = threadIdx.x; p < P; p += 256) {
+    const int e = tile_expert[p];
+    if (e >= 0 && e < E) tile_list[atomicAdd(&s_cur[e], 1)] = p;
+  }
+}
+
+// ---- the grouped GEMM -----------------------------------------------------------------------
+struct TcShared {
+  unsigned long long full[kStages];
+  unsigned long long empty[kStages];
+  unsigned long long tmem_full[2];
+  unsigned long long tmem_empty[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+template <bool SWIGLU>
+__global__ void __launch_bounds__(kTcThreads, 1)
+ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b1,
+              const __grid_constant__ CUtensorMap map_b2, const int* __restrict__ tile_list,
+              const int* __restrict__ expert_start, int E, int N, int Kd, __nv_bfloat16* __restrict__ C, int ldc,
+              int* __restrict__ status) {
+  constexpr int BN = SWIGLU ? 128 : 256;  // output columns per work item
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* stage_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  TcShared* sh = reinterpret_cast<TcShared*>(stage_base + kStages * kStageBytes);
+  __shared__ int s_start[257];
+
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  for (int i = threadIdx.x; i <= E; i += kTcThreads) s_start[i] = expert_start[i];
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(smem_u32(&sh->full[s]), 1);
+      mbar_init(smem_u32(&sh->empty[s]), 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      mbar_init(smem_u32(&sh->tmem_full[a]), 1);
+      mbar_init(smem_u32(&sh->tmem_empty[a]), 4);
+    }
+    sh->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // the MMA warp owns all 512 TMEM columns: two 128 x 256 fp32 accumulators
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
+                 "r"(512u) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = sh->tmem_base;
+  volatile int* abort_flag = &sh->abort_flag;
+
+  const int NB = (N + BN - 1) / BN;
+  const int KB = (Kd + kBK - 1) / kBK;
+  const int total_items = s_start[E] * NB;
+
+  // item -> (expert, column block, tile): expert-major, column-block-major, tile-minor
+  auto decode = [&](int item, int& e, int& nb, int& tile) {
+    int lo = 0, hi = E;  // largest e with s_start[e] * NB <= item
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) / 2;
+      if (s_start[mid] * NB <= item) lo = mid; else hi = mid;
+    }
+    e = lo;
+    const int m = s_start[e + 1] - s_start[e];
+    const int local = item - s_start[e] * NB;
+    nb = local / m;
+    tile = tile_list[s_start[e] + local % m];
+  };
+
+  int fail_site = 0;
+  if (warp == 0) {
+    // ===================== TMA producer =====================
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int armed[kStages];
+#pragma unroll
+      for (int s = 0; s < kStages; ++s) armed[s] = 0;
+      for (int item = blockIdx.x; item < total_items && !fail_site; item += gridDim.x) {
+        int e, nb, tile;
+        decode(item, e, nb, tile);
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, abort_flag)) { fail_site = kWaitMbarTma; break; }
+          const uint32_t full = smem_u32(&sh->full[stage]);
+          const uint32_t a_dst = smem_u32(stage_base + stage * kStageBytes);
+          const uint32_t b_dst = a_dst + kABytes;
+          mbar_expect_tx(full, kStageBytes);
+          tma_load_2d(a_dst, &map_a, full, kb * kBK, tile * kTileRows);
+          if (SWIGLU) {
+            tma_load_3d(b_dst, &map_b1, full, kb * kBK, nb * BN, e);
+            tma_load_3d(b_dst + kBBytes / 2, &map_b2, full, kb * kBK, nb * BN, e);
+          } else {
+            tma_load_3d(b_dst, &map_b1, full, kb * kBK, nb * BN, e);
+          }
+#pragma unroll
+          for (int s = 0; s < kStages; ++s)
+            if (s == stage) armed[s] += 1;
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (fail_site || *abort_flag) {
+        // Leave no copy in flight: wait (bounded) for the last fill of every stage.
+        sh->abort_flag = 1;
+#pragma unroll
+        for (int s = 0; s < kStages; ++s) {
+          if (armed[s] == 0) continue;
+          const uint32_t par = (uint32_t)((armed[s] - 1) & 1);
+          const unsigned long long t0 = globaltimer();
+          while (!mbar_try(smem_u32(&sh->full[s]), par))
+            if (globaltimer() - t0 > kWaitNs) break;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      int local_item = 0;
+      for (int item = blockIdx.x; item < total_items && !fail_site; item += gridDim.x, ++local_item) {
+        const int acc = local_item & 1;
+        const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
+        if (!mbar_wait(smem_u32(&sh->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) { fail_site = kWaitMbarTmemFree; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kUmmaN);
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!mbar_wait(smem_u32(&sh->full[stage]), phase, abort_flag)) { fail_site = kWaitMbarMma; break; }
+          tc_fence_after();
+          const uint32_t a_addr = smem_u32(stage_base + stage * kStageBytes);
+          const uint64_t adesc = smem_desc_sw128(a_addr);
+          const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
+#pragma unroll
+          for (int k = 0; k < kBK / 16; ++k)  // 16 k-elements = 32 bytes = 2 descriptor units per step
+            tc_mma(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
+          tc_commit(smem_u32(&sh->empty[stage]));  // the stage is free once these MMAs have read it
+          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (fail_site) break;
+        tc_commit(smem_u32(&sh->tmem_full[acc]));  // accumulator complete
+      }
+      if (fail_site) sh->abort_flag = 1;
+    }
+  } else {
+    // ===================== epilogue =====================
+    const int quarter = warp & 3;                 // TMEM lanes this warp may read
+    const int row_in_tile = quarter * 32 + lane;
+    int local_item = 0;
+    for (int item = blockIdx.x; item < total_items && !fail_site; item += gridDim.x, ++local_item) {
+      int e, nb, tile;
+      decode(item, e, nb, tile);
+      const int acc = local_item & 1;
+      const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
+      if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag)) { fail_site = kWaitMbarEpi; break; }
+      tc_fence_after();
+      const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kUmmaN);
+      __nv_bfloat16* out = C + ((size_t)tile * kTileRows + row_in_tile) * ldc + (size_t)nb * BN;
+      const int ncols = min(BN, N - nb * BN);
+      if (SWIGLU) {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 16) {
+          uint32_t g[16], u[16];
+          tc_ld16(t_row + c, g);
+          tc_ld16(t_row + 128 + c, u);
+          tc_wait_ld();
+          float s[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float gv = __uint_as_float(g[i]);
+            s[i] = gv / (1.0f + __expf(-gv)) * __uint_as_float(u[i]);
+          }
+          if (c + 8 <= ncols) *reinterpret_cast<uint4*>(out + c) = Vec16<__nv_bfloat16>::pack(s);
+          if (c + 16 <= ncols) *reinterpret_cast<uint4*>(out + c + 8) = Vec16<__nv_bfloat16>::pack(s + 8);
+        }
+      } else {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r0[16], r1[16];
+          tc_ld16(t_row + c, r0);
+          tc_ld16(t_row + c + 16, r1);
+          tc_wait_ld();
+          float f[32];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { f[i] = __uint_as_float(r0[i]); f[16 + i] = __uint_as_float(r1[i]); }
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            if (c + 8 * q + 8 <= ncols) *reinterpret_cast<uint4*>(out + c + 8 * q) = Vec16<__nv_bfloat16>::pack(f + 8 * q);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[acc]));
+    }
+    if (fail_site) sh->abort_flag = 1;
+  }
+  if (fail_site) set_status(status, MOE_ERR_TIMEOUT, fail_site);
+
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  if (warp == 1)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+}
+
+// ---- host side ------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static int get_encoder(moe_plan* p, EncodeTiledFn* fn) {
+  if (!p->encode_tiled) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess || !sym ||
+        q != cudaDriverEntryPointSuccess)
+      return MOE_ERR_CUDA;
+    p->encode_tiled = sym;
+  }
+  *fn = (EncodeTiledFn)p->encode_tiled;
+  return MOE_OK;
+}
+
+// bf16 matrix [rows, cols] (row-major, cols contiguous), box [box_rows, 64 cols], 128-byte swizzle.
+static int make_map_2d(EncodeTiledFn enc, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                       uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MOE_OK : MOE_ERR_CUDA;
+}
+// bf16 tensor [E, rows, cols], box [1, box_rows, 64].
+static int make_map_3d(EncodeTiledFn enc, CUtensorMap* m, const void* base, uint64_t E, uint64_t rows, uint64_t cols,
+                       uint32_t box_rows) {
+  cuuint64_t dims[3] = {cols, rows, E};
+  cuuint64_t strides[2] = {cols * 2, rows * cols * 2};
+  cuuint32_t box[3] = {(cuuint32_t)kBK, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MOE_OK : MOE_ERR_CUDA;
+}
+
+int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const void* wg, const void* wu,
+                  const void* wd, void* out_rows, cudaStream_t st) {
+  const moe_config_t& c = p->cfg;
+  if (p->P == 0 || c.T == 0) return 0;
+  EncodeTiledFn enc;
+  int rc = get_encoder(p, &enc);
+  if (rc != MOE_OK) return rc;
+  const uint64_t pool_rows = (uint64_t)p->P * kTileRows;
+  CUtensorMap a1, bg, bu, a2, bd;
+  if ((rc = make_map_2d(enc, &a1, recv, pool_rows, c.H, kTileRows)) != MOE_OK) return rc;
+  if ((rc = make_map_3d(enc, &bg, wg, c.E, c.F, c.H, 128)) != MOE_OK) return rc;
+  if ((rc = make_map_3d(enc, &bu, wu, c.E, c.F, c.H, 128)) != MOE_OK) return rc;
+  if ((rc = make_map_2d(enc, &a2, p->s.inter, pool_rows, c.F, kTileRows)) != MOE_OK) return rc;
+  if ((rc = make_map_3d(enc, &bd, wd, c.E, c.H, c.F, 256)) != MOE_OK) return rc;
+
+  static bool attr_done = false;  // per-process, idempotent
+  if (!attr_done) {
+    if (cudaFuncSetAttribute(ffn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(ffn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    attr_done = true;
+  }
+  worklist_kernel<<<1, 256, 0, st>>>(tile_expert, (int)p->P, c.E, p->s.tile_list, p->s.expert_start);
+  const int grid = p->sm_count;
+  ffn_tc_kernel<true><<<grid, kTcThreads, kTcSmem, st>>>(a1, bg, bu, p->s.tile_list, p->s.expert_start, c.E, c.F, c.H,
+                                                         (__nv_bfloat16*)p->s.inter, c.F, p->s.status);
+  ffn_tc_kernel<false><<<grid, kTcThreads, kTcSmem, st>>>(a2, bd, bd, p->s.tile_list, p->s.expert_start, c.E, c.H, c.F,
+                                                          (__nv_bfloat16*)out_rows, c.H, p->s.status);
+  p->launches += 3;
+  return cudaGetLastError() == cudaSuccess ? 0 : MOE_ERR_CUDA;
+}
+
+}  // namespace moehub

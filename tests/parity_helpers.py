@@ -1,0 +1,114 @@
+"""Shared plumbing of the GPU parity tests: upload host arrays, run the C-ABI stages, compare with
+the CPU oracle.  Nothing here computes any part of the method."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import oracle
+from paper_2605_05888_b200 import binding as B
+from paper_2605_05888_b200 import inputs
+
+TOL_Y = {inputs.FP32: 1e-4, inputs.BF16: 2e-2}
+
+
+def to_dev(a: np.ndarray | None, dtype: int | None = None):
+    """Host array -> device tensor. uint16 arrays with dtype==BF16 become bfloat16 tensors."""
+    if a is None:
+        return None
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if a.dtype == np.uint16:
+        t = t.view(torch.int16).cuda().view(torch.bfloat16)
+    else:
+        t = t.cuda()
+    return t
+
+
+def to_host_bits(t: torch.Tensor) -> np.ndarray:
+    """Device tensor -> host array in the oracle's storage convention (bf16 -> uint16 bits)."""
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).cpu().numpy().view(np.uint16)
+    return t.cpu().numpy()
+
+
+def to_host_f64(t: torch.Tensor) -> np.ndarray:
+    return t.to(torch.float64).cpu().numpy()
+
+
+def el_dtype(w: inputs.Workload):
+    return torch.bfloat16 if w.dtype == inputs.BF16 else torch.float32
+
+
+def make_plan(w: inputs.Workload, mode: int, **kw) -> B.Plan:
+    cfg = B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype, dispatch_mode=mode,
+                        identity_experts=int(w.identity_experts), **kw)
+    return B.Plan(cfg)
+
+
+def max_rel_err(got: np.ndarray, ref: np.ndarray) -> float:
+    """max_i |got_i - ref_i| / max(|ref_i|, rms(ref)): element-wise relative error with an rms floor."""
+    ref = ref.astype(np.float64)
+    got = got.astype(np.float64)
+    if ref.size == 0:
+        return 0.0
+    floor = float(np.sqrt(np.mean(ref * ref)))
+    denom = np.maximum(np.abs(ref), max(floor, 1e-30))
+    return float(np.max(np.abs(got - ref) / denom))
+
+
+def check_route(idx_gpu, w_gpu, idx_ref, w_ref):
+    idx_gpu, w_gpu = idx_gpu.cpu().numpy(), w_gpu.cpu().numpy()
+    bad = np.nonzero((idx_gpu != idx_ref).any(axis=1))[0]
+    assert bad.size == 0, f"{bad.size} tokens with wrong expert picks, first {bad[:5]}: gpu {idx_gpu[bad[:3]]} ref {idx_ref[bad[:3]]}"
+    err = np.abs(w_gpu.astype(np.float64) - w_ref) - (1e-5 * np.abs(w_ref) + 1e-7)
+    assert err.max(initial=-1.0) <= 0, f"routing weight off by {np.abs(w_gpu - w_ref).max()}"
+
+
+def check_dispatch(w: inputs.Workload, P: int, x_host, idx_ref, d_ref, recv, expert_count, tile_expert, src_info,
+                   slot_of, check_rows=True):
+    """Bit-exact comparison of a dispatch result with the oracle's, up to the order of rows inside an
+    expert (arrival order is free): every expert's rows are sorted by source id before comparing."""
+    T, K, E = w.T, w.K, w.E
+    cnt = expert_count.cpu().numpy()
+    te = tile_expert.cpu().numpy()
+    src = src_info.cpu().numpy()
+    slot = slot_of.cpu().numpy()
+    assert np.array_equal(cnt, d_ref["count"]), f"expert counts differ: {cnt} vs {d_ref['count']}"
+    assert cnt.sum() == T * K
+    # slot_of <-> src_info is a bijection on the T*K assignments
+    flat = slot.ravel()
+    assert flat.min(initial=0) >= 0 and flat.max(initial=0) < P * 128
+    assert np.unique(flat).size == T * K, "two assignments share a slot"
+    assert np.array_equal(src[flat], np.arange(T * K)), "src_info[slot_of[t,k]] != t*K+k"
+    assert (src >= 0).sum() == T * K, "src_info marks rows nobody wrote"
+    # every slot lies in a tile owned by the assignment's expert; tiles are dense
+    owner = te[flat // 128]
+    assert np.array_equal(owner, idx_ref.ravel()), "a row sits in a tile of the wrong expert"
+    used_tiles = np.unique(flat // 128)
+    assert np.array_equal(np.nonzero(te >= 0)[0], used_tiles), "tile_expert marks tiles without rows (or misses some)"
+    tiles_per_e = np.bincount(te[te >= 0], minlength=E)
+    assert np.array_equal(tiles_per_e, (cnt + 127) // 128), "an expert's rows are not densely packed into its tiles"
+    if not check_rows:
+        return
+    recv_h = to_host_bits(recv)
+    for e in range(E):
+        rows_e = np.nonzero(owner == e)[0]          # assignments of expert e in (t,k) order
+        got = recv_h[flat[rows_e]]                   # their rows, canonical order
+        ref = d_ref["recv"][d_ref["offset"][e]:d_ref["offset"][e + 1]]
+        assert got.shape == ref.shape and got.tobytes() == ref.tobytes(), f"expert {e}: receive rows differ"
+
+
+def oracle_inputs(w: inputs.Workload, with_experts=True):
+    x = inputs.make_x(w)
+    wr, bias = inputs.make_router(w)
+    if with_experts and not w.identity_experts:
+        wg, wu, wd = inputs.make_all_expert_weights(w)
+    else:
+        wg = wu = wd = None
+    return x, wr, bias, wg, wu, wd
+
+
+def oracle_layer_for(w: inputs.Workload, x, wr, bias, wg, wu, wd):
+    ws = (None, None, None) if wg is None else ([wg[e] for e in range(w.E)], [wu[e] for e in range(w.E)],
+                                                 [wd[e] for e in range(w.E)])
+    return oracle.layer(x, wr, bias, *ws, w.E, w.R, w.K, w.dtype, identity_experts=w.identity_experts)

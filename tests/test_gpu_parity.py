@@ -1,0 +1,211 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the CPU oracle on
+the same seeded inputs.  Routing indices and dispatch contents bit-exact (rows inside an expert
+compared after sorting by source id: arrival order is free, Section IV-B of the paper), routing
+weights within 1e-5 relative, combined output within 1e-4 (fp32) / 2e-2 (bf16) of the oracle under
+max_i |d_i| / max(|ref_i|, rms(ref))."""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2605_05888_b200 import binding as B
+from paper_2605_05888_b200 import inputs
+import parity_helpers as Hh
+
+pytestmark = pytest.mark.gpu
+FP32, BF16 = inputs.FP32, inputs.BF16
+MODES = [B.DISPATCH_SCAN, B.DISPATCH_ATOMIC_STATIC, B.DISPATCH_ATOMIC_PAGED]
+
+SMALL = [
+    inputs.C1,
+    inputs.C1.with_(seed=1), inputs.C1.with_(seed=2),
+    inputs.Workload("ragged_bf16", T=333, H=264, E=12, R=3, K=3, F=200, dtype=BF16),
+    inputs.Workload("qwen_small", T=97, H=512, E=60, R=4, K=4, F=352, dtype=BF16),
+    inputs.Workload("many_experts", T=300, H=256, E=256, R=32, K=8, F=128, dtype=BF16, zipf_s=1.0),
+    inputs.Workload("k_equals_e", T=50, H=64, E=4, R=2, K=4, F=64, dtype=FP32),
+    inputs.Workload("one_token", T=1, H=128, E=8, R=1, K=2, F=128, dtype=BF16),
+    inputs.Workload("top1", T=130, H=128, E=16, R=4, K=1, F=136, dtype=BF16, zipf_s=1.2),
+]
+
+
+def run_stages(w, mode, x, wr, bias, wg, wu, wd, ffn_kernel=0):
+    plan = Hh.make_plan(w, mode, ffn_kernel=ffn_kernel)
+    el = Hh.el_dtype(w)
+    dx, dwr, dbias = Hh.to_dev(x), Hh.to_dev(wr), Hh.to_dev(bias)
+    idx = torch.empty((w.T, w.K), dtype=torch.int32, device="cuda")
+    tw = torch.empty((w.T, w.K), dtype=torch.float32, device="cuda")
+    plan.moe_route(dx, dwr, dbias, idx, tw)
+    rows = plan.P * 128
+    recv = torch.zeros((rows, w.H), dtype=el, device="cuda")
+    cnt = torch.empty(w.E, dtype=torch.int32, device="cuda")
+    te = torch.empty(plan.P, dtype=torch.int32, device="cuda")
+    src = torch.empty(rows, dtype=torch.int32, device="cuda")
+    slot = torch.empty((w.T, w.K), dtype=torch.int32, device="cuda")
+    plan.moe_dispatch(dx, idx, recv, cnt, te, src, slot)
+    if w.identity_experts:
+        out_rows = recv
+    else:
+        out_rows = torch.zeros((rows, w.H), dtype=el, device="cuda")
+        plan.moe_expert_ffn(recv, te, Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd), out_rows)
+    y = torch.empty((w.T, w.H), dtype=el, device="cuda")
+    plan.moe_combine(out_rows, slot, tw, y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    return dict(plan=plan, idx=idx, tw=tw, recv=recv, cnt=cnt, te=te, src=src, slot=slot, out_rows=out_rows, y=y)
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("w", SMALL, ids=lambda w: w.name + f"_s{w.seed}")
+def test_stages_match_oracle(w, mode):
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    g = run_stages(w, mode, x, wr, bias, wg, wu, wd)
+    Hh.check_route(g["idx"], g["tw"], ref["topk_idx"], ref["topk_w"])
+    Hh.check_dispatch(w, g["plan"].P, x, ref["topk_idx"], ref, g["recv"], g["cnt"], g["te"], g["src"], g["slot"])
+    # expert outputs row by row (canonical order) and the combined result
+    slot = g["slot"].cpu().numpy()
+    got_rows = Hh.to_host_f64(g["out_rows"])[slot.ravel()]
+    ref_rows = ref["out_rows"][ref["slot_of"].ravel()]
+    assert Hh.max_rel_err(got_rows, ref_rows) <= Hh.TOL_Y[w.dtype], "expert outputs"
+    err = Hh.max_rel_err(Hh.to_host_f64(g["y"]), ref["y"])
+    assert err <= Hh.TOL_Y[w.dtype], f"combined output: max rel err {err}"
+
+
+@pytest.mark.parametrize("w", [SMALL[3], SMALL[4], SMALL[5]], ids=lambda w: w.name)
+def test_simt_ffn_matches_oracle_bf16(w):
+    """The fp32-FMA expert kernel on bf16 data: the second device implementation of step 3."""
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    g = run_stages(w, B.DISPATCH_SCAN, x, wr, bias, wg, wu, wd, ffn_kernel=1)
+    assert Hh.max_rel_err(Hh.to_host_f64(g["y"]), ref["y"]) <= Hh.TOL_Y[w.dtype]
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("w", [inputs.C1, SMALL[3], SMALL[5], inputs.C5(512), inputs.C5(256, 1.2)],
+                         ids=lambda w: w.name)
+def test_fused_layer_matches_oracle(w, mode):
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    plan = Hh.make_plan(w, mode)
+    y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
+    plan.moe_layer(Hh.to_dev(x), Hh.to_dev(wr), Hh.to_dev(bias), Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd), y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    assert plan.moe_last_launch_count() >= 3
+    Hh.check_route(plan.layer_tensor(0), plan.layer_tensor(1), ref["topk_idx"], ref["topk_w"])
+    Hh.check_dispatch(w, plan.P, x, ref["topk_idx"], ref, plan.layer_tensor(2), plan.layer_tensor(3),
+                      plan.layer_tensor(4), plan.layer_tensor(5), plan.layer_tensor(6))
+    err = Hh.max_rel_err(Hh.to_host_f64(y), ref["y"])
+    assert err <= Hh.TOL_Y[w.dtype], f"max rel err {err}"
+    # host-buffer entry point gives the same bytes
+    hx = torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
+    hy = torch.empty_like(hx).pin_memory()
+    plan.moe_layer_host(hx, Hh.to_dev(wr), Hh.to_dev(bias), Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd), hy)
+    y_bits = Hh.to_host_bits(y)
+    assert np.array_equal(hy.numpy().view(y_bits.dtype), y_bits)
+
+
+def test_identity_experts_closed_form():
+    """Identity experts make the layer return x * sum_k w (a property that holds at any size)."""
+    w = inputs.C5(2048, 1.2)
+    x, wr, bias, *_ = Hh.oracle_inputs(w, with_experts=False)
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED)
+    y = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+    dx = Hh.to_dev(x)
+    plan.moe_layer(dx, Hh.to_dev(wr), Hh.to_dev(bias), None, None, None, y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    ws = plan.layer_tensor(1).double().sum(1, keepdim=True)
+    ref = (dx.double() * ws).cpu().numpy()
+    assert Hh.max_rel_err(Hh.to_host_f64(y), ref) <= 2e-2
+
+
+# ------------------------------------------------------------------ router edge cases
+def test_router_tie_patterns_exhaustive():
+    """H = 8 >= E and Wr = [I | 0] make the logits equal x[:, :E]; x runs over {-1,0,1}^E, every tie
+    pattern of the top-K selection, K = 1..E."""
+    for E in (2, 3, 5):
+        grid = np.array(list(itertools.product([-1.0, 0.0, 1.0], repeat=E)), np.float32)
+        T = grid.shape[0]
+        x = np.zeros((T, 8), np.float32)
+        x[:, :E] = grid
+        wr = np.zeros((E, 8), np.float32)
+        wr[np.arange(E), np.arange(E)] = 1.0
+        for K in range(1, E + 1):
+            w = inputs.Workload("ties", T=T, H=8, E=E, R=1, K=K, F=8, dtype=FP32)
+            plan = Hh.make_plan(w, B.DISPATCH_SCAN)
+            idx = torch.empty((T, K), dtype=torch.int32, device="cuda")
+            tw = torch.empty((T, K), dtype=torch.float32, device="cuda")
+            plan.moe_route(Hh.to_dev(x), Hh.to_dev(wr), None, idx, tw)
+            ridx, rw, _ = oracle.route(x, wr, None, K, FP32)
+            Hh.check_route(idx, tw, ridx, rw)
+
+
+@pytest.mark.parametrize("renorm", [0, 1])
+def test_router_renormalize_and_bias(renorm):
+    w = inputs.Workload("renorm", T=200, H=512, E=60, R=4, K=4, F=8, dtype=BF16, zipf_s=1.0, seed=3)
+    x, wr, bias, *_ = Hh.oracle_inputs(w, with_experts=False)
+    cfg = B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype, renormalize=renorm)
+    plan = B.Plan(cfg)
+    idx = torch.empty((w.T, w.K), dtype=torch.int32, device="cuda")
+    tw = torch.empty((w.T, w.K), dtype=torch.float32, device="cuda")
+    plan.moe_route(Hh.to_dev(x), Hh.to_dev(wr), Hh.to_dev(bias), idx, tw)
+    ridx, rw, _ = oracle.route(x, wr, bias, w.K, w.dtype, renormalize=renorm)
+    Hh.check_route(idx, tw, ridx, rw)
+
+
+# ------------------------------------------------------------------ dispatch edge cases
+@pytest.mark.parametrize("mode", MODES)
+def test_dispatch_all_tokens_to_one_expert_and_empty_experts(mode):
+    w = inputs.Workload("skew", T=700, H=64, E=8, R=2, K=2, F=8, dtype=BF16)
+    x = inputs.make_x(w)
+    idx = np.zeros((w.T, w.K), np.int32)
+    idx[:, 0], idx[:, 1] = 5, 2           # experts 5 and 2 get T rows each, the others none
+    ref = oracle.dispatch(x, idx, w.E, w.R, w.dtype)
+    plan = Hh.make_plan(w, mode)
+    rows = plan.P * 128
+    recv = torch.zeros((rows, w.H), dtype=torch.bfloat16, device="cuda")
+    cnt = torch.empty(w.E, dtype=torch.int32, device="cuda")
+    te = torch.empty(plan.P, dtype=torch.int32, device="cuda")
+    src = torch.empty(rows, dtype=torch.int32, device="cuda")
+    slot = torch.empty((w.T, w.K), dtype=torch.int32, device="cuda")
+    plan.moe_dispatch(Hh.to_dev(x), Hh.to_dev(idx), recv, cnt, te, src, slot)
+    assert plan.moe_last_status() == (0, 0)
+    Hh.check_dispatch(w, plan.P, x, idx, ref, recv, cnt, te, src, slot)
+
+
+def test_static_region_overflow_is_reported_not_silent():
+    """Mode 1 with regions smaller than the load: the status word says overflow and names an expert,
+    counts stay exact, dropped assignments get slot -1, nothing is written out of bounds."""
+    w = inputs.Workload("overflow", T=600, H=64, E=4, R=1, K=1, F=8, dtype=BF16)
+    x = inputs.make_x(w)
+    idx = np.full((w.T, 1), 3, np.int32)
+    cfg = B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype, dispatch_mode=B.DISPATCH_ATOMIC_STATIC,
+                        capacity_rows=256)
+    plan = B.Plan(cfg)
+    rows = plan.P * 128
+    guard = torch.full((rows + 128, w.H), 7.0, dtype=torch.bfloat16, device="cuda")
+    cnt = torch.empty(w.E, dtype=torch.int32, device="cuda")
+    te = torch.empty(plan.P, dtype=torch.int32, device="cuda")
+    src = torch.empty(rows, dtype=torch.int32, device="cuda")
+    slot = torch.empty((w.T, w.K), dtype=torch.int32, device="cuda")
+    plan.moe_dispatch(Hh.to_dev(x), Hh.to_dev(idx), guard[:rows], cnt, te, src, slot)
+    code, detail = plan.moe_last_status()
+    assert code == -5 and detail == 3
+    assert cnt.cpu().tolist() == [0, 0, 0, 600]
+    s = slot.cpu().numpy().ravel()
+    assert (s >= 0).sum() == 256 and (s == -1).sum() == 600 - 256
+    assert torch.all(guard[rows:] == 7.0)
+
+
+def test_bad_arguments_are_refused_on_the_host():
+    cfg = B.make_config(16, 100, 8, 2, 2, 64, BF16)      # H*2 bytes not a multiple of 16
+    with pytest.raises(B.MoeError) as ei:
+        B.moe_workspace_bytes(cfg)
+    assert ei.value.code == -2
+    with pytest.raises(B.MoeError):
+        B.moe_workspace_bytes(B.make_config(16, 128, 8, 3, 2, 64, BF16))   # E % R != 0
+    with pytest.raises(B.MoeError):
+        B.moe_workspace_bytes(B.make_config(16, 128, 8, 2, 9, 64, BF16))   # K > E
