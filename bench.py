@@ -1,0 +1,330 @@
+#!/usr/bin/env python
+"""MoE-layer benchmark: tokens/s of the whole hot path (route -> dispatch -> expert FFN -> combine).
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA path
+    python bench.py --impl reference --steps K --warmup W    # the CPU oracle, bounded sample per step
+
+A step is one pass of the whole layer over one batch of seeded synthetic input.  At N > 1 (launched
+by torch.distributed.run, one process per GPU) every rank runs an independent replica on its own
+batch (the path does not shard: weak scaling, no data-path collective); the time is the max over
+ranks.  Rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+from paper_2605_05888_b200 import inputs  # noqa: E402
+
+METRIC = "MoE-layer tokens/s on 1 B200; dispatch+combine HBM GB/s and % of roofline"
+UNIT = "tokens/s"
+WORKLOADS = {"c1": inputs.C1, "c2": inputs.C2, "c3": inputs.C3, "c4": inputs.C4}
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
+# from the ncu capture summarised under profiles/; None until a capture exists for that workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def load_peaks() -> tuple[dict, str]:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+def workload_config(w: inputs.Workload, extra: dict) -> dict:
+    cfg = {"workload": w.name, "T": w.T, "H": w.H, "E": w.E, "R": w.R, "K": w.K, "F": w.F,
+           "router": "softmax top-K, zipf_s=%g" % w.zipf_s, "seed": w.seed}
+    cfg.update(extra)
+    return cfg
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs (the only places this file touches oracle/)
+def oracle_sample(w: inputs.Workload, n_tokens: int, x, wr, bias, wg, wu, wd) -> tuple[float, int]:
+    """Times the oracle layer on the first n_tokens tokens of the batch. Returns (seconds, threads)."""
+    import oracle
+    xs = np.ascontiguousarray(x[:n_tokens])
+    t0 = time.perf_counter()
+    if w.identity_experts:
+        oracle.layer(xs, wr, bias, None, None, None, w.E, w.R, w.K, w.dtype, identity_experts=True)
+    else:
+        oracle.layer(xs, wr, bias, list(wg), list(wu), list(wd), w.E, w.R, w.K, w.dtype)
+    return time.perf_counter() - t0, oracle.num_threads()
+
+
+def oracle_sample_tokens(w: inputs.Workload, threads: int) -> int:
+    """Tokens whose oracle layer costs roughly 10-20 s on `threads` cores at ~2.5 GFLOP/s per core."""
+    flop_per_token = 6.0 * w.K * w.H * max(w.F, 1) + 2.0 * w.H * w.E
+    n = int(15.0 * 2.5e9 * max(threads, 1) / flop_per_token)
+    return max(8, min(w.T, n))
+
+
+def run_reference(args, w: inputs.Workload) -> None:
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    x = inputs.make_x(w)
+    wr, bias = inputs.make_router(w)
+    wg, wu, wd = inputs.make_all_expert_weights(w) if not w.identity_experts else (None, None, None)
+    threads = oracle.num_threads()
+    # keep the whole run within a few minutes: (steps + warmup) samples of n tokens each
+    n = max(4, oracle_sample_tokens(w, threads) // max(1, (args.steps + args.warmup) // 2))
+    for _ in range(args.warmup):
+        oracle_sample(w, n, x, wr, bias, wg, wu, wd)
+    t = 0.0
+    for _ in range(args.steps):
+        dt, _ = oracle_sample(w, n, x, wr, bias, wg, wu, wd)
+        t += dt
+    value = n * args.steps / t
+    sample = f"first {n} of {w.T} tokens per step, whole layer (route, dispatch, experts, combine)"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(w, {"sample": sample}),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+                 getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+                 getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+                 getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+                 getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake"}
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                get = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or nv.nvmlDeviceGetCurrentClocksThrottleReasons
+                mask = get(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop_evt.wait(0.005)
+
+    def stop(self) -> dict:
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(1.0)
+        med = float(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def run_cuda(args, w: inputs.Workload) -> None:
+    import torch
+    import torch.distributed as dist
+
+    from paper_2605_05888_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the CUDA path has no CPU fallback (use --impl reference)")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    w = w.with_(seed=w.seed + rank)  # every rank its own batch
+
+    def dev(a):
+        if a is None:
+            return None
+        t = torch.from_numpy(a)
+        return t.view(torch.int16).cuda().view(torch.bfloat16) if a.dtype == np.uint16 else t.cuda()
+
+    x = inputs.make_x(w)
+    wr, bias = inputs.make_router(w)
+    if w.identity_experts:
+        wg = wu = wd = None
+    else:
+        wg, wu, wd = inputs.make_all_expert_weights(w.with_(seed=0))  # same parameters on every rank
+    dx, dwr, dbias, dwg, dwu, dwd = dev(x), dev(wr), dev(bias), dev(wg), dev(wu), dev(wd)
+    el = torch.bfloat16 if w.dtype == inputs.BF16 else torch.float32
+    mode = {"scan": B.DISPATCH_SCAN, "static": B.DISPATCH_ATOMIC_STATIC, "paged": B.DISPATCH_ATOMIC_PAGED}[args.dispatch]
+    plan = B.Plan(B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype, dispatch_mode=mode,
+                                identity_experts=int(w.identity_experts)))
+    y = torch.empty((w.T, w.H), dtype=el, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def step():
+        plan.moe_layer(dx, dwr, dbias, dwg, dwu, dwd, y)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    code, detail = plan.moe_last_status()
+    if code != 0:
+        raise SystemExit(f"bench.py: device status {code} ({B.strerror(code)}), detail {detail}")
+    launches_per_step = plan.moe_last_launch_count()
+
+    # ---- timed region: K steps, device-resident inputs ----
+    sampler = ClockSampler(local)
+    barrier()
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.stop()
+    barrier()
+
+    # ---- per-kernel device times: the same steps with an event after every kernel ----
+    stage_ms = np.zeros(len(B.STAGES))
+    for _ in range(args.steps):
+        stage_ms += np.array(plan.moe_layer_timed(dx, dwr, dbias, dwg, dwu, dwd, y))
+    stage_ms /= args.steps
+
+    # ---- end to end through the host-buffer entry point: H2D of x and D2H of y inside the timing ----
+    hx = torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
+    hy = torch.empty_like(hx).pin_memory()
+    for _ in range(3):
+        plan.moe_layer_host(hx, dwr, dbias, dwg, dwu, dwd, hy)
+    barrier()
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    f0.record(stream)
+    for _ in range(args.steps):
+        plan.moe_layer_host(hx, dwr, dbias, dwg, dwu, dwd, hy)
+    f1.record(stream)
+    torch.cuda.synchronize()
+    ms_e2e = f0.elapsed_time(f1)
+
+    if world > 1:
+        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e = t.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    eb = w.elem_bytes
+    rows = w.T * w.K
+    ms_step = ms_total / args.steps
+    value = world * w.T / (ms_step * 1e-3)
+
+    # algorithmic work per launch of each stage
+    disp_bytes = w.T * w.H * eb * (1 + w.K) + 12 * rows
+    comb_bytes = w.T * w.H * eb * (w.K + 1) + 8 * rows
+    route_bytes = w.T * w.H * eb + w.E * w.H * eb + 8 * rows
+    gemm1_flops = 4.0 * rows * w.H * w.F
+    gemm2_flops = 2.0 * rows * w.H * w.F
+    sm = dict(zip(B.STAGES, stage_ms.tolist()))
+    hbm_peak = peaks["hbm_gbs"]
+    stages = {
+        "route": {"ms": sm["route"], "GBps": route_bytes / sm["route"] / 1e6 if sm["route"] > 0 else None},
+        "dispatch": {"ms": sm["dispatch"], "GBps": disp_bytes / sm["dispatch"] / 1e6,
+                     "frac_hbm": disp_bytes / sm["dispatch"] / 1e6 / hbm_peak, "mode": args.dispatch},
+        "combine": {"ms": sm["combine"], "GBps": comb_bytes / sm["combine"] / 1e6,
+                    "frac_hbm": comb_bytes / sm["combine"] / 1e6 / hbm_peak},
+    }
+    if w.identity_experts or w.dtype != inputs.BF16:
+        dom = "dispatch"
+        roofline = {"kernel": "dispatch", "bound": "hbm", "achieved": stages["dispatch"]["GBps"], "peak": hbm_peak,
+                    "unit": "GB/s", "frac": stages["dispatch"]["frac_hbm"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                    "peak_source": f"{peak_kind} hbm_gbs"}
+    else:
+        t1, t2 = sm["gemm1"], sm["gemm2"]
+        stages["ffn_gemm1"] = {"ms": t1, "TFLOPs": gemm1_flops / t1 / 1e9}
+        stages["ffn_gemm2"] = {"ms": t2, "TFLOPs": gemm2_flops / t2 / 1e9}
+        stages["worklist"] = {"ms": sm["worklist"]}
+        tensor_peak = peaks["bf16_tflops"]
+        ach = gemm1_flops / t1 / 1e9
+        roofline = {"kernel": "ffn_tc_kernel<SWIGLU> (GEMM1 + SwiGLU epilogue)", "bound": "tensor", "achieved": ach,
+                    "peak": tensor_peak, "unit": "TFLOP/s", "frac": ach / tensor_peak,
+                    "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                    "peak_source": f"{peak_kind} bf16_tflops (burst)",
+                    "ffn_both_gemms_TFLOPs": (gemm1_flops + gemm2_flops) / (t1 + t2) / 1e9}
+
+    # the CPU oracle on a bounded sample of the same batch (N = 1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        n = oracle_sample_tokens(w, oracle.num_threads())
+        secs, threads = oracle_sample(w, n, x, wr, bias, wg, wu, wd)
+        cpu = {"value": n / secs, "unit": UNIT, "cores": threads, "kind": "oracle",
+               "sample": f"first {n} of {w.T} tokens, whole layer, {secs:.1f} s"}
+
+    h2d = w.T * w.H * eb
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if w.dtype == inputs.BF16 else "f32", "data": "synthetic",
+            "config": workload_config(w, {"dispatch_mode": args.dispatch, "parallelism": f"replicas x{world}",
+                                          "l2": "no flush: the per-step working set (weights + buffers, %.1f GB) "
+                                                "exceeds the 126 MB L2" % ((3 * w.E * w.F * w.H * eb + 4 * rows * w.H * eb) / 1e9)}),
+            "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
+            "e2e": {"value": world * w.T * args.steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": h2d, "api": "moe_layer_host (pinned host x and y)"},
+            "roofline": roofline, "cpu_baseline": cpu, "stages": stages, "dominant": roofline["kernel"]}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--dispatch", default="paged", choices=["scan", "static", "paged"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_cuda(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -141,6 +141,21 @@ int moe_layer(moe_plan_t* plan, const void* d_x, const void* d_wr, const float* 
 int moe_layer_host(moe_plan_t* plan, const void* h_x, const void* d_wr, const float* d_bias,
                    const void* d_wg, const void* d_wu, const void* d_wd, void* h_y, void* stream);
 
+/* moe_layer with a CUDA event recorded after every kernel: runs the layer once, synchronises the
+ * stream and writes the device time of each stage, in milliseconds, to h_stage_ms
+ * [MOE_STAGE_COUNT] (host): route, dispatch (all its kernels and counter resets), FFN work list,
+ * FFN GEMM1 (+SwiGLU), FFN GEMM2, combine.  For measurement only. */
+#define MOE_STAGE_ROUTE 0
+#define MOE_STAGE_DISPATCH 1
+#define MOE_STAGE_WORKLIST 2
+#define MOE_STAGE_GEMM1 3
+#define MOE_STAGE_GEMM2 4
+#define MOE_STAGE_COMBINE 5
+#define MOE_STAGE_COUNT 6
+int moe_layer_timed(moe_plan_t* plan, const void* d_x, const void* d_wr, const float* d_bias,
+                    const void* d_wg, const void* d_wu, const void* d_wd, void* d_y, void* stream,
+                    float* h_stage_ms);
+
 /* Device pointers of moe_layer's intermediate results inside the workspace (valid after a
  * moe_layer call completes): which = 0 topk_idx, 1 topk_w, 2 recv, 3 expert_count,
  * 4 tile_expert, 5 src_info, 6 slot_of, 7 out_rows. */

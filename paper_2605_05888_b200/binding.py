@@ -19,9 +19,10 @@ MOE_OK = 0
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 DISPATCH_SCAN, DISPATCH_ATOMIC_STATIC, DISPATCH_ATOMIC_PAGED = 0, 1, 2
 TILE_ROWS = 128
+STAGES = ["route", "dispatch", "worklist", "gemm1", "gemm2", "combine"]
 
 EXPORTS = ["moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
-           "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host", "moe_layer_buffer",
+           "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host", "moe_layer_timed", "moe_layer_buffer",
            "moe_last_launch_count", "moe_last_status", "moe_strerror"]
 
 
@@ -58,6 +59,7 @@ def lib() -> ctypes.CDLL:
         L.moe_combine.argtypes = [vp, vp, i32p, fp, vp, vp]
         L.moe_layer.argtypes = [vp] * 9
         L.moe_layer_host.argtypes = [vp] * 9
+        L.moe_layer_timed.argtypes = [vp] * 9 + [ctypes.POINTER(ctypes.c_float)]
         L.moe_layer_buffer.argtypes = [vp, ctypes.c_int, ctypes.POINTER(vp)]
         L.moe_last_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
         L.moe_last_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
@@ -162,6 +164,13 @@ class Plan:
         assert not h_x.is_cuda and not h_y.is_cuda
         _check(lib().moe_layer_host(self.handle, _ptr(h_x), _ptr(wr), _ptr(bias), _ptr(wg), _ptr(wu), _ptr(wd),
                                     _ptr(h_y), _stream(stream)), "moe_layer_host")
+
+    def moe_layer_timed(self, x, wr, bias, wg, wu, wd, y, stream=None) -> list[float]:
+        """Runs the layer once with an event after every kernel; returns ms per stage (see STAGES)."""
+        ms = (ctypes.c_float * len(STAGES))()
+        _check(lib().moe_layer_timed(self.handle, _ptr(x), _ptr(wr), _ptr(bias), _ptr(wg), _ptr(wu), _ptr(wd),
+                                     _ptr(y), _stream(stream), ms), "moe_layer_timed")
+        return list(ms)
 
     def moe_layer_buffer(self, which: int) -> int:
         out = ctypes.c_void_p()

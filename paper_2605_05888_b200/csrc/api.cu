@@ -132,6 +132,8 @@ int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, mo
   p->nblk = g.nblk;
   p->launches = 0;
   p->encode_tiled = nullptr;
+  p->timing = 0;
+  for (int i = 0; i <= MOE_STAGE_COUNT; ++i) p->tev[i] = nullptr;
   carve(*cfg, g, (char*)d_workspace, &p->s, &p->counters_bytes);
   if (cudaGetDevice(&p->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device) != cudaSuccess) {
@@ -148,6 +150,9 @@ int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, mo
 }
 
 int moe_plan_destroy(moe_plan_t* plan) {
+  if (plan)
+    for (int i = 0; i <= MOE_STAGE_COUNT; ++i)
+      if (plan->tev[i]) cudaEventDestroy(plan->tev[i]);
   delete plan;
   return MOE_OK;
 }
@@ -209,14 +214,37 @@ int moe_layer(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_b
   cudaStream_t st = (cudaStream_t)stream;
   Scratch& s = p->s;
   p->launches = 0;
+  mark(p, 0, st);
   if (launch_route(p, d_x, d_wr, d_bias, s.topk_idx, s.topk_w, st)) return MOE_ERR_CUDA;
+  mark(p, 1, st);
   if (launch_dispatch(p, d_x, s.topk_idx, s.recv, s.expert_count, s.tile_expert, s.src_info, s.slot_of, st))
     return MOE_ERR_CUDA;
+  mark(p, 2, st);
   if (!p->cfg.identity_experts) {
     int rc = ffn_dispatch(p, s.recv, s.tile_expert, d_wg, d_wu, d_wd, s.out_rows, st);
     if (rc != 0) return rc < 0 ? rc : MOE_ERR_CUDA;
+  } else {
+    mark(p, 3, st);
+    mark(p, 4, st);
   }
+  mark(p, 5, st);
   if (launch_combine(p, s.out_rows, s.slot_of, s.topk_w, d_y, st)) return MOE_ERR_CUDA;
+  mark(p, 6, st);
+  return MOE_OK;
+}
+
+int moe_layer_timed(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_bias, const void* d_wg,
+                    const void* d_wu, const void* d_wd, void* d_y, void* stream, float* h_stage_ms) {
+  if (!p || !h_stage_ms) return MOE_ERR_ARG;
+  for (int i = 0; i <= MOE_STAGE_COUNT; ++i)
+    if (!p->tev[i] && cudaEventCreate(&p->tev[i]) != cudaSuccess) return MOE_ERR_CUDA;
+  p->timing = 1;
+  int rc = moe_layer(p, d_x, d_wr, d_bias, d_wg, d_wu, d_wd, d_y, stream);
+  p->timing = 0;
+  if (rc != MOE_OK) return rc;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return MOE_ERR_CUDA;
+  for (int i = 0; i < MOE_STAGE_COUNT; ++i)
+    if (cudaEventElapsedTime(&h_stage_ms[i], p->tev[i], p->tev[i + 1]) != cudaSuccess) return MOE_ERR_CUDA;
   return MOE_OK;
 }
 

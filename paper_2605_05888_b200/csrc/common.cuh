@@ -65,9 +65,16 @@ struct moe_plan {
   size_t counters_bytes;     // leading part of the workspace cleared by dispatch
   moehub::Scratch s;
   void* encode_tiled;        // cuTensorMapEncodeTiled entry point (driver API), looked up once
+  int timing;                // moe_layer_timed: record an event after every kernel of the layer
+  cudaEvent_t tev[MOE_STAGE_COUNT + 1];
 };
 
 namespace moehub {
+
+// Timing marks of moe_layer_timed: mark i closes stage i-1.
+inline void mark(moe_plan* p, int i, cudaStream_t st) {
+  if (p->timing) cudaEventRecord(p->tev[i], st);
+}
 
 // ---- launchers (defined in the other .cu files); each returns a cudaError_t as int ------------
 int launch_route(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,

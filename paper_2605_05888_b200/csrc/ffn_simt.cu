@@ -90,9 +90,11 @@ static int launch_typed(moe_plan* p, const void* recv, const int* tile_expert, c
                         const void* wu, const void* wd, void* out_rows, cudaStream_t st) {
   const moe_config_t& c = p->cfg;
   const size_t stride = (size_t)c.F * c.H;
+  mark(p, 3, st);
   dim3 g1((c.F + kSimtBN - 1) / kSimtBN, (unsigned)p->P);
   ffn_simt_kernel<XT, true><<<g1, kSimtThreads, 0, st>>>((const XT*)recv, c.H, tile_expert, (const XT*)wg,
                                                          (const XT*)wu, stride, c.F, c.H, (XT*)p->s.inter, c.F);
+  mark(p, 4, st);
   dim3 g2((c.H + kSimtBN - 1) / kSimtBN, (unsigned)p->P);
   ffn_simt_kernel<XT, false><<<g2, kSimtThreads, 0, st>>>((const XT*)p->s.inter, c.F, tile_expert,
                                                           (const XT*)wd, nullptr, stride, c.H, c.F,

@@ -424,9 +424,11 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
     attr_done = true;
   }
   worklist_kernel<<<1, 256, 0, st>>>(tile_expert, (int)p->P, c.E, p->s.tile_list, p->s.expert_start);
+  mark(p, 3, st);
   const int grid = p->sm_count;
   ffn_tc_kernel<true><<<grid, kTcThreads, kTcSmem, st>>>(a1, bg, bu, p->s.tile_list, p->s.expert_start, c.E, c.F, c.H,
                                                          (__nv_bfloat16*)p->s.inter, c.F, p->s.status);
+  mark(p, 4, st);
   ffn_tc_kernel<false><<<grid, kTcThreads, kTcSmem, st>>>(a2, bd, bd, p->s.tile_list, p->s.expert_start, c.E, c.H, c.F,
                                                           (__nv_bfloat16*)out_rows, c.H, p->s.status);
   p->launches += 3;
