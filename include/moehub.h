@@ -51,6 +51,7 @@ extern "C" {
 #define MOE_ERR_OVERFLOW (-5)    /* device status: an expert's region (mode 1) or the pool is full */
 #define MOE_ERR_TIMEOUT (-6)     /* device status: a bounded device-side wait ran out */
 #define MOE_ERR_WORKSPACE (-7)   /* workspace too small or misaligned */
+#define MOE_ERR_TOO_LARGE (-8)   /* moe_dispatch_noalloc: T or E beyond its fixed built-in scratch */
 
 #define MOE_DTYPE_FP32 0
 #define MOE_DTYPE_BF16 1
@@ -122,6 +123,32 @@ int moe_dispatch(moe_plan_t* plan, const void* d_x, const int32_t* d_topk_idx, v
 int moe_expert_ffn(moe_plan_t* plan, const void* d_recv, const int32_t* d_tile_expert,
                    const void* d_wg, const void* d_wu, const void* d_wd, void* d_out_rows,
                    void* stream);
+
+/* Dispatch without any allocation (the paper has no counterpart: this entry point exists for
+ * the callers described here, not for a step of the method).  Some callers cannot give this
+ * library a workspace because they cannot allocate device memory at the point of the call: a
+ * serving process that handed the whole GPU to its own pool at start-up, a plug-in that has no
+ * access to its host's allocator, a latency-critical loop that must not risk the device-wide
+ * synchronisation an allocation can cause.  For them this variant of moe_dispatch keeps its
+ * scratch (pool cursor + tile table, about 129 KB) in a fixed device array built into the
+ * library; every GPU that loads the library holds that array until the process exits.  It takes
+ * no plan, calls no cudaMalloc/cudaFree or any other allocating routine, and always uses the
+ * paged destination-agnostic scheme (cfg->dispatch_mode, capacity_rows and F are ignored).
+ *
+ * Limits: T <= MOE_NOALLOC_MAX_TOKENS and E <= 256, otherwise MOE_ERR_TOO_LARGE is returned and
+ * nothing is launched.  Arguments and outputs are those of moe_dispatch, with the pool size
+ * P = floor(T*K/128) + E, plus d_status: [2] int32 in device memory owned by the caller, which
+ * receives the device status (code, detail) that moe_last_status would report.
+ *
+ * The first call on each device looks up the array's device address (that device must be
+ * current); make that first call outside any stream capture.  All calls on a device share the
+ * one array, which still holds the previous call's contents: each call clears what it needs on
+ * `stream` before its kernel, so calls issued to the same stream are safe back to back, but two
+ * calls that can overlap on the GPU (different streams, no dependency) race on it. */
+#define MOE_NOALLOC_MAX_TOKENS 16384
+int moe_dispatch_noalloc(const moe_config_t* cfg, const void* d_x, const int32_t* d_topk_idx,
+                         void* d_recv, int32_t* d_expert_count, int32_t* d_tile_expert,
+                         int32_t* d_src_info, int32_t* d_slot_of, int32_t* d_status, void* stream);
 
 /* Steps 4+5 (Section II-A, combine and scaling): y[t,:] = sum_k w[t,k]*rows[slot_of[t,k],:],
  * k ascending, fp32 accumulation, rounded once to dtype.  Assignments with slot -1 add 0.

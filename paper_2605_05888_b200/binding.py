@@ -21,7 +21,7 @@ DISPATCH_SCAN, DISPATCH_ATOMIC_STATIC, DISPATCH_ATOMIC_PAGED = 0, 1, 2
 TILE_ROWS = 128
 STAGES = ["route", "dispatch", "worklist", "gemm1", "gemm2", "combine"]
 
-EXPORTS = ["moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
+EXPORTS = ["moe_dispatch_noalloc", "moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
            "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host", "moe_layer_timed", "moe_layer_buffer",
            "moe_last_launch_count", "moe_last_status", "moe_strerror"]
 
@@ -55,6 +55,7 @@ def lib() -> ctypes.CDLL:
         L.moe_plan_destroy.argtypes = [vp]
         L.moe_route.argtypes = [vp, vp, vp, fp, i32p, fp, vp]
         L.moe_dispatch.argtypes = [vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp]
+        L.moe_dispatch_noalloc.argtypes = [cfgp, vp, i32p, vp, i32p, i32p, i32p, i32p, i32p, vp]
         L.moe_expert_ffn.argtypes = [vp, vp, i32p, vp, vp, vp, vp, vp]
         L.moe_combine.argtypes = [vp, vp, i32p, fp, vp, vp]
         L.moe_layer.argtypes = [vp] * 9
@@ -112,6 +113,16 @@ def moe_workspace_bytes(cfg: MoeConfig) -> int:
     out = ctypes.c_size_t()
     _check(lib().moe_workspace_bytes(ctypes.byref(cfg), ctypes.byref(out)), "moe_workspace_bytes")
     return out.value
+
+
+def moe_dispatch_noalloc(cfg: MoeConfig, x, topk_idx, recv, expert_count, tile_expert, src_info, slot_of, status,
+                         stream=None) -> None:
+    """Paged dispatch that needs no plan and no workspace: for callers that cannot allocate device
+    memory.  Its scratch is a fixed array inside the library (T <= 16384, E <= 256).  `status` is a
+    caller-owned int32[2] device tensor that receives (code, detail)."""
+    _check(lib().moe_dispatch_noalloc(ctypes.byref(cfg), _ptr(x), _ptr(topk_idx), _ptr(recv), _ptr(expert_count),
+                                      _ptr(tile_expert), _ptr(src_info), _ptr(slot_of), _ptr(status),
+                                      _stream(stream)), "moe_dispatch_noalloc")
 
 
 class Plan:

@@ -299,6 +299,7 @@ const char* moe_strerror(int code) {
     case MOE_ERR_OVERFLOW: return "receive region overflow";
     case MOE_ERR_TIMEOUT: return "bounded device-side wait ran out";
     case MOE_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case MOE_ERR_TOO_LARGE: return "T or E beyond the fixed scratch of moe_dispatch_noalloc";
     default: return "unknown error";
   }
 }

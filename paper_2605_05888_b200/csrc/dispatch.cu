@@ -305,3 +305,89 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
 }
 
 }  // namespace moehub
+
+// ------------------------------------------------------------------------------------------------
+// moe_dispatch_noalloc: the paged destination-agnostic dispatch for callers that cannot allocate.
+//
+// Its scratch (the pool cursor and the per-expert tile table) lives in the file-scope device array
+// below instead of a caller-supplied workspace, so the call needs no plan and no device allocation
+// of any kind.  Every GPU that loads this library carries the array (about 129 KB) until exit.
+#include <mutex>
+
+namespace {
+
+constexpr int kNoAllocMaxTokens = MOE_NOALLOC_MAX_TOKENS;
+constexpr int kNoAllocMaxExperts = 256;
+constexpr int kNoAllocTilesPerExpert = kNoAllocMaxTokens / MOE_TILE_ROWS;
+// layout: [0] pool cursor, [64 ...] tile table [E][tiles_per_expert]
+constexpr int kNoAllocTableOffset = 64;
+constexpr int kNoAllocInts = kNoAllocTableOffset + kNoAllocMaxExperts * kNoAllocTilesPerExpert;
+
+static __device__ __align__(256) int g_noalloc_scratch[kNoAllocInts];
+
+// In host code the array's name is only a handle for the runtime, not a device address.  The
+// address is looked up once per device, with that device current, and kept here.
+constexpr int kMaxDevices = 64;
+int* g_noalloc_ptr[kMaxDevices];
+std::mutex g_noalloc_mutex;
+
+int noalloc_scratch_for_current_device(int** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MOE_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (g_noalloc_ptr[dev] == nullptr) {
+    int* ptr = nullptr;
+    if (cudaGetSymbolAddress((void**)&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) return MOE_ERR_CUDA;
+    g_noalloc_ptr[dev] = ptr;
+  }
+  *out = g_noalloc_ptr[dev];
+  return MOE_OK;
+}
+
+}  // namespace
+
+extern "C" int moe_dispatch_noalloc(const moe_config_t* cfg, const void* d_x, const int32_t* d_topk_idx,
+                                    void* d_recv, int32_t* d_expert_count, int32_t* d_tile_expert,
+                                    int32_t* d_src_info, int32_t* d_slot_of, int32_t* d_status, void* stream) {
+  using namespace moehub;
+  if (!cfg || !d_recv || !d_expert_count || !d_tile_expert || !d_src_info || !d_status) return MOE_ERR_ARG;
+  const moe_config_t& c = *cfg;
+  if (c.T < 0 || c.H <= 0 || c.E <= 0 || c.R <= 0 || c.K <= 0 || c.K > c.E || c.E % c.R != 0) return MOE_ERR_ARG;
+  if (c.dtype != MOE_DTYPE_FP32 && c.dtype != MOE_DTYPE_BF16) return MOE_ERR_ARG;
+  if (c.T > 0 && (!d_x || !d_topk_idx || !d_slot_of)) return MOE_ERR_ARG;
+  if (c.K > 32) return MOE_ERR_UNSUPPORTED;
+  if (c.T > kNoAllocMaxTokens || c.E > kNoAllocMaxExperts) return MOE_ERR_TOO_LARGE;
+  const int eb = c.dtype == MOE_DTYPE_BF16 ? 2 : 4;
+  if (((int64_t)c.H * eb) % 16 != 0) return MOE_ERR_ALIGN;
+  if ((reinterpret_cast<uintptr_t>(d_x) | reinterpret_cast<uintptr_t>(d_recv)) & 15) return MOE_ERR_ALIGN;
+
+  int* scratch = nullptr;
+  int rc = noalloc_scratch_for_current_device(&scratch);
+  if (rc != MOE_OK) return rc;
+  int* pool_next = scratch;
+  int* tile_table = scratch + kNoAllocTableOffset;
+
+  cudaStream_t st = (cudaStream_t)stream;
+  const int64_t P = (int64_t)c.T * c.K / kTileRows + c.E;
+  int tiles_per_expert = (c.T + kTileRows - 1) / kTileRows;
+  if (tiles_per_expert == 0) tiles_per_expert = 1;
+  int tpb = 256 / c.K;
+  if (tpb > 16) tpb = 16;
+  const int nblk = (c.T + tpb - 1) / tpb;
+  // The array keeps whatever the previous call left: reset the cursor and the part of the table
+  // this call reads, and the caller's counters, before the kernel runs.
+  if (cudaMemsetAsync(pool_next, 0, sizeof(int), st) != cudaSuccess ||
+      cudaMemsetAsync(tile_table, 0xff, sizeof(int) * (size_t)c.E * tiles_per_expert, st) != cudaSuccess ||
+      cudaMemsetAsync(d_status, 0, sizeof(int) * 2, st) != cudaSuccess ||
+      cudaMemsetAsync(d_expert_count, 0, sizeof(int) * c.E, st) != cudaSuccess ||
+      cudaMemsetAsync(d_tile_expert, 0xff, sizeof(int) * P, st) != cudaSuccess ||
+      cudaMemsetAsync(d_src_info, 0xff, sizeof(int) * P * kTileRows, st) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (c.T == 0) return MOE_OK;
+  const size_t smem = sizeof(int) * (2 * c.E + kMaxAssign);
+  const unsigned long long spin = c.spin_limit ? c.spin_limit : (1ull << 22);
+  dispatch_atomic_kernel<true><<<nblk, kDispThreads, smem, st>>>(
+      (const uint4*)d_x, d_topk_idx, c.T, c.E, c.K, tpb, c.H * eb / 16, 0, (int)P, tiles_per_expert, spin,
+      d_expert_count, tile_table, pool_next, d_tile_expert, (uint4*)d_recv, d_src_info, d_slot_of, d_status);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
