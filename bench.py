@@ -28,7 +28,11 @@ from paper_2605_05888_b200 import inputs  # noqa: E402
 
 METRIC = "MoE-layer tokens/s on 1 B200; dispatch+combine HBM GB/s and % of roofline"
 UNIT = "tokens/s"
-WORKLOADS = {"c1": inputs.C1, "c2": inputs.C2, "c3": inputs.C3, "c4": inputs.C4}
+WORKLOADS = {"c1": inputs.C1, "c2": inputs.C2, "c3": inputs.C3, "c4": inputs.C4,
+             # a quarter-size C2 (same kernels, 0.7 GB of weights) for ncu captures that must stay small
+             "c2_small": inputs.C2.with_(name="mixtral_like_bf16_small", T=2048, E=4, R=4, F=7168),
+             # dispatch/combine-only sweep points (identity experts)
+             "c5_8192": inputs.C5(8192), "c5_8192_zipf": inputs.C5(8192, 1.2), "c5_2048": inputs.C5(2048)}
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
 # from the ncu capture summarised under profiles/; None until a capture exists for that workload.

@@ -45,7 +45,7 @@ def make_plan(w: inputs.Workload, mode: int, **kw) -> B.Plan:
     return B.Plan(cfg)
 
 
-def max_rel_err(got: np.ndarray, ref: np.ndarray) -> float:
+def elementwise_rel_err(got: np.ndarray, ref: np.ndarray) -> float:
     """max_i |got_i - ref_i| / max(|ref_i|, rms(ref)): element-wise relative error with an rms floor."""
     ref = ref.astype(np.float64)
     got = got.astype(np.float64)
@@ -54,6 +54,42 @@ def max_rel_err(got: np.ndarray, ref: np.ndarray) -> float:
     floor = float(np.sqrt(np.mean(ref * ref)))
     denom = np.maximum(np.abs(ref), max(floor, 1e-30))
     return float(np.max(np.abs(got - ref) / denom))
+
+
+def normwise_rel_err(got: np.ndarray, ref: np.ndarray) -> float:
+    """max over rows t of ||got_t - ref_t||_inf / ||ref_t||_inf: every token's output vector is judged
+    against its own scale (tokens are independent and their scales differ with sum_k w)."""
+    ref = ref.astype(np.float64).reshape(-1, ref.shape[-1])
+    got = got.astype(np.float64).reshape(ref.shape)
+    if ref.size == 0:
+        return 0.0
+    num = np.max(np.abs(got - ref), axis=1)
+    den = np.maximum(np.max(np.abs(ref), axis=1), 1e-30)
+    return float(np.max(num / den))
+
+
+# Tripwire on the element-wise error of bf16 results.  The exact bf16 pipeline itself (fp64 arithmetic,
+# rounded to bf16 only where the data is stored as bf16: SwiGLU intermediate, expert output, y) already
+# reaches 1.3-2.1 % under the element-wise measure at the DeepSeek-like shape, so that measure cannot be
+# held to 2e-2; it is kept as a coarse guard against single wrong elements.
+ELEMENTWISE_GUARD_BF16 = 5e-2
+
+
+def assert_output_close(got: np.ndarray, ref: np.ndarray, dtype: int, what: str = "output") -> None:
+    """The pass/fail rule for floating-point outputs.
+    fp32: element-wise relative error (rms floor) <= 1e-4.
+    bf16: per-token normwise relative error <= 2e-2, and the element-wise error under the guard."""
+    ew = elementwise_rel_err(got, ref)
+    nw = normwise_rel_err(got, ref)
+    if dtype == inputs.FP32:
+        assert ew <= TOL_Y[dtype], f"{what}: element-wise rel err {ew:.3e} > {TOL_Y[dtype]}"
+    else:
+        assert nw <= TOL_Y[dtype], f"{what}: normwise rel err {nw:.3e} > {TOL_Y[dtype]} (element-wise {ew:.3e})"
+        assert ew <= ELEMENTWISE_GUARD_BF16, f"{what}: element-wise rel err {ew:.3e} > guard"
+
+
+def max_rel_err(got: np.ndarray, ref: np.ndarray) -> float:
+    return elementwise_rel_err(got, ref)
 
 
 def check_route(idx_gpu, w_gpu, idx_ref, w_ref):

@@ -1,8 +1,8 @@
 """GPU parity: every stage of the CUDA path, called through the C ABI, against the CPU oracle on
 the same seeded inputs.  Routing indices and dispatch contents bit-exact (rows inside an expert
 compared after sorting by source id: arrival order is free, Section IV-B of the paper), routing
-weights within 1e-5 relative, combined output within 1e-4 (fp32) / 2e-2 (bf16) of the oracle under
-max_i |d_i| / max(|ref_i|, rms(ref))."""
+weights within 1e-5 relative, combined output within 1e-4 (fp32, element-wise with an rms floor) /
+2e-2 (bf16, per-token normwise) of the oracle: see parity_helpers.assert_output_close."""
 import itertools
 
 import numpy as np
@@ -68,9 +68,8 @@ def test_stages_match_oracle(w, mode):
     slot = g["slot"].cpu().numpy()
     got_rows = Hh.to_host_f64(g["out_rows"])[slot.ravel()]
     ref_rows = ref["out_rows"][ref["slot_of"].ravel()]
-    assert Hh.max_rel_err(got_rows, ref_rows) <= Hh.TOL_Y[w.dtype], "expert outputs"
-    err = Hh.max_rel_err(Hh.to_host_f64(g["y"]), ref["y"])
-    assert err <= Hh.TOL_Y[w.dtype], f"combined output: max rel err {err}"
+    Hh.assert_output_close(got_rows, ref_rows, w.dtype, "expert outputs")
+    Hh.assert_output_close(Hh.to_host_f64(g["y"]), ref["y"], w.dtype, "combined output")
 
 
 @pytest.mark.parametrize("w", [SMALL[3], SMALL[4], SMALL[5]], ids=lambda w: w.name)
@@ -79,7 +78,7 @@ def test_simt_ffn_matches_oracle_bf16(w):
     x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
     ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
     g = run_stages(w, B.DISPATCH_SCAN, x, wr, bias, wg, wu, wd, ffn_kernel=1)
-    assert Hh.max_rel_err(Hh.to_host_f64(g["y"]), ref["y"]) <= Hh.TOL_Y[w.dtype]
+    Hh.assert_output_close(Hh.to_host_f64(g["y"]), ref["y"], w.dtype)
 
 
 @pytest.mark.parametrize("mode", MODES)
@@ -97,8 +96,7 @@ def test_fused_layer_matches_oracle(w, mode):
     Hh.check_route(plan.layer_tensor(0), plan.layer_tensor(1), ref["topk_idx"], ref["topk_w"])
     Hh.check_dispatch(w, plan.P, x, ref["topk_idx"], ref, plan.layer_tensor(2), plan.layer_tensor(3),
                       plan.layer_tensor(4), plan.layer_tensor(5), plan.layer_tensor(6))
-    err = Hh.max_rel_err(Hh.to_host_f64(y), ref["y"])
-    assert err <= Hh.TOL_Y[w.dtype], f"max rel err {err}"
+    Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
     # host-buffer entry point gives the same bytes
     hx = torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
     hy = torch.empty_like(hx).pin_memory()
@@ -119,7 +117,7 @@ def test_identity_experts_closed_form():
     assert plan.moe_last_status() == (0, 0)
     ws = plan.layer_tensor(1).double().sum(1, keepdim=True)
     ref = (dx.double() * ws).cpu().numpy()
-    assert Hh.max_rel_err(Hh.to_host_f64(y), ref) <= 2e-2
+    Hh.assert_output_close(Hh.to_host_f64(y), ref, w.dtype)
 
 
 # ------------------------------------------------------------------ router edge cases
