@@ -153,6 +153,22 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples)}
 
 
+def max_over_ranks(values: list[float], device: str = "cpu") -> list[float]:
+    """Element-wise max of per-rank timings over the default process group (identity when single-process)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(values)
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Replicas: every rank processes tokens_per_rank tokens per step; time is the max over ranks."""
+    return world * tokens_per_rank / (ms_per_step * 1e-3)
+
+
 def run_cuda(args, w: inputs.Workload) -> None:
     import torch
     import torch.distributed as dist
@@ -240,10 +256,7 @@ def run_cuda(args, w: inputs.Workload) -> None:
     torch.cuda.synchronize()
     ms_e2e = f0.elapsed_time(f1)
 
-    if world > 1:
-        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = t.tolist()
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], "cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -253,7 +266,7 @@ def run_cuda(args, w: inputs.Workload) -> None:
     eb = w.elem_bytes
     rows = w.T * w.K
     ms_step = ms_total / args.steps
-    value = world * w.T / (ms_step * 1e-3)
+    value = whole_job_tokens_per_s(w.T, world, ms_step)
 
     # algorithmic work per launch of each stage
     disp_bytes = w.T * w.H * eb * (1 + w.K) + 12 * rows
@@ -305,7 +318,7 @@ def run_cuda(args, w: inputs.Workload) -> None:
                                           "l2": "no flush: the per-step working set (weights + buffers, %.1f GB) "
                                                 "exceeds the 126 MB L2" % ((3 * w.E * w.F * w.H * eb + 4 * rows * w.H * eb) / 1e9)}),
             "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
-            "e2e": {"value": world * w.T * args.steps / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "e2e": {"value": whole_job_tokens_per_s(w.T, world, ms_e2e / args.steps), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": h2d, "api": "moe_layer_host (pinned host x and y)"},
             "roofline": roofline, "cpu_baseline": cpu, "stages": stages, "dominant": roofline["kernel"]}
     print(json.dumps(line), flush=True)
