@@ -72,7 +72,8 @@ typedef struct {
   int32_t identity_experts;     /* 1: moe_layer skips the FFN (expert output = expert input)  */
   int32_t ffn_kernel;           /* 0: tensor-core (tcgen05) kernel for bf16, SIMT for fp32;
                                    1: SIMT fp32-FMA kernel for either dtype (check path)      */
-  int32_t reserved;
+  int32_t ffn_split;            /* 0: both expert GEMMs in one persistent launch (per-tile status
+                                   counters gate GEMM2); 1: one launch per GEMM                 */
   int64_t capacity_rows;        /* mode 1: rows per expert region, multiple of 128, 0 = T
                                    rounded up (overflow-free); modes 0/2: ignored            */
   uint64_t spin_limit;          /* bound on every device-side wait, 0 = default (1<<22)      */

@@ -30,7 +30,7 @@ class MoeConfig(ctypes.Structure):
     _fields_ = [("T", ctypes.c_int32), ("H", ctypes.c_int32), ("E", ctypes.c_int32), ("R", ctypes.c_int32),
                 ("K", ctypes.c_int32), ("F", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("renormalize", ctypes.c_int32), ("dispatch_mode", ctypes.c_int32),
-                ("identity_experts", ctypes.c_int32), ("ffn_kernel", ctypes.c_int32), ("reserved", ctypes.c_int32),
+                ("identity_experts", ctypes.c_int32), ("ffn_kernel", ctypes.c_int32), ("ffn_split", ctypes.c_int32),
                 ("capacity_rows", ctypes.c_int64), ("spin_limit", ctypes.c_uint64)]
 
 
@@ -98,8 +98,8 @@ def _stream(stream) -> int:
 
 
 def make_config(T, H, E, R, K, F, dtype, renormalize=0, dispatch_mode=DISPATCH_ATOMIC_PAGED, identity_experts=0,
-                ffn_kernel=0, capacity_rows=0, spin_limit=0) -> MoeConfig:
-    return MoeConfig(T, H, E, R, K, F, dtype, int(renormalize), dispatch_mode, int(identity_experts), ffn_kernel, 0,
+                ffn_kernel=0, capacity_rows=0, spin_limit=0, ffn_split=0) -> MoeConfig:
+    return MoeConfig(T, H, E, R, K, F, dtype, int(renormalize), dispatch_mode, int(identity_experts), ffn_kernel, int(ffn_split),
                      capacity_rows, spin_limit)
 
 

@@ -2,25 +2,31 @@
 // K rows its experts produced (their positions were recorded at dispatch time, the "source
 // information" of Section IV-B) and forms y[t,:] = sum_k w[t,k] * rows[slot_of[t,k],:].
 //
-// HBM-bound gather-reduce: one warp per token; for every 16-byte column chunk the K row loads
-// are issued together, the sum runs in fp32 in ascending k (so the result is deterministic),
-// and is rounded once to the storage type.
+// HBM-bound gather-reduce.  A warp owns a run of 64 consecutive 16-byte column chunks of one token
+// (so a token is spread over several warps and small batches still fill the GPU); lanes 0..K-1 fetch
+// the token's slots and weights once and broadcast them by shuffle; for every chunk the K row loads
+// are issued together, the sum runs in fp32 in ascending k (so the result is deterministic), and is
+// rounded once to the storage type.
 #include "common.cuh"
 
 namespace moehub {
 
 constexpr int kCombThreads = 256;
+constexpr int kCombRun = 64;  // 16-byte chunks per warp: two per lane
 
 template <typename XT, int KT>  // KT > 0: K known at compile time; KT == 0: runtime K (<= 32)
 __global__ void __launch_bounds__(kCombThreads)
 combine_kernel(const uint4* __restrict__ rows, const int* __restrict__ slot_of,
-               const float* __restrict__ topk_w, int T, int K_rt, int vec_per_row, uint4* __restrict__ y) {
+               const float* __restrict__ topk_w, int T, int K_rt, int vec_per_row, int runs_per_row,
+               uint4* __restrict__ y) {
   constexpr int N = Vec16<XT>::N;
+  constexpr int KMAX = KT > 0 ? KT : 1;
   const int K = KT > 0 ? KT : K_rt;
   const int lane = threadIdx.x % 32;
-  const int t = blockIdx.x * (kCombThreads / 32) + threadIdx.x / 32;
+  const long long wid = (long long)blockIdx.x * (kCombThreads / 32) + threadIdx.x / 32;
+  const int t = (int)(wid / runs_per_row);
   if (t >= T) return;
-  // lane k holds slot/weight k; broadcast by shuffle in the loop
+  const int v_begin = (int)(wid % runs_per_row) * kCombRun;
   int my_slot = -1;
   float my_w = 0.0f;
   if (lane < K) {
@@ -28,48 +34,57 @@ combine_kernel(const uint4* __restrict__ rows, const int* __restrict__ slot_of,
     my_w = topk_w[(size_t)t * K + lane];
   }
   uint4* dst = y + (size_t)t * vec_per_row;
+  const int v0 = v_begin + lane, v1 = v_begin + 32 + lane;
+  const bool ok0 = v0 < vec_per_row, ok1 = v1 < vec_per_row;
   if (KT > 0) {
-    const uint4* src[KT > 0 ? KT : 1];
-    float w[KT > 0 ? KT : 1];
+    uint4 r0[KMAX], r1[KMAX];
+    float w[KMAX];
 #pragma unroll
     for (int k = 0; k < KT; ++k) {
       const int s = __shfl_sync(0xffffffffu, my_slot, k);
       w[k] = __shfl_sync(0xffffffffu, my_w, k);
-      src[k] = s >= 0 ? rows + (size_t)s * vec_per_row : nullptr;
+      const uint4* src = rows + (size_t)(s >= 0 ? s : 0) * vec_per_row;
+      r0[k] = (s >= 0 && ok0) ? __ldcs(src + v0) : make_uint4(0, 0, 0, 0);
+      r1[k] = (s >= 0 && ok1) ? __ldcs(src + v1) : make_uint4(0, 0, 0, 0);
     }
-    for (int v = lane; v < vec_per_row; v += 32) {
-      uint4 r[KT > 0 ? KT : 1];
+    float a0[N], a1[N];
 #pragma unroll
-      for (int k = 0; k < KT; ++k) r[k] = src[k] ? __ldcs(src[k] + v) : make_uint4(0, 0, 0, 0);
-      float acc[N];
+    for (int q = 0; q < N; ++q) a0[q] = a1[q] = 0.0f;
 #pragma unroll
-      for (int q = 0; q < N; ++q) acc[q] = 0.0f;
+    for (int k = 0; k < KT; ++k) {
+      float f[N];
+      Vec16<XT>::unpack(r0[k], f);
 #pragma unroll
-      for (int k = 0; k < KT; ++k) {
-        float f[N];
-        Vec16<XT>::unpack(r[k], f);
+      for (int q = 0; q < N; ++q) a0[q] = __fmaf_rn(w[k], f[q], a0[q]);
+      Vec16<XT>::unpack(r1[k], f);
 #pragma unroll
-        for (int q = 0; q < N; ++q) acc[q] = __fmaf_rn(w[k], f[q], acc[q]);
-      }
-      dst[v] = Vec16<XT>::pack(acc);
+      for (int q = 0; q < N; ++q) a1[q] = __fmaf_rn(w[k], f[q], a1[q]);
     }
+    if (ok0) dst[v0] = Vec16<XT>::pack(a0);
+    if (ok1) dst[v1] = Vec16<XT>::pack(a1);
   } else {
-    for (int v0 = 0; v0 < vec_per_row; v0 += 32) {  // warp-uniform trip count: the shuffles need all lanes
-      const int v = v0 + lane;
-      float acc[N];
+    float a0[N], a1[N];
 #pragma unroll
-      for (int q = 0; q < N; ++q) acc[q] = 0.0f;
-      for (int k = 0; k < K; ++k) {
-        const int s = __shfl_sync(0xffffffffu, my_slot, k);
-        const float wk = __shfl_sync(0xffffffffu, my_w, k);
-        if (s < 0 || v >= vec_per_row) continue;
-        float f[N];
-        Vec16<XT>::unpack(__ldcs(rows + (size_t)s * vec_per_row + v), f);
+    for (int q = 0; q < N; ++q) a0[q] = a1[q] = 0.0f;
+    for (int k = 0; k < K; ++k) {  // warp-uniform trip count: the shuffles need all lanes
+      const int s = __shfl_sync(0xffffffffu, my_slot, k);
+      const float wk = __shfl_sync(0xffffffffu, my_w, k);
+      if (s < 0) continue;
+      const uint4* src = rows + (size_t)s * vec_per_row;
+      float f[N];
+      if (ok0) {
+        Vec16<XT>::unpack(__ldcs(src + v0), f);
 #pragma unroll
-        for (int q = 0; q < N; ++q) acc[q] = __fmaf_rn(wk, f[q], acc[q]);
+        for (int q = 0; q < N; ++q) a0[q] = __fmaf_rn(wk, f[q], a0[q]);
       }
-      if (v < vec_per_row) dst[v] = Vec16<XT>::pack(acc);
+      if (ok1) {
+        Vec16<XT>::unpack(__ldcs(src + v1), f);
+#pragma unroll
+        for (int q = 0; q < N; ++q) a1[q] = __fmaf_rn(wk, f[q], a1[q]);
+      }
     }
+    if (ok0) dst[v0] = Vec16<XT>::pack(a0);
+    if (ok1) dst[v1] = Vec16<XT>::pack(a1);
   }
 }
 
@@ -78,10 +93,12 @@ static int launch_typed(moe_plan* p, const void* rows, const int* slot_of, const
                         cudaStream_t st) {
   const moe_config_t& c = p->cfg;
   const int vec_per_row = c.H * (int)sizeof(XT) / 16;
-  const int grid = (c.T + kCombThreads / 32 - 1) / (kCombThreads / 32);
+  const int runs_per_row = (vec_per_row + kCombRun - 1) / kCombRun;
+  const long long warps = (long long)c.T * runs_per_row;
+  const int grid = (int)((warps + kCombThreads / 32 - 1) / (kCombThreads / 32));
 #define MOEHUB_COMBINE(KT)                                                                          \
   combine_kernel<XT, KT><<<grid, kCombThreads, 0, st>>>((const uint4*)rows, slot_of, topk_w, c.T, c.K, \
-                                                        vec_per_row, (uint4*)y)
+                                                        vec_per_row, runs_per_row, (uint4*)y)
   switch (c.K) {
     case 1: MOEHUB_COMBINE(1); break;
     case 2: MOEHUB_COMBINE(2); break;

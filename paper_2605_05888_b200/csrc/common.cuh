@@ -24,7 +24,7 @@ __device__ __forceinline__ void set_status(int* status, int code, int detail) {
 
 // Wait sites reported in the detail word of MOE_ERR_TIMEOUT.
 enum WaitSite { kWaitTileTable = 1, kWaitScanTicket = 2, kWaitMbarTma = 3, kWaitMbarMma = 4,
-                kWaitMbarEpi = 5, kWaitMbarTmemFree = 6 };
+                kWaitMbarEpi = 5, kWaitMbarTmemFree = 6, kWaitTileReady = 7 };
 
 struct Scratch {          // device pointers carved out of the caller's workspace
   int* status;            // [4]
@@ -36,6 +36,10 @@ struct Scratch {          // device pointers carved out of the caller's workspac
   int* tile_base;         // [E + 1]    mode 0: first pool tile of each expert
   int* tile_list;         // [P]   used tiles grouped by expert (FFN work list)
   int* expert_start;      // [E + 1] first work-list index of each expert
+  int* seg_start;         // [2E + 1] first item of each work segment
+  int* seg_info;          // [2E]   expert | type << 16 of each segment
+  int* work_meta;         // [4]    [0]: items before the first GEMM2 item (split launches)
+  int* gemm1_done;        // [P]    per-tile status counter: GEMM1 blocks finished (x4 epilogue warps)
   void* inter;            // [P*128, F] SwiGLU intermediate
   // moe_layer's internal buffers
   int* topk_idx;

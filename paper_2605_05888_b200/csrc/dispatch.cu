@@ -260,21 +260,37 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
 }
 
 // ------------------------------------------------------------------------------------------------
+// One launch that puts every per-call counter and table into its start state.
+__global__ void __launch_bounds__(kDispThreads)
+reset_kernel(int* __restrict__ counters, int n_counters, int* __restrict__ expert_count, int E,
+             int* __restrict__ tile_expert, int P, int* __restrict__ src_info, int n_src,
+             int* __restrict__ tile_table, int n_table) {
+  const int stride = gridDim.x * kDispThreads;
+  const int i0 = blockIdx.x * kDispThreads + threadIdx.x;
+  for (int i = i0; i < n_counters; i += stride) counters[i] = 0;
+  for (int i = i0; i < E; i += stride) expert_count[i] = 0;
+  for (int i = i0; i < P; i += stride) tile_expert[i] = -1;
+  for (int i = i0; i < n_table; i += stride) tile_table[i] = -1;
+  for (int i = i0; i < n_src; i += stride) src_info[i] = -1;
+}
+
+// ------------------------------------------------------------------------------------------------
 int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv, int* expert_count,
                     int* tile_expert, int* src_info, int* slot_of, cudaStream_t st) {
   const moe_config_t& c = p->cfg;
   const int eb = c.dtype == MOE_DTYPE_BF16 ? 2 : 4;
   const int vec_per_row = c.H * eb / 16;
-  cudaError_t err;
-  // Per-call reset: scratch counters and tables, the caller's counters, owner and source arrays.
-  if ((err = cudaMemsetAsync(p->s.status, 0, p->counters_bytes, st)) != cudaSuccess) return (int)err;
-  if (c.dispatch_mode == MOE_DISPATCH_ATOMIC_PAGED) {
-    if ((err = cudaMemsetAsync(p->s.tile_table, 0xff, sizeof(int) * (size_t)c.E * p->tiles_per_expert, st)) != cudaSuccess)
-      return (int)err;
+  // Per-call reset in one launch: scratch counters and tile table, the caller's counters, owner and
+  // source arrays.
+  {
+    const int table = c.dispatch_mode == MOE_DISPATCH_ATOMIC_PAGED ? c.E * p->tiles_per_expert : 0;
+    const long long most = max((long long)p->P * kTileRows, (long long)table);
+    const int grid = (int)max(1ll, (most + 4 * kDispThreads - 1) / (4 * kDispThreads));
+    reset_kernel<<<grid, kDispThreads, 0, st>>>(p->s.status, (int)(p->counters_bytes / sizeof(int)), expert_count,
+                                                c.E, tile_expert, (int)p->P, src_info, (int)(p->P * kTileRows),
+                                                p->s.tile_table, table);
+    p->launches += 1;
   }
-  if ((err = cudaMemsetAsync(expert_count, 0, sizeof(int) * c.E, st)) != cudaSuccess) return (int)err;
-  if ((err = cudaMemsetAsync(tile_expert, 0xff, sizeof(int) * p->P, st)) != cudaSuccess) return (int)err;
-  if ((err = cudaMemsetAsync(src_info, 0xff, sizeof(int) * p->P * kTileRows, st)) != cudaSuccess) return (int)err;
   if (c.T == 0) return 0;
   const int nblk = p->nblk, tpb = p->dispatch_tokens;
   if (c.dispatch_mode == MOE_DISPATCH_SCAN) {

@@ -15,10 +15,18 @@
 // Work order is expert-major, then column block, then tile, so that CTAs running at the same time
 // share the weight block through L2 and an expert's rows stay L2-resident across its column blocks.
 //
+// Both GEMMs run in ONE persistent launch.  A GEMM2 item of a tile may start only when all column
+// blocks of that tile's intermediate are written: the software form of the paper's data
+// availability manager (Section IV-D) - a per-tile status counter bumped (release) by every
+// epilogue warp that finished a GEMM1 block, and a consumer that waits (acquire, bounded) for the
+// counter to reach its threshold before its TMA loads touch the tile.  The GEMM2 items of an expert
+// are placed a few hundred items behind its GEMM1 items, so the wait is normally over before it
+// starts.  The same kernel also runs the two GEMMs as two launches (phase 1 / phase 2).
+//
 // Roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (owns the TMEM allocation),
-// warps 2-5 = epilogue (TMEM lane quarter = warp % 4).  Every mbarrier wait is bounded in time;
-// on expiry the CTA records MOE_ERR_TIMEOUT, drains its outstanding TMA copies (bounded), frees
-// its TMEM and returns.
+// warps 2-5 = epilogue (TMEM lane quarter = warp % 4).  Every wait is bounded in time; on expiry
+// the CTA records MOE_ERR_TIMEOUT, drains its outstanding TMA copies (bounded), frees its TMEM and
+// returns.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -122,17 +130,25 @@ constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kUm
 
 // ---- work list ------------------------------------------------------------------------------
 // tile_list: the used tiles grouped by expert; expert_start[e]: first index of expert e's tiles,
-// expert_start[E] = number of used tiles.
+// expert_start[E] = number of used tiles.  Segments: the item sequence is a list of at most 2E
+// segments, segment = all GEMM1 items or all GEMM2 items of one expert; seg_start[i] is the first
+// item of segment i (seg_start[2E] = number of items), seg_info[i] = expert | type << 16
+// (type 0: GEMM1, 1: GEMM2).  meta[0] = number of items that precede the first GEMM2 item when the
+// launch is split in two phases.
+constexpr int kMaxExperts = 256;
+
 __global__ void __launch_bounds__(256)
-worklist_kernel(const int* __restrict__ tile_expert, int P, int E, int* __restrict__ tile_list,
-                int* __restrict__ expert_start) {
-  __shared__ int s_cnt[256];
-  __shared__ int s_cur[256];
+worklist_kernel(const int* __restrict__ tile_expert, int P, int E, int NB1, int NB2, int lag, int fused,
+                int* __restrict__ tile_list, int* __restrict__ expert_start, int* __restrict__ seg_start,
+                int* __restrict__ seg_info, int* __restrict__ meta, int* __restrict__ gemm1_done) {
+  __shared__ int s_cnt[kMaxExperts];
+  __shared__ int s_cur[kMaxExperts];
   __shared__ int s_warp[8];
   const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
   s_cnt[threadIdx.x] = 0;
   __syncthreads();
   for (int p = threadIdx.x; p < P; p += 256) {
+    gemm1_done[p] = 0;
     const int e = tile_expert[p];
     if (e >= 0 && e < E) atomicAdd(&s_cnt[e], 1);
   }
@@ -157,6 +173,30 @@ worklist_kernel(const int* __restrict__ tile_expert, int P, int E, int* __restri
     const int e = tile_expert[p];
     if (e >= 0 && e < E) tile_list[atomicAdd(&s_cur[e], 1)] = p;
   }
+  if (threadIdx.x == 0) {
+    // Item order.  Split launches: all GEMM1 segments, then all GEMM2 segments.  One launch: the GEMM2
+    // segment of an expert follows once at least `lag` items were placed after its GEMM1 segment.
+    int pos = 0, nseg = 0, q = 0;
+    for (int e = 0; e < E; ++e) {
+      seg_start[nseg] = pos;
+      seg_info[nseg++] = e;
+      pos += s_cnt[e] * NB1;
+      s_cur[e] = pos;  // end of this expert's GEMM1 items
+      while (fused && q < e && pos - s_cur[q] >= lag) {
+        seg_start[nseg] = pos;
+        seg_info[nseg++] = q | (1 << 16);
+        pos += s_cnt[q] * NB2;
+        ++q;
+      }
+    }
+    meta[0] = fused ? 0 : pos;
+    for (; q < E; ++q) {
+      seg_start[nseg] = pos;
+      seg_info[nseg++] = q | (1 << 16);
+      pos += s_cnt[q] * NB2;
+    }
+    seg_start[nseg] = pos;  // nseg == 2E
+  }
 }
 
 // ---- the grouped GEMM -----------------------------------------------------------------------
@@ -169,20 +209,31 @@ struct TcShared {
   int abort_flag;
 };
 
-template <bool SWIGLU>
+struct Item {
+  int type;   // 0: GEMM1 (+SwiGLU), 1: GEMM2
+  int e, nb, tile;
+};
+
 __global__ void __launch_bounds__(kTcThreads, 1)
-ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b1,
-              const __grid_constant__ CUtensorMap map_b2, const int* __restrict__ tile_list,
-              const int* __restrict__ expert_start, int E, int N, int Kd, __nv_bfloat16* __restrict__ C, int ldc,
+ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_bg,
+              const __grid_constant__ CUtensorMap map_bu, const __grid_constant__ CUtensorMap map_a2,
+              const __grid_constant__ CUtensorMap map_bd, const int* __restrict__ tile_list,
+              const int* __restrict__ expert_start, const int* __restrict__ seg_start,
+              const int* __restrict__ seg_info, const int* __restrict__ meta, int phase, int E, int F, int H,
+              __nv_bfloat16* __restrict__ inter, __nv_bfloat16* __restrict__ out, int* __restrict__ gemm1_done,
               int* __restrict__ status) {
-  constexpr int BN = SWIGLU ? 128 : 256;  // output columns per work item
   extern __shared__ uint8_t smem_raw[];
   uint8_t* stage_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   TcShared* sh = reinterpret_cast<TcShared*>(stage_base + kStages * kStageBytes);
-  __shared__ int s_start[257];
+  __shared__ int s_estart[kMaxExperts + 1];
+  __shared__ int s_seg_start[2 * kMaxExperts + 1];
+  __shared__ int s_seg_info[2 * kMaxExperts];
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  for (int i = threadIdx.x; i <= E; i += kTcThreads) s_start[i] = expert_start[i];
+  const int nseg = 2 * E;
+  for (int i = threadIdx.x; i <= E; i += kTcThreads) s_estart[i] = expert_start[i];
+  for (int i = threadIdx.x; i <= nseg; i += kTcThreads) s_seg_start[i] = seg_start[i];
+  for (int i = threadIdx.x; i < nseg; i += kTcThreads) s_seg_info[i] = seg_info[i];
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&sh->full[s]), 1);
@@ -206,53 +257,74 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
   const uint32_t tmem_base = sh->tmem_base;
   volatile int* abort_flag = &sh->abort_flag;
 
-  const int NB = (N + BN - 1) / BN;
-  const int KB = (Kd + kBK - 1) / kBK;
-  const int total_items = s_start[E] * NB;
+  const int NB1 = (F + 127) / 128, NB2 = (H + 255) / 256;
+  const int KB1 = (H + kBK - 1) / kBK, KB2 = (F + kBK - 1) / kBK;
+  int item_begin = 0, item_end = s_seg_start[nseg];
+  if (phase == 1) item_end = meta[0];
+  if (phase == 2) item_begin = meta[0];
 
-  // item -> (expert, column block, tile): expert-major, column-block-major, tile-minor
-  auto decode = [&](int item, int& e, int& nb, int& tile) {
-    int lo = 0, hi = E;  // largest e with s_start[e] * NB <= item
+  // item -> (type, expert, column block, tile); inside a segment column-block-major, tile-minor
+  auto decode = [&](int item) {
+    int lo = 0, hi = nseg;  // largest segment whose first item is <= item
     while (hi - lo > 1) {
       const int mid = (lo + hi) / 2;
-      if (s_start[mid] * NB <= item) lo = mid; else hi = mid;
+      if (s_seg_start[mid] <= item) lo = mid; else hi = mid;
     }
-    e = lo;
-    const int m = s_start[e + 1] - s_start[e];
-    const int local = item - s_start[e] * NB;
-    nb = local / m;
-    tile = tile_list[s_start[e] + local % m];
+    Item it;
+    it.type = s_seg_info[lo] >> 16;
+    it.e = s_seg_info[lo] & 0xffff;
+    const int m = s_estart[it.e + 1] - s_estart[it.e];
+    const int local = item - s_seg_start[lo];
+    it.nb = local / m;
+    it.tile = tile_list[s_estart[it.e] + local % m];
+    return it;
   };
+  const int first_item = item_begin + blockIdx.x;
 
   int fail_site = 0;
   if (warp == 0) {
     // ===================== TMA producer =====================
     if (lane == 0) {
       int stage = 0;
-      uint32_t phase = 0;
+      uint32_t phase_bit = 0;
       int armed[kStages];
 #pragma unroll
       for (int s = 0; s < kStages; ++s) armed[s] = 0;
-      for (int item = blockIdx.x; item < total_items && !fail_site; item += gridDim.x) {
-        int e, nb, tile;
-        decode(item, e, nb, tile);
+      for (int item = first_item; item < item_end && !fail_site; item += gridDim.x) {
+        const Item it = decode(item);
+        if (it.type == 1) {
+          // Availability of this tile's intermediate: every epilogue warp of every GEMM1 block bumps
+          // the tile's counter once.  Bounded wait, then order the async proxy behind what was seen.
+          const int need = 4 * NB1;
+          if (ld_acquire(&gemm1_done[it.tile]) < need) {
+            const unsigned long long t0 = globaltimer();
+            while (ld_acquire(&gemm1_done[it.tile]) < need) {
+              if (*abort_flag || globaltimer() - t0 > kWaitNs) { fail_site = kWaitTileReady; break; }
+              __nanosleep(64);
+            }
+            if (fail_site) break;
+          }
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+        }
+        const CUtensorMap* ma = it.type == 0 ? &map_a1 : &map_a2;
+        const int KB = it.type == 0 ? KB1 : KB2;
         for (int kb = 0; kb < KB; ++kb) {
-          if (!mbar_wait(smem_u32(&sh->empty[stage]), phase ^ 1u, abort_flag)) { fail_site = kWaitMbarTma; break; }
+          if (!mbar_wait(smem_u32(&sh->empty[stage]), phase_bit ^ 1u, abort_flag)) { fail_site = kWaitMbarTma; break; }
           const uint32_t full = smem_u32(&sh->full[stage]);
           const uint32_t a_dst = smem_u32(stage_base + stage * kStageBytes);
           const uint32_t b_dst = a_dst + kABytes;
           mbar_expect_tx(full, kStageBytes);
-          tma_load_2d(a_dst, &map_a, full, kb * kBK, tile * kTileRows);
-          if (SWIGLU) {
-            tma_load_3d(b_dst, &map_b1, full, kb * kBK, nb * BN, e);
-            tma_load_3d(b_dst + kBBytes / 2, &map_b2, full, kb * kBK, nb * BN, e);
+          tma_load_2d(a_dst, ma, full, kb * kBK, it.tile * kTileRows);
+          if (it.type == 0) {
+            tma_load_3d(b_dst, &map_bg, full, kb * kBK, it.nb * 128, it.e);
+            tma_load_3d(b_dst + kBBytes / 2, &map_bu, full, kb * kBK, it.nb * 128, it.e);
           } else {
-            tma_load_3d(b_dst, &map_b1, full, kb * kBK, nb * BN, e);
+            tma_load_3d(b_dst, &map_bd, full, kb * kBK, it.nb * 256, it.e);
           }
 #pragma unroll
           for (int s = 0; s < kStages; ++s)
             if (s == stage) armed[s] += 1;
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (++stage == kStages) { stage = 0; phase_bit ^= 1u; }
         }
       }
       if (fail_site || *abort_flag) {
@@ -272,16 +344,18 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     // ===================== MMA issuer =====================
     if (lane == 0) {
       int stage = 0;
-      uint32_t phase = 0;
+      uint32_t phase_bit = 0;
       int local_item = 0;
-      for (int item = blockIdx.x; item < total_items && !fail_site; item += gridDim.x, ++local_item) {
+      for (int item = first_item; item < item_end && !fail_site; item += gridDim.x, ++local_item) {
+        const Item it = decode(item);
+        const int KB = it.type == 0 ? KB1 : KB2;
         const int acc = local_item & 1;
         const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
         if (!mbar_wait(smem_u32(&sh->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) { fail_site = kWaitMbarTmemFree; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kUmmaN);
         for (int kb = 0; kb < KB; ++kb) {
-          if (!mbar_wait(smem_u32(&sh->full[stage]), phase, abort_flag)) { fail_site = kWaitMbarMma; break; }
+          if (!mbar_wait(smem_u32(&sh->full[stage]), phase_bit, abort_flag)) { fail_site = kWaitMbarMma; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(stage_base + stage * kStageBytes);
           const uint64_t adesc = smem_desc_sw128(a_addr);
@@ -290,7 +364,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
           for (int k = 0; k < kBK / 16; ++k)  // 16 k-elements = 32 bytes = 2 descriptor units per step
             tc_mma(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
           tc_commit(smem_u32(&sh->empty[stage]));  // the stage is free once these MMAs have read it
-          if (++stage == kStages) { stage = 0; phase ^= 1u; }
+          if (++stage == kStages) { stage = 0; phase_bit ^= 1u; }
         }
         if (fail_site) break;
         tc_commit(smem_u32(&sh->tmem_full[acc]));  // accumulator complete
@@ -299,22 +373,22 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
     }
   } else {
     // ===================== epilogue =====================
-    const int quarter = warp & 3;                 // TMEM lanes this warp may read
+    const int quarter = warp & 3;  // TMEM lanes this warp may read
     const int row_in_tile = quarter * 32 + lane;
     int local_item = 0;
-    for (int item = blockIdx.x; item < total_items && !fail_site; item += gridDim.x, ++local_item) {
-      int e, nb, tile;
-      decode(item, e, nb, tile);
+    for (int item = first_item; item < item_end && !fail_site; item += gridDim.x, ++local_item) {
+      const Item it = decode(item);
       const int acc = local_item & 1;
       const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
       if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag)) { fail_site = kWaitMbarEpi; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kUmmaN);
-      __nv_bfloat16* out = C + ((size_t)tile * kTileRows + row_in_tile) * ldc + (size_t)nb * BN;
-      const int ncols = min(BN, N - nb * BN);
-      if (SWIGLU) {
+      const size_t row = (size_t)it.tile * kTileRows + row_in_tile;
+      if (it.type == 0) {
+        __nv_bfloat16* dst = inter + row * F + (size_t)it.nb * 128;
+        const int ncols = min(128, F - it.nb * 128);
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 16) {
+        for (int c = 0; c < 128; c += 16) {
           uint32_t g[16], u[16];
           tc_ld16(t_row + c, g);
           tc_ld16(t_row + 128 + c, u);
@@ -325,12 +399,14 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
             const float gv = __uint_as_float(g[i]);
             s[i] = gv / (1.0f + __expf(-gv)) * __uint_as_float(u[i]);
           }
-          if (c + 8 <= ncols) *reinterpret_cast<uint4*>(out + c) = Vec16<__nv_bfloat16>::pack(s);
-          if (c + 16 <= ncols) *reinterpret_cast<uint4*>(out + c + 8) = Vec16<__nv_bfloat16>::pack(s + 8);
+          if (c + 8 <= ncols) *reinterpret_cast<uint4*>(dst + c) = Vec16<__nv_bfloat16>::pack(s);
+          if (c + 16 <= ncols) *reinterpret_cast<uint4*>(dst + c + 8) = Vec16<__nv_bfloat16>::pack(s + 8);
         }
       } else {
+        __nv_bfloat16* dst = out + row * H + (size_t)it.nb * 256;
+        const int ncols = min(256, H - it.nb * 256);
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 32) {
+        for (int c = 0; c < 256; c += 32) {
           uint32_t r0[16], r1[16];
           tc_ld16(t_row + c, r0);
           tc_ld16(t_row + c + 16, r1);
@@ -340,12 +416,21 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__
           for (int i = 0; i < 16; ++i) { f[i] = __uint_as_float(r0[i]); f[16 + i] = __uint_as_float(r1[i]); }
 #pragma unroll
           for (int q = 0; q < 4; ++q)
-            if (c + 8 * q + 8 <= ncols) *reinterpret_cast<uint4*>(out + c + 8 * q) = Vec16<__nv_bfloat16>::pack(f + 8 * q);
+            if (c + 8 * q + 8 <= ncols) *reinterpret_cast<uint4*>(dst + c + 8 * q) = Vec16<__nv_bfloat16>::pack(f + 8 * q);
         }
       }
       tc_fence_before();
+      if (it.type == 0) {
+        // This warp's part of the block is written: make it visible (also to the async proxy, which
+        // is how the GEMM2 producer will read it) and bump the tile's status counter.
+        asm volatile("fence.proxy.async.global;" ::: "memory");
+        __threadfence();
+      }
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&sh->tmem_empty[acc]));
+      if (lane == 0) {
+        mbar_arrive(smem_u32(&sh->tmem_empty[acc]));
+        if (it.type == 0) asm volatile("red.release.gpu.global.add.s32 [%0], 1;" ::"l"(gemm1_done + it.tile) : "memory");
+      }
     }
     if (fail_site) sh->abort_flag = 1;
   }
@@ -418,20 +503,33 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
 
   static bool attr_done = false;  // per-process, idempotent
   if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem) != cudaSuccess ||
-        cudaFuncSetAttribute(ffn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem) != cudaSuccess)
+    if (cudaFuncSetAttribute(ffn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem) != cudaSuccess)
       return MOE_ERR_CUDA;
     attr_done = true;
   }
-  worklist_kernel<<<1, 256, 0, st>>>(tile_expert, (int)p->P, c.E, p->s.tile_list, p->s.expert_start);
-  mark(p, 3, st);
   const int grid = p->sm_count;
-  ffn_tc_kernel<true><<<grid, kTcThreads, kTcSmem, st>>>(a1, bg, bu, p->s.tile_list, p->s.expert_start, c.E, c.F, c.H,
-                                                         (__nv_bfloat16*)p->s.inter, c.F, p->s.status);
-  mark(p, 4, st);
-  ffn_tc_kernel<false><<<grid, kTcThreads, kTcSmem, st>>>(a2, bd, bd, p->s.tile_list, p->s.expert_start, c.E, c.H, c.F,
-                                                          (__nv_bfloat16*)out_rows, c.H, p->s.status);
-  p->launches += 3;
+  const int NB1 = (c.F + 127) / 128, NB2 = (c.H + 255) / 256;
+  // One launch for both GEMMs, except under moe_layer_timed, which wants a time for each.
+  const int fused = (p->timing || c.ffn_split) ? 0 : 1;
+  worklist_kernel<<<1, 256, 0, st>>>(tile_expert, (int)p->P, c.E, NB1, NB2, 2 * grid, fused, p->s.tile_list,
+                                     p->s.expert_start, p->s.seg_start, p->s.seg_info, p->s.work_meta,
+                                     p->s.gemm1_done);
+  mark(p, 3, st);
+  auto launch = [&](int phase) {
+    ffn_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(a1, bg, bu, a2, bd, p->s.tile_list, p->s.expert_start,
+                                                     p->s.seg_start, p->s.seg_info, p->s.work_meta, phase, c.E, c.F,
+                                                     c.H, (__nv_bfloat16*)p->s.inter, (__nv_bfloat16*)out_rows,
+                                                     p->s.gemm1_done, p->s.status);
+  };
+  if (fused) {
+    launch(0);
+    p->launches += 2;
+  } else {
+    launch(1);
+    mark(p, 4, st);
+    launch(2);
+    p->launches += 3;
+  }
   return cudaGetLastError() == cudaSuccess ? 0 : MOE_ERR_CUDA;
 }
 

@@ -15,12 +15,11 @@
 namespace moehub {
 
 constexpr int kRouteThreads = 256;
-constexpr int kHC = 32;  // h elements per staged chunk
 
-template <typename XT, int ROWS>
-struct ChunkRegs {  // the 16-byte vectors one thread holds of a [ROWS][kHC] chunk
+template <typename XT, int ROWS, int HC>
+struct ChunkRegs {  // the 16-byte vectors one thread holds of a [ROWS][HC] chunk
   static constexpr int N = Vec16<XT>::N;
-  static constexpr int PARTS = kHC / N;
+  static constexpr int PARTS = HC / N;
   static constexpr int NVEC = ROWS * PARTS;
   static constexpr int PER_THREAD = (NVEC + kRouteThreads - 1) / kRouteThreads;
   uint4 v[PER_THREAD];
@@ -36,7 +35,7 @@ struct ChunkRegs {  // the 16-byte vectors one thread holds of a [ROWS][kHC] chu
         v[i] = __ldg(reinterpret_cast<const uint4*>(base + (size_t)(row0 + r) * H + h));
     }
   }
-  // smem layout [kHC][ROWS + 1] (transposed; the odd width keeps the transposing stores conflict-free)
+  // smem layout [HC][ROWS + 1] (transposed; the odd width keeps the transposing stores conflict-free)
   __device__ __forceinline__ void store(float* s) const {
 #pragma unroll
     for (int i = 0; i < PER_THREAD; ++i) {
@@ -52,70 +51,12 @@ struct ChunkRegs {  // the 16-byte vectors one thread holds of a [ROWS][kHC] chu
   }
 };
 
-template <typename XT, int TX, int TE, int TY, int TM>
-__global__ void __launch_bounds__(kRouteThreads)
-route_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias,
-             int T, int H, int E, int K, int renorm, int* __restrict__ topk_idx,
-             float* __restrict__ topk_w) {
-  static_assert(TX * TY == kRouteThreads, "thread layout");
-  constexpr int TB = TY * TM, EP = TX * TE;
-  constexpr int XW = TB + 1, WW = EP + 1;
-  extern __shared__ float smem[];
-  float* xs = smem;             // [kHC][XW]
-  float* ws = smem + kHC * XW;  // [kHC][WW]
-  float* ls = smem;             // [TB][EP], reuses the staging area after the h loop
-
-  const int tx = threadIdx.x % TX, ty = threadIdx.x / TX;
-  const int t0 = blockIdx.x * TB;
-  const int tvalid = min(TB, T - t0);
-
-  float acc[TM][TE];
-#pragma unroll
-  for (int j = 0; j < TM; ++j)
-#pragma unroll
-    for (int i = 0; i < TE; ++i) acc[j][i] = 0.0f;
-
-  ChunkRegs<XT, TB> xr;
-  ChunkRegs<XT, EP> wrg;
-  xr.load(x, t0, tvalid, H, 0);
-  wrg.load(wr, 0, E, H, 0);
-
-  for (int h0 = 0; h0 < H; h0 += kHC) {
-    __syncthreads();  // previous chunk fully consumed
-    xr.store(xs);
-    wrg.store(ws);
-    __syncthreads();
-    if (h0 + kHC < H) {  // prefetch the next chunk while this one is computed
-      xr.load(x, t0, tvalid, H, h0 + kHC);
-      wrg.load(wr, 0, E, H, h0 + kHC);
-    }
-    const int hmax = min(kHC, H - h0);
-#pragma unroll 4
-    for (int hh = 0; hh < hmax; ++hh) {
-      float xv[TM], wv[TE];
-#pragma unroll
-      for (int j = 0; j < TM; ++j) xv[j] = xs[hh * XW + ty + TY * j];
-#pragma unroll
-      for (int i = 0; i < TE; ++i) wv[i] = ws[hh * WW + tx + TX * i];
-#pragma unroll
-      for (int j = 0; j < TM; ++j)
-#pragma unroll
-        for (int i = 0; i < TE; ++i) acc[j][i] = __fmaf_rn(xv[j], wv[i], acc[j][i]);
-    }
-  }
-  __syncthreads();
-#pragma unroll
-  for (int j = 0; j < TM; ++j)
-#pragma unroll
-    for (int i = 0; i < TE; ++i) {
-      const int e = tx + TX * i;
-      float l = acc[j][i];
-      if (bias != nullptr && e < E) l = l + bias[e];
-      ls[(ty + TY * j) * EP + e] = l;
-    }
-  __syncthreads();
-
-  // ---- one warp per token: top-K by K rounds of arg-max, then softmax weights ----
+// One warp per token: the token's logits sit in registers (EP/32 per lane); K rounds of a shuffle
+// arg-max on (value, lowest index); then the softmax weights of the picks.  ls: [tokens][EP] logits
+// in shared memory.
+template <int EP>
+__device__ __forceinline__ void select_topk(const float* ls, int tvalid, int t0, int E, int K, int renorm,
+                                            int* __restrict__ topk_idx, float* __restrict__ topk_w) {
   constexpr int NJ = (EP + 31) / 32;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   for (int tl = warp; tl < tvalid; tl += kRouteThreads / 32) {
@@ -168,14 +109,80 @@ route_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* _
   }
 }
 
-template <typename XT, int TX, int TE, int TY, int TM>
+template <typename XT, int TX, int TE, int TY, int TM, int HC>
+__global__ void __launch_bounds__(kRouteThreads)
+route_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias,
+             int T, int H, int E, int K, int renorm, int* __restrict__ topk_idx,
+             float* __restrict__ topk_w) {
+  static_assert(TX * TY == kRouteThreads, "thread layout");
+  constexpr int TB = TY * TM, EP = TX * TE;
+  constexpr int XW = TB + 1, WW = EP + 1;
+  extern __shared__ float smem[];
+  float* xs = smem;            // [HC][XW]
+  float* ws = smem + HC * XW;  // [HC][WW]
+  float* ls = smem;             // [TB][EP], reuses the staging area after the h loop
+
+  const int tx = threadIdx.x % TX, ty = threadIdx.x / TX;
+  const int t0 = blockIdx.x * TB;
+  const int tvalid = min(TB, T - t0);
+
+  float acc[TM][TE];
+#pragma unroll
+  for (int j = 0; j < TM; ++j)
+#pragma unroll
+    for (int i = 0; i < TE; ++i) acc[j][i] = 0.0f;
+
+  ChunkRegs<XT, TB, HC> xr;
+  ChunkRegs<XT, EP, HC> wrg;
+  xr.load(x, t0, tvalid, H, 0);
+  wrg.load(wr, 0, E, H, 0);
+
+  for (int h0 = 0; h0 < H; h0 += HC) {
+    __syncthreads();  // previous chunk fully consumed
+    xr.store(xs);
+    wrg.store(ws);
+    __syncthreads();
+    if (h0 + HC < H) {  // prefetch the next chunk while this one is computed
+      xr.load(x, t0, tvalid, H, h0 + HC);
+      wrg.load(wr, 0, E, H, h0 + HC);
+    }
+    const int hmax = min(HC, H - h0);
+#pragma unroll 4
+    for (int hh = 0; hh < hmax; ++hh) {
+      float xv[TM], wv[TE];
+#pragma unroll
+      for (int j = 0; j < TM; ++j) xv[j] = xs[hh * XW + ty + TY * j];
+#pragma unroll
+      for (int i = 0; i < TE; ++i) wv[i] = ws[hh * WW + tx + TX * i];
+#pragma unroll
+      for (int j = 0; j < TM; ++j)
+#pragma unroll
+        for (int i = 0; i < TE; ++i) acc[j][i] = __fmaf_rn(xv[j], wv[i], acc[j][i]);
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < TM; ++j)
+#pragma unroll
+    for (int i = 0; i < TE; ++i) {
+      const int e = tx + TX * i;
+      float l = acc[j][i];
+      if (bias != nullptr && e < E) l = l + bias[e];
+      ls[(ty + TY * j) * EP + e] = l;
+    }
+  __syncthreads();
+
+  select_topk<EP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w);
+}
+
+template <typename XT, int TX, int TE, int TY, int TM, int HC>
 static int launch_cfg(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
                       float* topk_w, cudaStream_t st) {
   constexpr int TB = TY * TM, EP = TX * TE;
-  const size_t stage = sizeof(float) * kHC * (TB + 1 + EP + 1);
+  const size_t stage = sizeof(float) * HC * (TB + 1 + EP + 1);
   const size_t logits = sizeof(float) * TB * EP;
   const size_t smem = stage > logits ? stage : logits;
-  auto kern = route_kernel<XT, TX, TE, TY, TM>;
+  auto kern = route_kernel<XT, TX, TE, TY, TM, HC>;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
@@ -188,14 +195,285 @@ static int launch_cfg(moe_plan* p, const void* x, const void* wr, const float* b
   return (int)cudaGetLastError();
 }
 
+// The compute-bound shape (64 < E <= 256): 64 tokens x 256 experts per CTA, 8 x 8 chains per thread,
+// every shared-memory read of the inner loop a 16-byte vector: 4 loads feed 64 FMAs.  The staging
+// stores are conflict-free because consecutive lanes handle consecutive rows of one 16-byte column
+// group.
+constexpr int kWideTB = 64, kWideEP = 256, kWideHC = 32;
+
+template <typename XT, int ROWS>
+struct WideChunk {
+  static constexpr int N = Vec16<XT>::N;
+  static constexpr int PARTS = kWideHC / N;
+  static constexpr int PER_THREAD = ROWS * PARTS / kRouteThreads;
+  uint4 v[PER_THREAD];
+  __device__ __forceinline__ void load(const XT* base, int row0, int nrows_valid, int H, int h0) {
+#pragma unroll
+    for (int i = 0; i < PER_THREAD; ++i) {
+      const int idx = threadIdx.x + i * kRouteThreads;
+      const int r = idx % ROWS, part = idx / ROWS;
+      const int h = h0 + part * N;
+      v[i] = make_uint4(0, 0, 0, 0);
+      if (r < nrows_valid && h < H) v[i] = __ldg(reinterpret_cast<const uint4*>(base + (size_t)(row0 + r) * H + h));
+    }
+  }
+  __device__ __forceinline__ void store(float* s) const {  // s: [kWideHC][ROWS]
+#pragma unroll
+    for (int i = 0; i < PER_THREAD; ++i) {
+      const int idx = threadIdx.x + i * kRouteThreads;
+      const int r = idx % ROWS, part = idx / ROWS;
+      float f[N];
+      Vec16<XT>::unpack(v[i], f);
+#pragma unroll
+      for (int q = 0; q < N; ++q) s[(part * N + q) * ROWS + r] = f[q];
+    }
+  }
+};
+
+template <typename XT>
+__global__ void __launch_bounds__(kRouteThreads)
+route_wide_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias, int T,
+                  int H, int E, int K, int renorm, int* __restrict__ topk_idx, float* __restrict__ topk_w) {
+  extern __shared__ __align__(16) float smem[];
+  float* xs = smem;                      // [32][64]
+  float* ws = smem + kWideHC * kWideTB;  // [32][256]
+  float* ls = smem;                      // [64][256] after the h loop
+  // A warp is an 8 (token groups) x 4 (expert groups) grid of lanes and owns 32 experts for all 64
+  // tokens: per h it reads 256 B of x and 128 B of Wr from shared memory for 2048 FMAs.
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int ly = lane / 4, lx = lane % 4;
+  const int ebase = 32 * warp + 4 * lx;  // experts ebase..ebase+3 and ebase+16..ebase+19
+  const int t0 = blockIdx.x * kWideTB;
+  const int tvalid = min(kWideTB, T - t0);
+
+  float acc[8][8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j)
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[j][i] = 0.0f;
+
+  WideChunk<XT, kWideTB> xr;
+  WideChunk<XT, kWideEP> wrg;
+  xr.load(x, t0, tvalid, H, 0);
+  wrg.load(wr, 0, E, H, 0);
+  for (int h0 = 0; h0 < H; h0 += kWideHC) {
+    __syncthreads();
+    xr.store(xs);
+    wrg.store(ws);
+    __syncthreads();
+    if (h0 + kWideHC < H) {
+      xr.load(x, t0, tvalid, H, h0 + kWideHC);
+      wrg.load(wr, 0, E, H, h0 + kWideHC);
+    }
+    const int hmax = min(kWideHC, H - h0);
+    // software pipeline: the operands of step hh+1 are loaded while step hh is computed
+    float4 xa = *reinterpret_cast<const float4*>(xs + 4 * ly);
+    float4 xb = *reinterpret_cast<const float4*>(xs + 32 + 4 * ly);
+    float4 wa = *reinterpret_cast<const float4*>(ws + ebase);
+    float4 wb = *reinterpret_cast<const float4*>(ws + ebase + 16);
+#pragma unroll 2
+    for (int hh = 0; hh < hmax; ++hh) {
+      const int hn = min(hh + 1, kWideHC - 1);
+      const float4 nxa = *reinterpret_cast<const float4*>(xs + hn * kWideTB + 4 * ly);
+      const float4 nxb = *reinterpret_cast<const float4*>(xs + hn * kWideTB + 32 + 4 * ly);
+      const float4 nwa = *reinterpret_cast<const float4*>(ws + hn * kWideEP + ebase);
+      const float4 nwb = *reinterpret_cast<const float4*>(ws + hn * kWideEP + ebase + 16);
+      const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+      const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+#pragma unroll
+      for (int j = 0; j < 8; ++j)
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[j][i] = __fmaf_rn(xv[j], wv[i], acc[j][i]);
+      xa = nxa; xb = nxb; wa = nwa; wb = nwb;
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const int tl = (j < 4) ? 4 * ly + j : 32 + 4 * ly + (j - 4);
+#pragma unroll
+    for (int g = 0; g < 2; ++g) {
+      const int e0 = ebase + 16 * g;
+      float l[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        l[i] = acc[j][g * 4 + i];
+        if (bias != nullptr && e0 + i < E) l[i] = l[i] + bias[e0 + i];
+      }
+      *reinterpret_cast<float4*>(ls + tl * kWideEP + e0) = make_float4(l[0], l[1], l[2], l[3]);
+    }
+  }
+  __syncthreads();
+  select_topk<kWideEP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w);
+}
+
+template <typename XT>
+static int launch_wide(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
+                       float* topk_w, cudaStream_t st) {
+  const size_t smem = sizeof(float) * kWideTB * kWideEP;  // the logits tile; the staging area is smaller
+  auto kern = route_wide_kernel<XT>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return (int)e;
+  const moe_config_t& c = p->cfg;
+  kern<<<(c.T + kWideTB - 1) / kWideTB, kRouteThreads, smem, st>>>((const XT*)x, (const XT*)wr, bias, c.T, c.H,
+                                                                   c.E, c.K, c.renormalize, topk_idx, topk_w);
+  p->launches += 1;
+  return (int)cudaGetLastError();
+}
+
+// The latency-bound shapes (E <= 64): one lane per chain (or two chains for 32 < E <= 64).  A token's
+// experts sit on LE consecutive lanes; x and Wr tiles stay in their natural [row][h] layout in shared
+// memory (fp32, converted while staging), so a lane reads four consecutive h of its token and of its
+// expert with two 16-byte loads and runs its chain over them.  The time is close to the latency of
+// the chain itself (4 cycles per h) once the chunk loads are overlapped.
+template <typename XT, int ROWS, int HC>
+struct NaturalChunk {
+  static constexpr int N = Vec16<XT>::N;
+  static constexpr int PARTS = HC / N;
+  static constexpr int NVEC = ROWS * PARTS;
+  static constexpr int PER_THREAD = (NVEC + kRouteThreads - 1) / kRouteThreads;
+  static constexpr int PITCH = HC + 4;  // floats; rows land on different banks
+  uint4 v[PER_THREAD];
+  __device__ __forceinline__ void load(const XT* base, int row0, int nrows_valid, int H, int h0) {
+#pragma unroll
+    for (int i = 0; i < PER_THREAD; ++i) {
+      const int idx = threadIdx.x + i * kRouteThreads;
+      const int r = idx / PARTS, part = idx % PARTS;
+      const int h = h0 + part * N;
+      v[i] = make_uint4(0, 0, 0, 0);
+      if (idx < NVEC && r < nrows_valid && h < H)
+        v[i] = __ldg(reinterpret_cast<const uint4*>(base + (size_t)(row0 + r) * H + h));
+    }
+  }
+  __device__ __forceinline__ void store(float* s) const {  // s: [ROWS][PITCH]
+#pragma unroll
+    for (int i = 0; i < PER_THREAD; ++i) {
+      const int idx = threadIdx.x + i * kRouteThreads;
+      if (idx < NVEC) {
+        const int r = idx / PARTS, part = idx % PARTS;
+        float f[N];
+        Vec16<XT>::unpack(v[i], f);
+        float4* dst = reinterpret_cast<float4*>(s + r * PITCH + part * N);
+#pragma unroll
+        for (int q = 0; q < N / 4; ++q) dst[q] = make_float4(f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
+      }
+    }
+  }
+};
+
+template <typename XT, int LE, int TE, int HC>
+__global__ void __launch_bounds__(kRouteThreads)
+route_narrow_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias, int T,
+                    int H, int E, int K, int renorm, int* __restrict__ topk_idx, float* __restrict__ topk_w) {
+  constexpr int EP = LE * TE;              // experts covered (padded)
+  constexpr int TW = 32 / LE;              // tokens per warp
+  constexpr int TB = TW * (kRouteThreads / 32);
+  constexpr int PITCH = HC + 4;
+  extern __shared__ __align__(16) float smem[];
+  float* xs = smem;               // [TB][PITCH]
+  float* ws = smem + TB * PITCH;  // [EP][PITCH]
+  float* ls = smem;               // [TB][EP] after the h loop
+  const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+  const int tl = warp * TW + lane / LE;  // this lane's token inside the block
+  const int le = lane % LE;              // this lane's experts: le + LE*i
+  const int t0 = blockIdx.x * TB;
+  const int tvalid = min(TB, T - t0);
+
+  float acc[TE];
+#pragma unroll
+  for (int i = 0; i < TE; ++i) acc[i] = 0.0f;
+  NaturalChunk<XT, TB, HC> xr;
+  NaturalChunk<XT, EP, HC> wrg;
+  xr.load(x, t0, tvalid, H, 0);
+  wrg.load(wr, 0, E, H, 0);
+  for (int h0 = 0; h0 < H; h0 += HC) {
+    __syncthreads();
+    xr.store(xs);
+    wrg.store(ws);
+    __syncthreads();
+    if (h0 + HC < H) {
+      xr.load(x, t0, tvalid, H, h0 + HC);
+      wrg.load(wr, 0, E, H, h0 + HC);
+    }
+    const int hmax = min(HC, H - h0);
+    // Groups of 16 h: the next group's operands are loaded while this group's 16-step chain runs, so
+    // the shared-memory latency hides behind the chain.  The tail of a short last chunk is zero in
+    // shared memory (loads past H are zero-filled) and fma(0, 0, acc) leaves acc's value alone.
+    const float* xrow = xs + tl * PITCH;
+    const float* wrow = ws + le * PITCH;
+    constexpr int G = 4;
+    float4 xv[G], wv[TE][G];
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      xv[g] = *reinterpret_cast<const float4*>(xrow + 4 * g);
+#pragma unroll
+      for (int i = 0; i < TE; ++i) wv[i][g] = *reinterpret_cast<const float4*>(wrow + LE * i * PITCH + 4 * g);
+    }
+    for (int hh = 0; hh < hmax; hh += 4 * G) {
+      const int hn = min(hh + 4 * G, HC - 4 * G);
+      float4 nxv[G], nwv[TE][G];
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        nxv[g] = *reinterpret_cast<const float4*>(xrow + hn + 4 * g);
+#pragma unroll
+        for (int i = 0; i < TE; ++i) nwv[i][g] = *reinterpret_cast<const float4*>(wrow + LE * i * PITCH + hn + 4 * g);
+      }
+#pragma unroll
+      for (int g = 0; g < G; ++g)
+#pragma unroll
+        for (int i = 0; i < TE; ++i) {
+          acc[i] = __fmaf_rn(xv[g].x, wv[i][g].x, acc[i]);
+          acc[i] = __fmaf_rn(xv[g].y, wv[i][g].y, acc[i]);
+          acc[i] = __fmaf_rn(xv[g].z, wv[i][g].z, acc[i]);
+          acc[i] = __fmaf_rn(xv[g].w, wv[i][g].w, acc[i]);
+        }
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        xv[g] = nxv[g];
+#pragma unroll
+        for (int i = 0; i < TE; ++i) wv[i][g] = nwv[i][g];
+      }
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int i = 0; i < TE; ++i) {
+    const int e = le + LE * i;
+    float l = acc[i];
+    if (bias != nullptr && e < E) l = l + bias[e];
+    ls[tl * EP + e] = l;
+  }
+  __syncthreads();
+  select_topk<EP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w);
+}
+
+template <typename XT, int LE, int TE, int HC>
+static int launch_narrow(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
+                         float* topk_w, cudaStream_t st) {
+  constexpr int EP = LE * TE, TB = (32 / LE) * (kRouteThreads / 32);
+  const size_t smem = sizeof(float) * (TB + EP) * (HC + 4);
+  auto kern = route_narrow_kernel<XT, LE, TE, HC>;
+  if (smem > 48 * 1024) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return (int)e;
+  }
+  const moe_config_t& c = p->cfg;
+  kern<<<(c.T + TB - 1) / TB, kRouteThreads, smem, st>>>((const XT*)x, (const XT*)wr, bias, c.T, c.H, c.E, c.K,
+                                                          c.renormalize, topk_idx, topk_w);
+  p->launches += 1;
+  return (int)cudaGetLastError();
+}
+
 template <typename XT>
 static int launch_typed(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
                         float* topk_w, cudaStream_t st) {
   const moe_config_t& c = p->cfg;
-  if (c.E <= 8) return launch_cfg<XT, 8, 1, 32, 1>(p, x, wr, bias, topk_idx, topk_w, st);
-  if (c.E <= 64) return launch_cfg<XT, 16, 4, 16, 1>(p, x, wr, bias, topk_idx, topk_w, st);
-  if (c.T >= 2048) return launch_cfg<XT, 32, 8, 8, 8>(p, x, wr, bias, topk_idx, topk_w, st);
-  return launch_cfg<XT, 32, 8, 8, 2>(p, x, wr, bias, topk_idx, topk_w, st);
+  // Small E is bound by the latency of the chain: one lane per chain, long chunks.
+  if (c.E <= 8) return launch_narrow<XT, 8, 1, 512>(p, x, wr, bias, topk_idx, topk_w, st);
+  if (c.E <= 16) return launch_narrow<XT, 16, 1, 512>(p, x, wr, bias, topk_idx, topk_w, st);
+  if (c.E <= 32) return launch_narrow<XT, 32, 1, 512>(p, x, wr, bias, topk_idx, topk_w, st);
+  if (c.E <= 64) return launch_narrow<XT, 32, 2, 256>(p, x, wr, bias, topk_idx, topk_w, st);
+  return launch_wide<XT>(p, x, wr, bias, topk_idx, topk_w, st);
 }
 
 int launch_route(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
