@@ -62,11 +62,13 @@ size_t carve(const moe_config_t& c, const Geometry& g, char* base, Scratch* s, s
   };
   Scratch t;
   memset(&t, 0, sizeof t);
-  // leading block, cleared by every dispatch: status, pool_next, scan_ticket
+  // leading block, cleared by every dispatch: status, pool_next, scan_ticket, rows_done
   t.status = (int*)take(sizeof(int) * 4);
   t.pool_next = (int*)take(sizeof(int));
   t.scan_ticket = (int*)take(sizeof(int));
+  t.rows_done = (int*)take(sizeof(int));
   if (counters_bytes) *counters_bytes = off;
+  t.tile_count = (int*)take(sizeof(int) * (size_t)(g.P > 0 ? g.P : 1));
   t.tile_table = (int*)take(sizeof(int) * (size_t)c.E * g.tiles_per_expert);
   t.cta_count = (int*)take(sizeof(int) * (size_t)(g.nblk > 0 ? g.nblk : 1) * c.E);
   t.cta_base = (int*)take(sizeof(int) * (size_t)(g.nblk > 0 ? g.nblk : 1) * c.E);
@@ -181,9 +183,9 @@ int moe_dispatch(moe_plan_t* p, const void* d_x, const int32_t* d_topk_idx, void
 }
 
 static int ffn_dispatch(moe_plan* p, const void* recv, const int* tile_expert, const void* wg, const void* wu,
-                        const void* wd, void* out_rows, cudaStream_t st) {
+                        const void* wd, void* out_rows, bool gate_on_dispatch, cudaStream_t st) {
   if (p->cfg.dtype == MOE_DTYPE_BF16 && p->cfg.ffn_kernel == 0)
-    return launch_ffn_tc(p, recv, tile_expert, wg, wu, wd, out_rows, st);
+    return launch_ffn_tc(p, recv, tile_expert, wg, wu, wd, out_rows, gate_on_dispatch, st);
   return launch_ffn_simt(p, recv, tile_expert, wg, wu, wd, out_rows, st);
 }
 
@@ -194,7 +196,7 @@ int moe_expert_ffn(moe_plan_t* p, const void* d_recv, const int32_t* d_tile_expe
   if (misaligned(d_recv) || misaligned(d_wg) || misaligned(d_wu) || misaligned(d_wd) || misaligned(d_out_rows))
     return MOE_ERR_ALIGN;
   p->launches = 0;
-  int rc = ffn_dispatch(p, d_recv, d_tile_expert, d_wg, d_wu, d_wd, d_out_rows, (cudaStream_t)stream);
+  int rc = ffn_dispatch(p, d_recv, d_tile_expert, d_wg, d_wu, d_wd, d_out_rows, false, (cudaStream_t)stream);
   return rc == 0 ? MOE_OK : (rc < 0 ? rc : MOE_ERR_CUDA);
 }
 
@@ -225,7 +227,7 @@ int moe_layer(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_b
     return MOE_ERR_CUDA;
   mark(p, 2, st);
   if (!p->cfg.identity_experts) {
-    int rc = ffn_dispatch(p, s.recv, s.tile_expert, d_wg, d_wu, d_wd, s.out_rows, st);
+    int rc = ffn_dispatch(p, s.recv, s.tile_expert, d_wg, d_wu, d_wd, s.out_rows, true, st);
     if (rc != 0) return rc < 0 ? rc : MOE_ERR_CUDA;
   } else {
     mark(p, 3, st);

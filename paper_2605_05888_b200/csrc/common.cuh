@@ -30,6 +30,8 @@ struct Scratch {          // device pointers carved out of the caller's workspac
   int* status;            // [4]
   int* pool_next;         // [1]   paged mode: next free tile
   int* scan_ticket;       // [1]   mode 0: CTAs of the scan kernel that finished
+  int* rows_done;         // [1]   assignments whose rows are stored (global completion counter)
+  int* tile_count;        // [P]   rows stored per tile (per-tile status counter)
   int* tile_table;        // [E * tiles_per_expert] paged mode: expert-local tile -> pool tile
   int* cta_count;         // [nblk * E] mode 0: per token-block histogram
   int* cta_base;          // [nblk * E] mode 0: exclusive prefix inside the expert
@@ -89,8 +91,10 @@ int launch_combine(moe_plan* p, const void* rows, const int* slot_of, const floa
                    cudaStream_t st);
 int launch_ffn_simt(moe_plan* p, const void* recv, const int* tile_expert, const void* wg,
                     const void* wu, const void* wd, void* out_rows, cudaStream_t st);
+// gate_on_dispatch: the GEMM1 producer waits for the dispatch counters of this plan (tile_count,
+// rows_done) before it reads a tile; false when the rows come from somewhere else.
 int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const void* wg,
-                  const void* wu, const void* wd, void* out_rows, cudaStream_t st);
+                  const void* wu, const void* wd, void* out_rows, bool gate_on_dispatch, cudaStream_t st);
 
 // ---- element helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ float to_float(float v) { return v; }

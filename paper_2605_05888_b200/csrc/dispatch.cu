@@ -55,6 +55,26 @@ __device__ __forceinline__ void copy_rows(const uint4* __restrict__ x, uint4* __
 }
 
 // ------------------------------------------------------------------------------------------------
+// Availability signalling (the software form of the paper's data availability manager, Section
+// IV-D): after a block's rows are stored, every 128-row tile it wrote into gets its status counter
+// raised by the number of rows (release), and the global counter by the block's assignments.  A
+// consumer may read a tile once its counter shows 128 rows, or once the global counter shows all
+// T*K assignments (partly filled last tiles are then final; tiles at zero never become work).
+__device__ __forceinline__ void signal_rows(const int* s_slot, int na, int* __restrict__ tile_count,
+                                            int* __restrict__ rows_done) {
+  asm volatile("fence.proxy.async.global;" ::: "memory");  // consumers read the rows through TMA
+  __threadfence();
+  __syncthreads();
+  const int a = threadIdx.x;
+  const int slot = a < na ? s_slot[a] : -1;
+  const int tile = slot >= 0 ? slot / kTileRows : -1;
+  const unsigned peers = __match_any_sync(0xffffffffu, tile);
+  if (tile >= 0 && (threadIdx.x % 32) == __ffs(peers) - 1)
+    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(tile_count + tile), "r"(__popc(peers)) : "memory");
+  if (threadIdx.x == 0) asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(rows_done), "r"(na) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
 // Mode 0, kernel 1: histogram of one token block.  cta_count[blk][e].
 __global__ void __launch_bounds__(kDispThreads)
 hist_kernel(const int* __restrict__ topk_idx, int T, int E, int K, int tok_per_blk,
@@ -138,7 +158,7 @@ __global__ void __launch_bounds__(kDispThreads)
 scatter_kernel(const uint4* __restrict__ x, const int* __restrict__ topk_idx, int T, int E, int K,
                int tok_per_blk, int vec_per_row, const int* __restrict__ cta_base,
                const int* __restrict__ tile_base, uint4* __restrict__ recv, int* __restrict__ src_info,
-               int* __restrict__ slot_of) {
+               int* __restrict__ slot_of, int* __restrict__ tile_count, int* __restrict__ rows_done) {
   extern __shared__ int smem_i[];
   int* s_wcnt = smem_i;                          // [8][E] per-warp counts
   int* s_slot = smem_i + (kDispThreads / 32) * E;  // [kMaxAssign]
@@ -167,6 +187,7 @@ scatter_kernel(const uint4* __restrict__ x, const int* __restrict__ topk_idx, in
   }
   __syncthreads();
   copy_rows<4>(x, recv, s_slot, t0, ntok, K, vec_per_row);
+  signal_rows(s_slot, na, tile_count, rows_done);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -178,7 +199,8 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
                        unsigned long long spin_limit, int* __restrict__ row_pointer,
                        int* __restrict__ tile_table, int* __restrict__ pool_next,
                        int* __restrict__ tile_expert, uint4* __restrict__ recv, int* __restrict__ src_info,
-                       int* __restrict__ slot_of, int* __restrict__ status) {
+                       int* __restrict__ slot_of, int* __restrict__ status, int* __restrict__ tile_count,
+                       int* __restrict__ rows_done) {
   extern __shared__ int smem_i[];
   int* s_cnt = smem_i;        // [E] rows this block sends to expert e
   int* s_base = smem_i + E;   // [E] first LocalRowID this block got from expert e's row pointer
@@ -257,6 +279,7 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
   }
   __syncthreads();
   copy_rows<4>(x, recv, s_slot, t0, ntok, K, vec_per_row);
+  if (tile_count != nullptr) signal_rows(s_slot, na, tile_count, rows_done);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -264,12 +287,15 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
 __global__ void __launch_bounds__(kDispThreads)
 reset_kernel(int* __restrict__ counters, int n_counters, int* __restrict__ expert_count, int E,
              int* __restrict__ tile_expert, int P, int* __restrict__ src_info, int n_src,
-             int* __restrict__ tile_table, int n_table) {
+             int* __restrict__ tile_table, int n_table, int* __restrict__ tile_count) {
   const int stride = gridDim.x * kDispThreads;
   const int i0 = blockIdx.x * kDispThreads + threadIdx.x;
   for (int i = i0; i < n_counters; i += stride) counters[i] = 0;
   for (int i = i0; i < E; i += stride) expert_count[i] = 0;
-  for (int i = i0; i < P; i += stride) tile_expert[i] = -1;
+  for (int i = i0; i < P; i += stride) {
+    tile_expert[i] = -1;
+    tile_count[i] = 0;
+  }
   for (int i = i0; i < n_table; i += stride) tile_table[i] = -1;
   for (int i = i0; i < n_src; i += stride) src_info[i] = -1;
 }
@@ -288,7 +314,7 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
     const int grid = (int)max(1ll, (most + 4 * kDispThreads - 1) / (4 * kDispThreads));
     reset_kernel<<<grid, kDispThreads, 0, st>>>(p->s.status, (int)(p->counters_bytes / sizeof(int)), expert_count,
                                                 c.E, tile_expert, (int)p->P, src_info, (int)(p->P * kTileRows),
-                                                p->s.tile_table, table);
+                                                p->s.tile_table, table, p->s.tile_count);
     p->launches += 1;
   }
   if (c.T == 0) return 0;
@@ -300,7 +326,7 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
     const size_t smem = sizeof(int) * ((kDispThreads / 32) * c.E + kMaxAssign);
     scatter_kernel<<<nblk, kDispThreads, smem, st>>>((const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row,
                                                      p->s.cta_base, p->s.tile_base, (uint4*)recv, src_info,
-                                                     slot_of);
+                                                     slot_of, p->s.tile_count, p->s.rows_done);
     p->launches += 3;
   } else {
     const size_t smem = sizeof(int) * (2 * c.E + kMaxAssign);
@@ -309,12 +335,12 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
       dispatch_atomic_kernel<true><<<nblk, kDispThreads, smem, st>>>(
           (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row, (int)p->cap_rows, (int)p->P,
           p->tiles_per_expert, spin, expert_count, p->s.tile_table, p->s.pool_next, tile_expert, (uint4*)recv,
-          src_info, slot_of, p->s.status);
+          src_info, slot_of, p->s.status, p->s.tile_count, p->s.rows_done);
     else
       dispatch_atomic_kernel<false><<<nblk, kDispThreads, smem, st>>>(
           (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row, (int)p->cap_rows, (int)p->P,
           p->tiles_per_expert, spin, expert_count, p->s.tile_table, p->s.pool_next, tile_expert, (uint4*)recv,
-          src_info, slot_of, p->s.status);
+          src_info, slot_of, p->s.status, p->s.tile_count, p->s.rows_done);
     p->launches += 1;
   }
   return (int)cudaGetLastError();
@@ -404,6 +430,7 @@ extern "C" int moe_dispatch_noalloc(const moe_config_t* cfg, const void* d_x, co
   const unsigned long long spin = c.spin_limit ? c.spin_limit : (1ull << 22);
   dispatch_atomic_kernel<true><<<nblk, kDispThreads, smem, st>>>(
       (const uint4*)d_x, d_topk_idx, c.T, c.E, c.K, tpb, c.H * eb / 16, 0, (int)P, tiles_per_expert, spin,
-      d_expert_count, tile_table, pool_next, d_tile_expert, (uint4*)d_recv, d_src_info, d_slot_of, d_status);
+      d_expert_count, tile_table, pool_next, d_tile_expert, (uint4*)d_recv, d_src_info, d_slot_of, d_status,
+      nullptr, nullptr);
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

@@ -221,6 +221,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
               const int* __restrict__ expert_start, const int* __restrict__ seg_start,
               const int* __restrict__ seg_info, const int* __restrict__ meta, int phase, int E, int F, int H,
               __nv_bfloat16* __restrict__ inter, __nv_bfloat16* __restrict__ out, int* __restrict__ gemm1_done,
+              const int* __restrict__ tile_count, const int* __restrict__ rows_done, int total_rows,
               int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* stage_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -292,6 +293,19 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       for (int s = 0; s < kStages; ++s) armed[s] = 0;
       for (int item = first_item; item < item_end && !fail_site; item += gridDim.x) {
         const Item it = decode(item);
+        if (it.type == 0 && tile_count != nullptr) {
+          // Availability of this tile's rows (dispatch side): 128 rows stored, or every assignment of
+          // the batch stored (then a partly filled tile is final).
+          if (ld_acquire(&tile_count[it.tile]) < kTileRows && ld_acquire(rows_done) < total_rows) {
+            const unsigned long long t0 = globaltimer();
+            while (ld_acquire(&tile_count[it.tile]) < kTileRows && ld_acquire(rows_done) < total_rows) {
+              if (*abort_flag || globaltimer() - t0 > kWaitNs) { fail_site = kWaitTileReady; break; }
+              __nanosleep(64);
+            }
+            if (fail_site) break;
+          }
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+        }
         if (it.type == 1) {
           // Availability of this tile's intermediate: every epilogue warp of every GEMM1 block bumps
           // the tile's counter once.  Bounded wait, then order the async proxy behind what was seen.
@@ -487,7 +501,7 @@ static int make_map_3d(EncodeTiledFn enc, CUtensorMap* m, const void* base, uint
 }
 
 int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const void* wg, const void* wu,
-                  const void* wd, void* out_rows, cudaStream_t st) {
+                  const void* wd, void* out_rows, bool gate_on_dispatch, cudaStream_t st) {
   const moe_config_t& c = p->cfg;
   if (p->P == 0 || c.T == 0) return 0;
   EncodeTiledFn enc;
@@ -519,7 +533,8 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
     ffn_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(a1, bg, bu, a2, bd, p->s.tile_list, p->s.expert_start,
                                                      p->s.seg_start, p->s.seg_info, p->s.work_meta, phase, c.E, c.F,
                                                      c.H, (__nv_bfloat16*)p->s.inter, (__nv_bfloat16*)out_rows,
-                                                     p->s.gemm1_done, p->s.status);
+                                                     p->s.gemm1_done, gate_on_dispatch ? p->s.tile_count : nullptr,
+                                                     p->s.rows_done, c.T * c.K, p->s.status);
   };
   if (fused) {
     launch(0);
