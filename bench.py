@@ -201,7 +201,8 @@ def run_cuda(args, w: inputs.Workload) -> None:
     el = torch.bfloat16 if w.dtype == inputs.BF16 else torch.float32
     mode = {"scan": B.DISPATCH_SCAN, "static": B.DISPATCH_ATOMIC_STATIC, "paged": B.DISPATCH_ATOMIC_PAGED}[args.dispatch]
     plan = B.Plan(B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype, dispatch_mode=mode,
-                                identity_experts=int(w.identity_experts), ffn_split=int(args.ffn_split)))
+                                identity_experts=int(w.identity_experts), ffn_split=int(args.ffn_split),
+                                ffn_kernel=args.ffn_kernel))
     y = torch.empty((w.T, w.H), dtype=el, device="cuda")
     stream = torch.cuda.current_stream()
 
@@ -335,6 +336,8 @@ def main() -> None:
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
     ap.add_argument("--dispatch", default="paged", choices=["scan", "static", "paged"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ffn-kernel", type=int, default=0, choices=[0, 1, 2],
+                    help="0: tcgen05 one CTA per tile (default), 2: tcgen05 CTA pairs, 1: SIMT check path")
     ap.add_argument("--ffn-split", action="store_true", help="one launch per expert GEMM instead of one for both")
     args = ap.parse_args()
     w = WORKLOADS[args.workload]

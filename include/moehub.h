@@ -70,8 +70,10 @@ typedef struct {
   int32_t renormalize;          /* 0: w = softmax prob. of the picked experts; 1: / their sum */
   int32_t dispatch_mode;        /* MOE_DISPATCH_*                                            */
   int32_t identity_experts;     /* 1: moe_layer skips the FFN (expert output = expert input)  */
-  int32_t ffn_kernel;           /* 0: tensor-core (tcgen05) kernel for bf16, SIMT for fp32;
-                                   1: SIMT fp32-FMA kernel for either dtype (check path)      */
+  int32_t ffn_kernel;           /* 0: tensor-core (tcgen05) kernel, one CTA per tile, for bf16,
+                                   SIMT for fp32; 1: SIMT fp32-FMA kernel for either dtype
+                                   (check path); 2: tensor-core kernel on CTA pairs
+                                   (cta_group::2, two tiles per MMA; bf16)                    */
   int32_t ffn_split;            /* 0: both expert GEMMs in one persistent launch (per-tile status
                                    counters gate GEMM2); 1: one launch per GEMM                 */
   int64_t capacity_rows;        /* mode 1: rows per expert region, multiple of 128, 0 = T

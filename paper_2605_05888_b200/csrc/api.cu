@@ -184,7 +184,7 @@ int moe_dispatch(moe_plan_t* p, const void* d_x, const int32_t* d_topk_idx, void
 
 static int ffn_dispatch(moe_plan* p, const void* recv, const int* tile_expert, const void* wg, const void* wu,
                         const void* wd, void* out_rows, bool gate_on_dispatch, cudaStream_t st) {
-  if (p->cfg.dtype == MOE_DTYPE_BF16 && p->cfg.ffn_kernel == 0)
+  if (p->cfg.dtype == MOE_DTYPE_BF16 && p->cfg.ffn_kernel != 1)
     return launch_ffn_tc(p, recv, tile_expert, wg, wu, wd, out_rows, gate_on_dispatch, st);
   return launch_ffn_simt(p, recv, tile_expert, wg, wu, wd, out_rows, st);
 }

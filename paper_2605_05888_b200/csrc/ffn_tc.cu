@@ -27,118 +27,19 @@
 // warps 2-5 = epilogue (TMEM lane quarter = warp % 4).  Every wait is bounded in time; on expiry
 // the CTA records MOE_ERR_TIMEOUT, drains its outstanding TMA copies (bounded), frees its TMEM and
 // returns.
-#include <cuda.h>
-
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace moehub {
-
-constexpr int kTcThreads = 192;
-constexpr int kStages = 4;
-constexpr int kBK = 64;                       // k elements per stage (128 bytes of bf16)
-constexpr int kUmmaN = 256;
-constexpr int kABytes = kTileRows * kBK * 2;  // 16 KB
-constexpr int kBBytes = kUmmaN * kBK * 2;     // 32 KB
-constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kTcSmem = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr unsigned long long kWaitNs = 2000000000ull;  // 2 s bound on any single wait
-
-// ---- PTX wrappers ---------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long globaltimer() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false when the time limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (mbar_try(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer();
-  for (unsigned it = 1;; ++it) {
-    if (mbar_try(bar, parity)) return true;
-    if ((it & 31u) == 0u) {
-      if (*abort_flag) return false;
-      if (globaltimer() - t0 > kWaitNs) return false;
-    }
-  }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
-                                            int c2) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                       uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t* r) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 bf16) in the
-// 128-byte swizzle: 8-row groups are 1024 bytes apart.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
-  uint64_t d = 0;
-  d |= (uint64_t)((addr >> 4) & 0x3fff);   // start address, 16-byte units
-  d |= (uint64_t)1 << 16;                  // leading byte offset (unused with swizzle, K-major)
-  d |= (uint64_t)(1024 >> 4) << 32;        // stride byte offset between 8-row groups
-  d |= (uint64_t)1 << 46;                  // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;                  // 128-byte swizzle
-  return d;
-}
-// Instruction descriptor: bf16 x bf16 -> fp32, A and B K-major, M = 128, N = 256.
-constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kUmmaN >> 3) << 17) |
-                            ((uint32_t)(kTileRows >> 4) << 24);
 
 // ---- work list ------------------------------------------------------------------------------
 // tile_list: the used tiles grouped by expert; expert_start[e]: first index of expert e's tiles,
 // expert_start[E] = number of used tiles.  Segments: the item sequence is a list of at most 2E
 // segments, segment = all GEMM1 items or all GEMM2 items of one expert; seg_start[i] is the first
 // item of segment i (seg_start[2E] = number of items), seg_info[i] = expert | type << 16
-// (type 0: GEMM1, 1: GEMM2).  meta[0] = number of items that precede the first GEMM2 item when the
+// (type 0: GEMM1, 1: GEMM2).  pair = 2 counts one item per PAIR of tiles (CTA-pair kernel).  meta[0] = number of items that precede the first GEMM2 item when the
 // launch is split in two phases.
-constexpr int kMaxExperts = 256;
-
 __global__ void __launch_bounds__(256)
-worklist_kernel(const int* __restrict__ tile_expert, int P, int E, int NB1, int NB2, int lag, int fused,
+worklist_kernel(const int* __restrict__ tile_expert, int P, int E, int NB1, int NB2, int lag, int fused, int pair,
                 int* __restrict__ tile_list, int* __restrict__ expert_start, int* __restrict__ seg_start,
                 int* __restrict__ seg_info, int* __restrict__ meta, int* __restrict__ gemm1_done) {
   __shared__ int s_cnt[kMaxExperts];
@@ -180,12 +81,12 @@ worklist_kernel(const int* __restrict__ tile_expert, int P, int E, int NB1, int 
     for (int e = 0; e < E; ++e) {
       seg_start[nseg] = pos;
       seg_info[nseg++] = e;
-      pos += s_cnt[e] * NB1;
+      pos += (s_cnt[e] + pair - 1) / pair * NB1;
       s_cur[e] = pos;  // end of this expert's GEMM1 items
       while (fused && q < e && pos - s_cur[q] >= lag) {
         seg_start[nseg] = pos;
         seg_info[nseg++] = q | (1 << 16);
-        pos += s_cnt[q] * NB2;
+        pos += (s_cnt[q] + pair - 1) / pair * NB2;
         ++q;
       }
     }
@@ -193,7 +94,7 @@ worklist_kernel(const int* __restrict__ tile_expert, int P, int E, int NB1, int 
     for (; q < E; ++q) {
       seg_start[nseg] = pos;
       seg_info[nseg++] = q | (1 << 16);
-      pos += s_cnt[q] * NB2;
+      pos += (s_cnt[q] + pair - 1) / pair * NB2;
     }
     seg_start[nseg] = pos;  // nseg == 2E
   }
@@ -209,20 +110,23 @@ struct TcShared {
   int abort_flag;
 };
 
-struct Item {
-  int type;   // 0: GEMM1 (+SwiGLU), 1: GEMM2
-  int e, nb, tile;
-};
-
 __global__ void __launch_bounds__(kTcThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_bg,
               const __grid_constant__ CUtensorMap map_bu, const __grid_constant__ CUtensorMap map_a2,
-              const __grid_constant__ CUtensorMap map_bd, const int* __restrict__ tile_list,
-              const int* __restrict__ expert_start, const int* __restrict__ seg_start,
-              const int* __restrict__ seg_info, const int* __restrict__ meta, int phase, int E, int F, int H,
-              __nv_bfloat16* __restrict__ inter, __nv_bfloat16* __restrict__ out, int* __restrict__ gemm1_done,
-              const int* __restrict__ tile_count, const int* __restrict__ rows_done, int total_rows,
-              int* __restrict__ status) {
+              const __grid_constant__ CUtensorMap map_bd, const FfnParams prm) {
+  const int* __restrict__ tile_list = prm.tile_list;
+  const int* __restrict__ expert_start = prm.expert_start;
+  const int* __restrict__ seg_start = prm.seg_start;
+  const int* __restrict__ seg_info = prm.seg_info;
+  const int* __restrict__ meta = prm.meta;
+  const int phase = prm.phase, E = prm.E, F = prm.F, H = prm.H;
+  __nv_bfloat16* __restrict__ inter = prm.inter;
+  __nv_bfloat16* __restrict__ out = prm.out;
+  int* __restrict__ gemm1_done = prm.gemm1_done;
+  const int* __restrict__ tile_count = prm.tile_count;
+  const int* __restrict__ rows_done = prm.rows_done;
+  const int total_rows = prm.total_rows;
+  int* __restrict__ status = prm.status;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* stage_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   TcShared* sh = reinterpret_cast<TcShared*>(stage_base + kStages * kStageBytes);
@@ -513,7 +417,7 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   if ((rc = make_map_3d(enc, &bg, wg, c.E, c.F, c.H, 128)) != MOE_OK) return rc;
   if ((rc = make_map_3d(enc, &bu, wu, c.E, c.F, c.H, 128)) != MOE_OK) return rc;
   if ((rc = make_map_2d(enc, &a2, p->s.inter, pool_rows, c.F, kTileRows)) != MOE_OK) return rc;
-  if ((rc = make_map_3d(enc, &bd, wd, c.E, c.H, c.F, 256)) != MOE_OK) return rc;
+  if ((rc = make_map_3d(enc, &bd, wd, c.E, c.H, c.F, c.ffn_kernel == 2 ? 128 : 256)) != MOE_OK) return rc;
 
   static bool attr_done = false;  // per-process, idempotent
   if (!attr_done) {
@@ -525,24 +429,41 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   const int NB1 = (c.F + 127) / 128, NB2 = (c.H + 255) / 256;
   // One launch for both GEMMs, except under moe_layer_timed, which wants a time for each.
   const int fused = (p->timing || c.ffn_split) ? 0 : 1;
-  worklist_kernel<<<1, 256, 0, st>>>(tile_expert, (int)p->P, c.E, NB1, NB2, 2 * grid, fused, p->s.tile_list,
-                                     p->s.expert_start, p->s.seg_start, p->s.seg_info, p->s.work_meta,
-                                     p->s.gemm1_done);
+  const bool pairs = c.ffn_kernel == 2;  // opt-in: the CTA-pair kernel
+  const int workers = pairs ? grid / 2 : grid;
+  worklist_kernel<<<1, 256, 0, st>>>(tile_expert, (int)p->P, c.E, NB1, NB2, 2 * workers, fused, pairs ? 2 : 1,
+                                     p->s.tile_list, p->s.expert_start, p->s.seg_start, p->s.seg_info,
+                                     p->s.work_meta, p->s.gemm1_done);
   mark(p, 3, st);
-  auto launch = [&](int phase) {
-    ffn_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(a1, bg, bu, a2, bd, p->s.tile_list, p->s.expert_start,
-                                                     p->s.seg_start, p->s.seg_info, p->s.work_meta, phase, c.E, c.F,
-                                                     c.H, (__nv_bfloat16*)p->s.inter, (__nv_bfloat16*)out_rows,
-                                                     p->s.gemm1_done, gate_on_dispatch ? p->s.tile_count : nullptr,
-                                                     p->s.rows_done, c.T * c.K, p->s.status);
+  FfnParams prm;
+  prm.tile_list = p->s.tile_list;
+  prm.expert_start = p->s.expert_start;
+  prm.seg_start = p->s.seg_start;
+  prm.seg_info = p->s.seg_info;
+  prm.meta = p->s.work_meta;
+  prm.E = c.E;
+  prm.F = c.F;
+  prm.H = c.H;
+  prm.inter = (__nv_bfloat16*)p->s.inter;
+  prm.out = (__nv_bfloat16*)out_rows;
+  prm.gemm1_done = p->s.gemm1_done;
+  prm.tile_count = gate_on_dispatch ? p->s.tile_count : nullptr;
+  prm.rows_done = p->s.rows_done;
+  prm.total_rows = c.T * c.K;
+  prm.status = p->s.status;
+  auto launch = [&](int phase) -> int {
+    prm.phase = phase;
+    if (pairs) return launch_ffn_tc2_kernel(a1, bg, bu, a2, bd, prm, grid, st);
+    ffn_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(a1, bg, bu, a2, bd, prm);
+    return cudaGetLastError() == cudaSuccess ? 0 : MOE_ERR_CUDA;
   };
   if (fused) {
-    launch(0);
+    if ((rc = launch(0)) != 0) return rc;
     p->launches += 2;
   } else {
-    launch(1);
+    if ((rc = launch(1)) != 0) return rc;
     mark(p, 4, st);
-    launch(2);
+    if ((rc = launch(2)) != 0) return rc;
     p->launches += 3;
   }
   return cudaGetLastError() == cudaSuccess ? 0 : MOE_ERR_CUDA;
