@@ -226,6 +226,7 @@ def run_cuda(args, w: inputs.Workload) -> None:
     # ---- timed region: K steps, device-resident inputs ----
     sampler = ClockSampler(local)
     barrier()
+    plan.moe_ffn_clock_mhz(reset=True)
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
@@ -235,6 +236,8 @@ def run_cuda(args, w: inputs.Workload) -> None:
     torch.cuda.synchronize()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop()
+    # SM clock the tensor-core expert kernel really ran at (cycles / time measured inside the kernel)
+    clocks["ffn_kernel_sm_mhz"] = round(plan.moe_ffn_clock_mhz(reset=True), 1)
     barrier()
 
     # ---- per-kernel device times: the same steps with an event after every kernel ----

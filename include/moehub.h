@@ -191,6 +191,12 @@ int moe_layer_timed(moe_plan_t* plan, const void* d_x, const void* d_wr, const f
  * 4 tile_expert, 5 src_info, 6 slot_of, 7 out_rows. */
 int moe_layer_buffer(moe_plan_t* plan, int which, void** out_ptr);
 
+/* Effective SM clock inside the tensor-core expert kernels since the last reset: one CTA of every
+ * launch accumulates its elapsed SM cycles and nanoseconds; *out_mhz = cycles / time (0 if none ran).
+ * Synchronises `stream` when out_mhz is given; reset != 0 clears the accumulators afterwards.
+ * For measurement: tells a kernel slowed by a power-capped clock from one that waits for data. */
+int moe_ffn_clock_mhz(moe_plan_t* plan, void* stream, int reset, float* out_mhz);
+
 /* Number of kernels the last stage call (or moe_layer) launched. */
 int moe_last_launch_count(moe_plan_t* plan, int32_t* out);
 

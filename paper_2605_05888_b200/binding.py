@@ -23,7 +23,7 @@ STAGES = ["route", "dispatch", "worklist", "gemm1", "gemm2", "combine"]
 
 EXPORTS = ["moe_dispatch_noalloc", "moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
            "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host", "moe_layer_timed", "moe_layer_buffer",
-           "moe_last_launch_count", "moe_last_status", "moe_strerror"]
+           "moe_ffn_clock_mhz", "moe_last_launch_count", "moe_last_status", "moe_strerror"]
 
 
 class MoeConfig(ctypes.Structure):
@@ -62,6 +62,7 @@ def lib() -> ctypes.CDLL:
         L.moe_layer_host.argtypes = [vp] * 9
         L.moe_layer_timed.argtypes = [vp] * 9 + [ctypes.POINTER(ctypes.c_float)]
         L.moe_layer_buffer.argtypes = [vp, ctypes.c_int, ctypes.POINTER(vp)]
+        L.moe_ffn_clock_mhz.argtypes = [vp, vp, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
         L.moe_last_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
         L.moe_last_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
         L.moe_strerror.argtypes = [ctypes.c_int]
@@ -186,6 +187,11 @@ class Plan:
     def moe_layer_buffer(self, which: int) -> int:
         out = ctypes.c_void_p()
         _check(lib().moe_layer_buffer(self.handle, which, ctypes.byref(out)), "moe_layer_buffer")
+        return out.value
+
+    def moe_ffn_clock_mhz(self, reset: bool = True, stream=None) -> float:
+        out = ctypes.c_float()
+        _check(lib().moe_ffn_clock_mhz(self.handle, _stream(stream), int(reset), ctypes.byref(out)), "moe_ffn_clock_mhz")
         return out.value
 
     def moe_last_launch_count(self) -> int:

@@ -78,6 +78,7 @@ size_t carve(const moe_config_t& c, const Geometry& g, char* base, Scratch* s, s
   t.seg_start = (int*)take(sizeof(int) * (size_t)(2 * c.E + 1));
   t.seg_info = (int*)take(sizeof(int) * (size_t)(2 * c.E));
   t.work_meta = (int*)take(sizeof(int) * 4);
+  t.clock_probe = (unsigned long long*)take(sizeof(unsigned long long) * 2);
   t.gemm1_done = (int*)take(sizeof(int) * (size_t)(g.P > 0 ? g.P : 1));
   const size_t pool_rows = (size_t)g.P * kTileRows;
   if (!c.identity_experts) t.inter = take(pool_rows * c.F * g.eb);
@@ -147,7 +148,8 @@ int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, mo
     return MOE_ERR_CUDA;
   }
   // The status word must start clean even if a stage other than dispatch is called first.
-  if (cudaMemset(p->s.status, 0, p->counters_bytes) != cudaSuccess) {
+  if (cudaMemset(p->s.status, 0, p->counters_bytes) != cudaSuccess ||
+      cudaMemset(p->s.clock_probe, 0, 2 * sizeof(unsigned long long)) != cudaSuccess) {
     delete p;
     return MOE_ERR_CUDA;
   }
@@ -275,6 +277,20 @@ int moe_layer_buffer(moe_plan_t* p, int which, void** out_ptr) {
   void* tab[8] = {s.topk_idx, s.topk_w, s.recv, s.expert_count, s.tile_expert, s.src_info, s.slot_of, s.out_rows};
   if (which < 0 || which >= 8) return MOE_ERR_ARG;
   *out_ptr = tab[which];
+  return MOE_OK;
+}
+
+int moe_ffn_clock_mhz(moe_plan_t* p, void* stream, int reset, float* out_mhz) {
+  if (!p) return MOE_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned long long host[2] = {0, 0};
+  if (out_mhz) {
+    if (cudaMemcpyAsync(host, p->s.clock_probe, sizeof host, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    *out_mhz = host[1] ? (float)(1e3 * (double)host[0] / (double)host[1]) : 0.0f;
+  }
+  if (reset && cudaMemsetAsync(p->s.clock_probe, 0, sizeof host, st) != cudaSuccess) return MOE_ERR_CUDA;
   return MOE_OK;
 }
 

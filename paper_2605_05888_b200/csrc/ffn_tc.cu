@@ -161,6 +161,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
   volatile int* abort_flag = &sh->abort_flag;
+  ClockProbe probe(prm.clock_probe);
 
   const int NB1 = (F + 127) / 128, NB2 = (H + 255) / 256;
   const int KB1 = (H + kBK - 1) / kBK, KB2 = (F + kBK - 1) / kBK;
@@ -298,7 +299,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       const Item it = decode(item);
       const int acc = local_item & 1;
       const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
-      if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag)) { fail_site = kWaitMbarEpi; break; }
+      if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag, 500)) { fail_site = kWaitMbarEpi; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kUmmaN);
       const size_t row = (size_t)it.tile * kTileRows + row_in_tile;
@@ -357,6 +358,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  probe.finish();
   if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
 }
@@ -451,6 +453,7 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   prm.rows_done = p->s.rows_done;
   prm.total_rows = c.T * c.K;
   prm.status = p->s.status;
+  prm.clock_probe = reinterpret_cast<unsigned long long*>(p->s.clock_probe);
   auto launch = [&](int phase) -> int {
     prm.phase = phase;
     if (pairs) return launch_ffn_tc2_kernel(a1, bg, bu, a2, bd, prm, grid, st);

@@ -127,6 +127,7 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
   tc_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
   volatile int* abort_flag = &sh->abort_flag;
+  ClockProbe probe(prm.clock_probe);
 
   const int NB1 = (F + 127) / 128, NB2 = (H + 255) / 256;
   const int KB1 = (H + kBK - 1) / kBK, KB2 = (F + kBK - 1) / kBK;
@@ -257,7 +258,7 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
       const Item it = decode(item, fill);
       const int acc = local_item & 1;
       const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
-      if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag)) { fail_site = kWaitMbarEpi; break; }
+      if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag, 500)) { fail_site = kWaitMbarEpi; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kUmmaN);
       if (it.tile >= 0) {
@@ -318,6 +319,7 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
   __syncthreads();
   cluster_sync_all();  // neither CTA leaves while its partner may still touch its shared memory or TMEM
   tc_fence_after();
+  probe.finish();
   if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
 }

@@ -42,10 +42,14 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false when the time limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+// sleep_ns > 0 backs off between polls: for waits that are long by design (an epilogue warp waiting
+// for a whole main loop) polling at full rate only burns power the tensor pipe could use.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned sleep_ns = 0) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = globaltimer();
   for (unsigned it = 1;; ++it) {
+    if (sleep_ns) __nanosleep(sleep_ns);
     if (mbar_try(bar, parity)) return true;
     if ((it & 31u) == 0u) {
       if (*abort_flag) return false;
@@ -123,6 +127,26 @@ struct FfnParams {
   const int* rows_done;
   int total_rows;
   int* status;
+  unsigned long long* clock_probe;  // [2]: SM cycles and nanoseconds CTA 0 spent in the kernel (accumulated)
+};
+
+// Effective SM clock while a kernel runs: CTA 0 adds its elapsed %clock64 and %globaltimer.
+struct ClockProbe {
+  unsigned long long* out;
+  long long c0;
+  unsigned long long t0;
+  __device__ explicit ClockProbe(unsigned long long* o) : out(o), c0(0), t0(0) {
+    if (out != nullptr && blockIdx.x == 0 && threadIdx.x == 0) {
+      c0 = clock64();
+      t0 = globaltimer();
+    }
+  }
+  __device__ void finish() {
+    if (out != nullptr && blockIdx.x == 0 && threadIdx.x == 0) {
+      atomicAdd(out, (unsigned long long)(clock64() - c0));
+      atomicAdd(out + 1, globaltimer() - t0);
+    }
+  }
 };
 
 // The CTA-pair (cta_group::2) kernel lives in ffn_tc2.cu.
