@@ -27,6 +27,8 @@ combine_kernel(const uint4* __restrict__ rows, const int* __restrict__ slot_of,
   const int t = (int)(wid / runs_per_row);
   if (t >= T) return;
   const int v_begin = (int)(wid % runs_per_row) * kCombRun;
+  pdl_wait();
+  pdl_trigger();
   int my_slot = -1;
   float my_w = 0.0f;
   if (lane < K) {
@@ -97,8 +99,8 @@ static int launch_typed(moe_plan* p, const void* rows, const int* slot_of, const
   const long long warps = (long long)c.T * runs_per_row;
   const int grid = (int)((warps + kCombThreads / 32 - 1) / (kCombThreads / 32));
 #define MOEHUB_COMBINE(KT)                                                                          \
-  combine_kernel<XT, KT><<<grid, kCombThreads, 0, st>>>((const uint4*)rows, slot_of, topk_w, c.T, c.K, \
-                                                        vec_per_row, runs_per_row, (uint4*)y)
+  launch_pdl(combine_kernel<XT, KT>, dim3(grid), dim3(kCombThreads), 0, st, (const uint4*)rows, slot_of, topk_w, \
+             c.T, c.K, vec_per_row, runs_per_row, (uint4*)y)
   switch (c.K) {
     case 1: MOEHUB_COMBINE(1); break;
     case 2: MOEHUB_COMBINE(2); break;

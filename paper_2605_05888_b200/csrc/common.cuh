@@ -83,6 +83,28 @@ inline void mark(moe_plan* p, int i, cudaStream_t st) {
   if (p->timing) cudaEventRecord(p->tev[i], st);
 }
 
+// Launch with the programmatic-stream-serialization attribute (see pdl_wait / pdl_trigger).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_maybe_pdl(bool pdl, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                    cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+  return launch_maybe_pdl(true, kern, grid, block, smem, st, static_cast<Args&&>(args)...);
+}
+
 // ---- launchers (defined in the other .cu files); each returns a cudaError_t as int ------------
 int launch_route(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
                  float* topk_w, cudaStream_t st);
@@ -139,6 +161,14 @@ template <> struct Vec16<__nv_bfloat16> {
     return make_uint4(w[0], w[1], w[2], w[3]);
   }
 };
+
+// Programmatic dependent launch: the kernels of the layer (all but the first, the router: starting
+// it while the previous layer call drains measured slower) are launched so that they may start while
+// their predecessor in the stream is still draining.  pdl_wait() blocks until the predecessor has
+// completed and its writes are visible; nothing before it may touch global memory.  pdl_trigger()
+// lets the successor begin launching.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ int ld_acquire(const int* p) {
   int v;

@@ -82,6 +82,8 @@ hist_kernel(const int* __restrict__ topk_idx, int T, int E, int K, int tok_per_b
   extern __shared__ int s_cnt[];  // [E]
   for (int e = threadIdx.x; e < E; e += kDispThreads) s_cnt[e] = 0;
   __syncthreads();
+  pdl_wait();
+  pdl_trigger();
   const int t0 = blockIdx.x * tok_per_blk;
   const int na = min(tok_per_blk, T - t0) * K;
   for (int a = threadIdx.x; a < na; a += kDispThreads) atomicAdd(&s_cnt[topk_idx[(size_t)t0 * K + a]], 1);
@@ -103,6 +105,8 @@ scan_kernel(const int* __restrict__ cta_count, int nblk, int E, int P, int* __re
   const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
   if (threadIdx.x == 0) s_carry = 0;
   __syncthreads();
+  pdl_wait();
+  pdl_trigger();
   for (int b0 = 0; b0 < nblk; b0 += kDispThreads) {
     const int b = b0 + threadIdx.x;
     const int c = (b < nblk) ? cta_count[(size_t)b * E + e] : 0;
@@ -168,6 +172,8 @@ scatter_kernel(const uint4* __restrict__ x, const int* __restrict__ topk_idx, in
   const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
   for (int i = threadIdx.x; i < (kDispThreads / 32) * E; i += kDispThreads) s_wcnt[i] = 0;
   __syncthreads();
+  pdl_wait();
+  pdl_trigger();
   const int a = threadIdx.x;  // one assignment per thread, na <= 256
   int e = -1, wrank = 0;
   if (a < na) e = topk_idx[(size_t)t0 * K + a];
@@ -211,6 +217,8 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
   const int lane = threadIdx.x % 32;
   for (int e = threadIdx.x; e < E; e += kDispThreads) s_cnt[e] = 0;
   __syncthreads();
+  pdl_wait();
+  pdl_trigger();
 
   // (a) rank inside the block: warp-aggregated shared-memory atomics
   const int a = threadIdx.x;
@@ -290,6 +298,8 @@ reset_kernel(int* __restrict__ counters, int n_counters, int* __restrict__ exper
              int* __restrict__ tile_table, int n_table, int* __restrict__ tile_count) {
   const int stride = gridDim.x * kDispThreads;
   const int i0 = blockIdx.x * kDispThreads + threadIdx.x;
+  pdl_wait();
+  pdl_trigger();
   for (int i = i0; i < n_counters; i += stride) counters[i] = 0;
   for (int i = i0; i < E; i += stride) expert_count[i] = 0;
   for (int i = i0; i < P; i += stride) {
@@ -312,35 +322,30 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
     const int table = c.dispatch_mode == MOE_DISPATCH_ATOMIC_PAGED ? c.E * p->tiles_per_expert : 0;
     const long long most = max((long long)p->P * kTileRows, (long long)table);
     const int grid = (int)max(1ll, (most + 4 * kDispThreads - 1) / (4 * kDispThreads));
-    reset_kernel<<<grid, kDispThreads, 0, st>>>(p->s.status, (int)(p->counters_bytes / sizeof(int)), expert_count,
-                                                c.E, tile_expert, (int)p->P, src_info, (int)(p->P * kTileRows),
-                                                p->s.tile_table, table, p->s.tile_count);
+    launch_pdl(reset_kernel, dim3(grid), dim3(kDispThreads), 0, st, p->s.status,
+               (int)(p->counters_bytes / sizeof(int)), expert_count, c.E, tile_expert, (int)p->P, src_info,
+               (int)(p->P * kTileRows), p->s.tile_table, table, p->s.tile_count);
     p->launches += 1;
   }
   if (c.T == 0) return 0;
   const int nblk = p->nblk, tpb = p->dispatch_tokens;
   if (c.dispatch_mode == MOE_DISPATCH_SCAN) {
-    hist_kernel<<<nblk, kDispThreads, sizeof(int) * c.E, st>>>(topk_idx, c.T, c.E, c.K, tpb, p->s.cta_count);
-    scan_kernel<<<c.E, kDispThreads, 0, st>>>(p->s.cta_count, nblk, c.E, (int)p->P, p->s.cta_base, expert_count,
-                                              p->s.tile_base, tile_expert, p->s.scan_ticket);
+    launch_pdl(hist_kernel, dim3(nblk), dim3(kDispThreads), sizeof(int) * c.E, st, topk_idx, c.T, c.E, c.K, tpb,
+               p->s.cta_count);
+    launch_pdl(scan_kernel, dim3(c.E), dim3(kDispThreads), 0, st, p->s.cta_count, nblk, c.E, (int)p->P, p->s.cta_base,
+               expert_count, p->s.tile_base, tile_expert, p->s.scan_ticket);
     const size_t smem = sizeof(int) * ((kDispThreads / 32) * c.E + kMaxAssign);
-    scatter_kernel<<<nblk, kDispThreads, smem, st>>>((const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row,
-                                                     p->s.cta_base, p->s.tile_base, (uint4*)recv, src_info,
-                                                     slot_of, p->s.tile_count, p->s.rows_done);
+    launch_pdl(scatter_kernel, dim3(nblk), dim3(kDispThreads), smem, st, (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb,
+               vec_per_row, p->s.cta_base, p->s.tile_base, (uint4*)recv, src_info, slot_of, p->s.tile_count,
+               p->s.rows_done);
     p->launches += 3;
   } else {
     const size_t smem = sizeof(int) * (2 * c.E + kMaxAssign);
     const unsigned long long spin = c.spin_limit ? c.spin_limit : (1ull << 22);
-    if (c.dispatch_mode == MOE_DISPATCH_ATOMIC_PAGED)
-      dispatch_atomic_kernel<true><<<nblk, kDispThreads, smem, st>>>(
-          (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row, (int)p->cap_rows, (int)p->P,
-          p->tiles_per_expert, spin, expert_count, p->s.tile_table, p->s.pool_next, tile_expert, (uint4*)recv,
-          src_info, slot_of, p->s.status, p->s.tile_count, p->s.rows_done);
-    else
-      dispatch_atomic_kernel<false><<<nblk, kDispThreads, smem, st>>>(
-          (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row, (int)p->cap_rows, (int)p->P,
-          p->tiles_per_expert, spin, expert_count, p->s.tile_table, p->s.pool_next, tile_expert, (uint4*)recv,
-          src_info, slot_of, p->s.status, p->s.tile_count, p->s.rows_done);
+    auto kern = c.dispatch_mode == MOE_DISPATCH_ATOMIC_PAGED ? dispatch_atomic_kernel<true> : dispatch_atomic_kernel<false>;
+    launch_pdl(kern, dim3(nblk), dim3(kDispThreads), smem, st, (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row,
+               (int)p->cap_rows, (int)p->P, p->tiles_per_expert, spin, expert_count, p->s.tile_table, p->s.pool_next,
+               tile_expert, (uint4*)recv, src_info, slot_of, p->s.status, p->s.tile_count, p->s.rows_done);
     p->launches += 1;
   }
   return (int)cudaGetLastError();

@@ -19,6 +19,8 @@ ffn_simt_kernel(const XT* __restrict__ A, int lda, const int* __restrict__ tile_
                 const XT* __restrict__ B1, const XT* __restrict__ B2, size_t expert_stride, int N, int Kd,
                 XT* __restrict__ C, int ldc) {
   const int p = blockIdx.y;
+  pdl_wait();
+  pdl_trigger();
   const int e = tile_expert[p];
   if (e < 0) return;
   const int n0 = blockIdx.x * kSimtBN;
@@ -92,13 +94,12 @@ static int launch_typed(moe_plan* p, const void* recv, const int* tile_expert, c
   const size_t stride = (size_t)c.F * c.H;
   mark(p, 3, st);
   dim3 g1((c.F + kSimtBN - 1) / kSimtBN, (unsigned)p->P);
-  ffn_simt_kernel<XT, true><<<g1, kSimtThreads, 0, st>>>((const XT*)recv, c.H, tile_expert, (const XT*)wg,
-                                                         (const XT*)wu, stride, c.F, c.H, (XT*)p->s.inter, c.F);
+  launch_pdl(ffn_simt_kernel<XT, true>, g1, dim3(kSimtThreads), 0, st, (const XT*)recv, c.H, tile_expert,
+             (const XT*)wg, (const XT*)wu, stride, c.F, c.H, (XT*)p->s.inter, c.F);
   mark(p, 4, st);
   dim3 g2((c.H + kSimtBN - 1) / kSimtBN, (unsigned)p->P);
-  ffn_simt_kernel<XT, false><<<g2, kSimtThreads, 0, st>>>((const XT*)p->s.inter, c.F, tile_expert,
-                                                          (const XT*)wd, nullptr, stride, c.H, c.F,
-                                                          (XT*)out_rows, c.H);
+  launch_pdl(ffn_simt_kernel<XT, false>, g2, dim3(kSimtThreads), 0, st, (const XT*)p->s.inter, c.F, tile_expert,
+             (const XT*)wd, (const XT*)nullptr, stride, c.H, c.F, (XT*)out_rows, c.H);
   p->launches += 2;
   return (int)cudaGetLastError();
 }

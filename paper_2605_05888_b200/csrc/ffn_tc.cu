@@ -48,6 +48,8 @@ worklist_kernel(const int* __restrict__ tile_expert, int P, int E, int NB1, int 
   const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
   s_cnt[threadIdx.x] = 0;
   __syncthreads();
+  pdl_wait();
+  pdl_trigger();
   for (int p = threadIdx.x; p < P; p += 256) {
     gemm1_done[p] = 0;
     const int e = tile_expert[p];
@@ -136,9 +138,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int nseg = 2 * E;
-  for (int i = threadIdx.x; i <= E; i += kTcThreads) s_estart[i] = expert_start[i];
-  for (int i = threadIdx.x; i <= nseg; i += kTcThreads) s_seg_start[i] = seg_start[i];
-  for (int i = threadIdx.x; i < nseg; i += kTcThreads) s_seg_info[i] = seg_info[i];
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(smem_u32(&sh->full[s]), 1);
@@ -156,6 +155,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
                  "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  pdl_wait();  // everything above needs no global data and overlaps the predecessor's tail
+  for (int i = threadIdx.x; i <= E; i += kTcThreads) s_estart[i] = expert_start[i];
+  for (int i = threadIdx.x; i <= nseg; i += kTcThreads) s_seg_start[i] = seg_start[i];
+  for (int i = threadIdx.x; i < nseg; i += kTcThreads) s_seg_info[i] = seg_info[i];
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -358,6 +361,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
+  pdl_trigger();
   probe.finish();
   if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -433,9 +437,9 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   const int fused = (p->timing || c.ffn_split) ? 0 : 1;
   const bool pairs = c.ffn_kernel == 2;  // opt-in: the CTA-pair kernel
   const int workers = pairs ? grid / 2 : grid;
-  worklist_kernel<<<1, 256, 0, st>>>(tile_expert, (int)p->P, c.E, NB1, NB2, 2 * workers, fused, pairs ? 2 : 1,
-                                     p->s.tile_list, p->s.expert_start, p->s.seg_start, p->s.seg_info,
-                                     p->s.work_meta, p->s.gemm1_done);
+  launch_pdl(worklist_kernel, dim3(1), dim3(256), 0, st, tile_expert, (int)p->P, c.E, NB1, NB2, 2 * workers, fused,
+             pairs ? 2 : 1, p->s.tile_list, p->s.expert_start, p->s.seg_start, p->s.seg_info, p->s.work_meta,
+             p->s.gemm1_done);
   mark(p, 3, st);
   FfnParams prm;
   prm.tile_list = p->s.tile_list;
@@ -457,8 +461,8 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   auto launch = [&](int phase) -> int {
     prm.phase = phase;
     if (pairs) return launch_ffn_tc2_kernel(a1, bg, bu, a2, bd, prm, grid, st);
-    ffn_tc_kernel<<<grid, kTcThreads, kTcSmem, st>>>(a1, bg, bu, a2, bd, prm);
-    return cudaGetLastError() == cudaSuccess ? 0 : MOE_ERR_CUDA;
+    return launch_pdl(ffn_tc_kernel, dim3(grid), dim3(kTcThreads), kTcSmem, st, a1, bg, bu, a2, bd, prm) == cudaSuccess
+               ? 0 : MOE_ERR_CUDA;
   };
   if (fused) {
     if ((rc = launch(0)) != 0) return rc;

@@ -101,9 +101,6 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
   const bool leader = rank == 0;
   const int E = prm.E, F = prm.F, H = prm.H;
   const int nseg = 2 * E;
-  for (int i = threadIdx.x; i <= E; i += kTcThreads) s_estart[i] = prm.expert_start[i];
-  for (int i = threadIdx.x; i <= nseg; i += kTcThreads) s_seg_start[i] = prm.seg_start[i];
-  for (int i = threadIdx.x; i < nseg; i += kTcThreads) s_seg_info[i] = prm.seg_info[i];
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages2; ++s) {
       mbar_init(smem_u32(&sh->full[s]), 2);
@@ -121,6 +118,10 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
                  "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
+  pdl_wait();  // everything above needs no global data and overlaps the predecessor's tail
+  for (int i = threadIdx.x; i <= E; i += kTcThreads) s_estart[i] = prm.expert_start[i];
+  for (int i = threadIdx.x; i <= nseg; i += kTcThreads) s_seg_start[i] = prm.seg_start[i];
+  for (int i = threadIdx.x; i < nseg; i += kTcThreads) s_seg_info[i] = prm.seg_info[i];
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();  // both CTAs' barriers exist before anything arrives on them
@@ -319,6 +320,7 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
   __syncthreads();
   cluster_sync_all();  // neither CTA leaves while its partner may still touch its shared memory or TMEM
   tc_fence_after();
+  pdl_trigger();
   probe.finish();
   if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -332,8 +334,8 @@ int launch_ffn_tc2_kernel(const CUtensorMap& a1, const CUtensorMap& bg, const CU
       return MOE_ERR_CUDA;
     attr_done = true;
   }
-  ffn_tc2_kernel<<<grid & ~1, kTcThreads, kTcSmem2, st>>>(a1, bg, bu, a2, bd, prm);
-  return cudaGetLastError() == cudaSuccess ? 0 : MOE_ERR_CUDA;
+  return launch_pdl(ffn_tc2_kernel, dim3(grid & ~1), dim3(kTcThreads), kTcSmem2, st, a1, bg, bu, a2, bd, prm) ==
+                 cudaSuccess ? 0 : MOE_ERR_CUDA;
 }
 
 }  // namespace moehub

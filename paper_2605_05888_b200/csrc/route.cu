@@ -1,13 +1,14 @@
 // Step 1 of the MoE layer (paper Section II-A, routing): gate logits, softmax, top-K.
 //
-// Each CTA owns a block of TB tokens and all E experts.  The logit of (token, expert) is ONE
+// Each CTA owns a block of tokens and all E experts.  The logit of (token, expert) is ONE
 // ascending fp32 FMA chain over h (no split of the h range, no tensor cores), because the
 // logit decides which experts are picked and the pick has to be reproducible bit for bit.
 // The parallelism is across the T*E independent chains: x and Wr chunks are staged in shared
-// memory (16-byte global loads, next chunk prefetched into registers), every thread carries a
-// TM x TE register tile of chains.  Afterwards the logits go through shared memory to one warp
-// per token, which keeps them in registers (E/32 per lane) and runs K rounds of a shuffle
-// arg-max (ties: lowest expert index), then the softmax weights.
+// memory as fp32 (16-byte global loads, next chunk prefetched into registers).  Two shapes:
+// E <= 64 is bound by the latency of the chain itself - one lane per chain; 64 < E <= 256 is
+// bound by fp32 FMA issue - an 8 x 8 register tile of chains per thread.  Afterwards the logits
+// go through shared memory to one warp per token, which keeps them in registers (E/32 per lane)
+// and runs K rounds of a shuffle arg-max (ties: lowest expert index), then the softmax weights.
 #include <float.h>
 
 #include "common.cuh"
@@ -15,41 +16,6 @@
 namespace moehub {
 
 constexpr int kRouteThreads = 256;
-
-template <typename XT, int ROWS, int HC>
-struct ChunkRegs {  // the 16-byte vectors one thread holds of a [ROWS][HC] chunk
-  static constexpr int N = Vec16<XT>::N;
-  static constexpr int PARTS = HC / N;
-  static constexpr int NVEC = ROWS * PARTS;
-  static constexpr int PER_THREAD = (NVEC + kRouteThreads - 1) / kRouteThreads;
-  uint4 v[PER_THREAD];
-
-  __device__ __forceinline__ void load(const XT* base, int row0, int nrows_valid, int H, int h0) {
-#pragma unroll
-    for (int i = 0; i < PER_THREAD; ++i) {
-      const int idx = threadIdx.x + i * kRouteThreads;
-      const int r = idx / PARTS, part = idx % PARTS;
-      const int h = h0 + part * N;
-      v[i] = make_uint4(0, 0, 0, 0);
-      if (idx < NVEC && r < nrows_valid && h < H)
-        v[i] = __ldg(reinterpret_cast<const uint4*>(base + (size_t)(row0 + r) * H + h));
-    }
-  }
-  // smem layout [HC][ROWS + 1] (transposed; the odd width keeps the transposing stores conflict-free)
-  __device__ __forceinline__ void store(float* s) const {
-#pragma unroll
-    for (int i = 0; i < PER_THREAD; ++i) {
-      const int idx = threadIdx.x + i * kRouteThreads;
-      if (idx < NVEC) {
-        const int r = idx / PARTS, part = idx % PARTS;
-        float f[N];
-        Vec16<XT>::unpack(v[i], f);
-#pragma unroll
-        for (int q = 0; q < N; ++q) s[(part * N + q) * (ROWS + 1) + r] = f[q];
-      }
-    }
-  }
-};
 
 // One warp per token: the token's logits sit in registers (EP/32 per lane); K rounds of a shuffle
 // arg-max on (value, lowest index); then the softmax weights of the picks.  ls: [tokens][EP] logits
@@ -107,92 +73,6 @@ __device__ __forceinline__ void select_topk(const float* ls, int tvalid, int t0,
       topk_w[(size_t)(t0 + tl) * K + lane] = p;
     }
   }
-}
-
-template <typename XT, int TX, int TE, int TY, int TM, int HC>
-__global__ void __launch_bounds__(kRouteThreads)
-route_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias,
-             int T, int H, int E, int K, int renorm, int* __restrict__ topk_idx,
-             float* __restrict__ topk_w) {
-  static_assert(TX * TY == kRouteThreads, "thread layout");
-  constexpr int TB = TY * TM, EP = TX * TE;
-  constexpr int XW = TB + 1, WW = EP + 1;
-  extern __shared__ float smem[];
-  float* xs = smem;            // [HC][XW]
-  float* ws = smem + HC * XW;  // [HC][WW]
-  float* ls = smem;             // [TB][EP], reuses the staging area after the h loop
-
-  const int tx = threadIdx.x % TX, ty = threadIdx.x / TX;
-  const int t0 = blockIdx.x * TB;
-  const int tvalid = min(TB, T - t0);
-
-  float acc[TM][TE];
-#pragma unroll
-  for (int j = 0; j < TM; ++j)
-#pragma unroll
-    for (int i = 0; i < TE; ++i) acc[j][i] = 0.0f;
-
-  ChunkRegs<XT, TB, HC> xr;
-  ChunkRegs<XT, EP, HC> wrg;
-  xr.load(x, t0, tvalid, H, 0);
-  wrg.load(wr, 0, E, H, 0);
-
-  for (int h0 = 0; h0 < H; h0 += HC) {
-    __syncthreads();  // previous chunk fully consumed
-    xr.store(xs);
-    wrg.store(ws);
-    __syncthreads();
-    if (h0 + HC < H) {  // prefetch the next chunk while this one is computed
-      xr.load(x, t0, tvalid, H, h0 + HC);
-      wrg.load(wr, 0, E, H, h0 + HC);
-    }
-    const int hmax = min(HC, H - h0);
-#pragma unroll 4
-    for (int hh = 0; hh < hmax; ++hh) {
-      float xv[TM], wv[TE];
-#pragma unroll
-      for (int j = 0; j < TM; ++j) xv[j] = xs[hh * XW + ty + TY * j];
-#pragma unroll
-      for (int i = 0; i < TE; ++i) wv[i] = ws[hh * WW + tx + TX * i];
-#pragma unroll
-      for (int j = 0; j < TM; ++j)
-#pragma unroll
-        for (int i = 0; i < TE; ++i) acc[j][i] = __fmaf_rn(xv[j], wv[i], acc[j][i]);
-    }
-  }
-  __syncthreads();
-#pragma unroll
-  for (int j = 0; j < TM; ++j)
-#pragma unroll
-    for (int i = 0; i < TE; ++i) {
-      const int e = tx + TX * i;
-      float l = acc[j][i];
-      if (bias != nullptr && e < E) l = l + bias[e];
-      ls[(ty + TY * j) * EP + e] = l;
-    }
-  __syncthreads();
-
-  select_topk<EP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w);
-}
-
-template <typename XT, int TX, int TE, int TY, int TM, int HC>
-static int launch_cfg(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
-                      float* topk_w, cudaStream_t st) {
-  constexpr int TB = TY * TM, EP = TX * TE;
-  const size_t stage = sizeof(float) * HC * (TB + 1 + EP + 1);
-  const size_t logits = sizeof(float) * TB * EP;
-  const size_t smem = stage > logits ? stage : logits;
-  auto kern = route_kernel<XT, TX, TE, TY, TM, HC>;
-  if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return (int)e;
-  }
-  const moe_config_t& c = p->cfg;
-  const int grid = (c.T + TB - 1) / TB;
-  kern<<<grid, kRouteThreads, smem, st>>>((const XT*)x, (const XT*)wr, bias, c.T, c.H, c.E, c.K,
-                                          c.renormalize, topk_idx, topk_w);
-  p->launches += 1;
-  return (int)cudaGetLastError();
 }
 
 // The compute-bound shape (64 < E <= 256): 64 tokens x 256 experts per CTA, 8 x 8 chains per thread,
@@ -254,6 +134,8 @@ route_wide_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const flo
 
   WideChunk<XT, kWideTB> xr;
   WideChunk<XT, kWideEP> wrg;
+  pdl_wait();
+  pdl_trigger();
   xr.load(x, t0, tvalid, H, 0);
   wrg.load(wr, 0, E, H, 0);
   for (int h0 = 0; h0 < H; h0 += kWideHC) {
@@ -315,10 +197,9 @@ static int launch_wide(moe_plan* p, const void* x, const void* wr, const float* 
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return (int)e;
   const moe_config_t& c = p->cfg;
-  kern<<<(c.T + kWideTB - 1) / kWideTB, kRouteThreads, smem, st>>>((const XT*)x, (const XT*)wr, bias, c.T, c.H,
-                                                                   c.E, c.K, c.renormalize, topk_idx, topk_w);
   p->launches += 1;
-  return (int)cudaGetLastError();
+  return (int)launch_maybe_pdl(false, kern, dim3((c.T + kWideTB - 1) / kWideTB), dim3(kRouteThreads), smem, st, (const XT*)x,
+                         (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w);
 }
 
 // The latency-bound shapes (E <= 64): one lane per chain (or two chains for 32 < E <= 64).  A token's
@@ -384,6 +265,8 @@ route_narrow_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const f
   for (int i = 0; i < TE; ++i) acc[i] = 0.0f;
   NaturalChunk<XT, TB, HC> xr;
   NaturalChunk<XT, EP, HC> wrg;
+  pdl_wait();
+  pdl_trigger();
   xr.load(x, t0, tvalid, H, 0);
   wrg.load(wr, 0, E, H, 0);
   for (int h0 = 0; h0 < H; h0 += HC) {
@@ -458,10 +341,9 @@ static int launch_narrow(moe_plan* p, const void* x, const void* wr, const float
     if (e != cudaSuccess) return (int)e;
   }
   const moe_config_t& c = p->cfg;
-  kern<<<(c.T + TB - 1) / TB, kRouteThreads, smem, st>>>((const XT*)x, (const XT*)wr, bias, c.T, c.H, c.E, c.K,
-                                                          c.renormalize, topk_idx, topk_w);
   p->launches += 1;
-  return (int)cudaGetLastError();
+  return (int)launch_maybe_pdl(false, kern, dim3((c.T + TB - 1) / TB), dim3(kRouteThreads), smem, st, (const XT*)x,
+                         (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w);
 }
 
 template <typename XT>
