@@ -47,6 +47,7 @@ int check_config(const moe_config_t* c, Geometry* g) {
   int tpb = 256 / c->K;  // at most 256 assignments per dispatch CTA
   if (tpb > 16) tpb = 16;
   if (tpb < 1) tpb = 1;
+  while (tpb > 1 && (c->T + tpb - 1) / tpb < 2 * 148) tpb /= 2;  // small batches: enough CTAs to fill the GPU
   g->dispatch_tokens = tpb;
   g->nblk = (c->T + tpb - 1) / tpb;
   return MOE_OK;

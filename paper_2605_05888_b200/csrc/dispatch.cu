@@ -25,30 +25,33 @@ constexpr int kDispThreads = 256;
 constexpr int kMaxAssign = 256;  // assignments (token,k pairs) per CTA
 
 // ------------------------------------------------------------------------------------------------
-// Row copy: warp `warp` of the CTA copies token rows tl = warp, warp+8, ... to their K slots.
+// Row copy: the block's rows are cut into runs of 32*UNROLL 16-byte vectors; the warps take runs
+// round-robin, so a block with a single token still uses all its warps.  A run is read once and
+// stored to the token's K slots.
 template <int UNROLL>
 __device__ __forceinline__ void copy_rows(const uint4* __restrict__ x, uint4* __restrict__ recv,
                                           const int* s_slot, int t0, int ntok, int K, int vec_per_row) {
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  for (int tl = warp; tl < ntok; tl += kDispThreads / 32) {
+  constexpr int RUN = 32 * UNROLL;
+  const int runs = (vec_per_row + RUN - 1) / RUN;
+  for (int u = warp; u < ntok * runs; u += kDispThreads / 32) {
+    const int tl = u / runs, v0 = (u % runs) * RUN;
     const uint4* src = x + (size_t)(t0 + tl) * vec_per_row;
     const int* slots = s_slot + tl * K;
-    for (int v0 = 0; v0 < vec_per_row; v0 += 32 * UNROLL) {
-      uint4 r[UNROLL];
+    uint4 r[UNROLL];
 #pragma unroll
-      for (int u = 0; u < UNROLL; ++u) {
-        const int v = v0 + u * 32 + lane;
-        if (v < vec_per_row) r[u] = __ldg(src + v);
-      }
-      for (int k = 0; k < K; ++k) {
-        const int slot = slots[k];
-        if (slot < 0) continue;
-        uint4* dst = recv + (size_t)slot * vec_per_row;
+    for (int i = 0; i < UNROLL; ++i) {
+      const int v = v0 + i * 32 + lane;
+      if (v < vec_per_row) r[i] = __ldg(src + v);
+    }
+    for (int k = 0; k < K; ++k) {
+      const int slot = slots[k];
+      if (slot < 0) continue;
+      uint4* dst = recv + (size_t)slot * vec_per_row;
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-          const int v = v0 + u * 32 + lane;
-          if (v < vec_per_row) __stcs(dst + v, r[u]);
-        }
+      for (int i = 0; i < UNROLL; ++i) {
+        const int v = v0 + i * 32 + lane;
+        if (v < vec_per_row) __stcs(dst + v, r[i]);
       }
     }
   }
@@ -330,12 +333,12 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
   if (c.T == 0) return 0;
   const int nblk = p->nblk, tpb = p->dispatch_tokens;
   if (c.dispatch_mode == MOE_DISPATCH_SCAN) {
-    launch_pdl(hist_kernel, dim3(nblk), dim3(kDispThreads), sizeof(int) * c.E, st, topk_idx, c.T, c.E, c.K, tpb,
+    launch_maybe_pdl(false, hist_kernel, dim3(nblk), dim3(kDispThreads), sizeof(int) * c.E, st, topk_idx, c.T, c.E, c.K, tpb,
                p->s.cta_count);
-    launch_pdl(scan_kernel, dim3(c.E), dim3(kDispThreads), 0, st, p->s.cta_count, nblk, c.E, (int)p->P, p->s.cta_base,
+    launch_maybe_pdl(false, scan_kernel, dim3(c.E), dim3(kDispThreads), 0, st, p->s.cta_count, nblk, c.E, (int)p->P, p->s.cta_base,
                expert_count, p->s.tile_base, tile_expert, p->s.scan_ticket);
     const size_t smem = sizeof(int) * ((kDispThreads / 32) * c.E + kMaxAssign);
-    launch_pdl(scatter_kernel, dim3(nblk), dim3(kDispThreads), smem, st, (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb,
+    launch_maybe_pdl(false, scatter_kernel, dim3(nblk), dim3(kDispThreads), smem, st, (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb,
                vec_per_row, p->s.cta_base, p->s.tile_base, (uint4*)recv, src_info, slot_of, p->s.tile_count,
                p->s.rows_done);
     p->launches += 3;
@@ -420,6 +423,7 @@ extern "C" int moe_dispatch_noalloc(const moe_config_t* cfg, const void* d_x, co
   if (tiles_per_expert == 0) tiles_per_expert = 1;
   int tpb = 256 / c.K;
   if (tpb > 16) tpb = 16;
+  while (tpb > 1 && (c.T + tpb - 1) / tpb < 2 * 148) tpb /= 2;
   const int nblk = (c.T + tpb - 1) / tpb;
   // The array keeps whatever the previous call left: reset the cursor and the part of the table
   // this call reads, and the caller's counters, before the kernel runs.

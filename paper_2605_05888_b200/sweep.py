@@ -1,0 +1,96 @@
+"""Dispatch/combine-only sweep (identity experts): H = 7168, E = 256 on R = 32 logical ranks, top-8, bf16,
+T from 128 to 65536 in powers of two, unbiased and Zipf(1.2) routing.  For every point it times the
+dispatch stage (baseline scan scheme and the destination-agnostic paged scheme) and the combine stage
+with CUDA events and prints algorithmic GB/s and the fraction of the measured HBM copy bandwidth.
+
+    python -m paper_2605_05888_b200.sweep [--max-t 65536] [--iters 20] [--markdown]
+
+Algorithmic bytes: dispatch T*H*b*(1+K) + 12*T*K (row read once, written K times; indices in, slot and
+source info out); combine T*H*b*(K+1) + 8*T*K.  Below T = 2048 the stages take a few microseconds and are
+bound by launch latency, not bandwidth: read the microseconds there, not the GB/s.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import inputs
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def hbm_peak_gbs() -> tuple[float, str]:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        return json.load(open(path))["hbm_gbs"], "measured"
+    return 6650.0, "fallback"
+
+
+def time_point(w: inputs.Workload, mode: int, iters: int) -> dict:
+    x = inputs.make_x(w)
+    wr, bias = inputs.make_router(w)
+    dx = torch.from_numpy(x).view(torch.int16).cuda().view(torch.bfloat16)
+    dwr = torch.from_numpy(wr).view(torch.int16).cuda().view(torch.bfloat16)
+    dbias = None if bias is None else torch.from_numpy(bias).cuda()
+    plan = B.Plan(B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype, dispatch_mode=mode, identity_experts=1))
+    y = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+    for _ in range(3):
+        plan.moe_layer(dx, dwr, dbias, None, None, None, y)
+    torch.cuda.synchronize()
+    code, detail = plan.moe_last_status()
+    assert code == 0, (code, detail)
+    ms = np.array([plan.moe_layer_timed(dx, dwr, dbias, None, None, None, y) for _ in range(iters)])
+    med = np.median(ms, axis=0)
+    cnt = plan.layer_tensor(3).cpu().numpy()
+    return {"dispatch_ms": float(med[B.STAGES.index("dispatch")]), "combine_ms": float(med[B.STAGES.index("combine")]),
+            "route_ms": float(med[B.STAGES.index("route")]), "hottest_share": float(cnt.max() / w.T),
+            "imbalance_std": float(np.std(cnt / (w.T * w.K)))}
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--min-t", type=int, default=128)
+    ap.add_argument("--max-t", type=int, default=65536)
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--markdown", action="store_true")
+    args = ap.parse_args()
+    peak, kind = hbm_peak_gbs()
+    rows = []
+    T = args.min_t
+    while T <= args.max_t:
+        for zipf in (0.0, 1.2):
+            w = inputs.C5(T, zipf)
+            eb, n = w.elem_bytes, w.T * w.K
+            disp_bytes = w.T * w.H * eb * (1 + w.K) + 12 * n
+            comb_bytes = w.T * w.H * eb * (w.K + 1) + 8 * n
+            scan = time_point(w, B.DISPATCH_SCAN, args.iters)
+            paged = time_point(w, B.DISPATCH_ATOMIC_PAGED, args.iters)
+            rows.append({"T": T, "routing": "zipf1.2" if zipf else "uniform", "hottest_share": paged["hottest_share"],
+                         "dispatch_scan_us": 1e3 * scan["dispatch_ms"], "dispatch_paged_us": 1e3 * paged["dispatch_ms"],
+                         "dispatch_scan_GBps": disp_bytes / scan["dispatch_ms"] / 1e6,
+                         "dispatch_paged_GBps": disp_bytes / paged["dispatch_ms"] / 1e6,
+                         "combine_us": 1e3 * paged["combine_ms"], "combine_GBps": comb_bytes / paged["combine_ms"] / 1e6})
+            torch.cuda.empty_cache()
+        T *= 2
+    if args.markdown:
+        print(f"HBM copy peak: {peak:.1f} GB/s ({kind}). Times are medians of {args.iters} runs, CUDA events around the stage.")
+        print()
+        print("| T | routing | hottest expert (rows/T) | dispatch scan us | GB/s | % | dispatch paged us | GB/s | % | combine us | GB/s | % |")
+        print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+        for r in rows:
+            print(f"| {r['T']} | {r['routing']} | {r['hottest_share']:.2f} | {r['dispatch_scan_us']:.1f} | "
+                  f"{r['dispatch_scan_GBps']:.0f} | {100 * r['dispatch_scan_GBps'] / peak:.0f} | {r['dispatch_paged_us']:.1f} | "
+                  f"{r['dispatch_paged_GBps']:.0f} | {100 * r['dispatch_paged_GBps'] / peak:.0f} | {r['combine_us']:.1f} | "
+                  f"{r['combine_GBps']:.0f} | {100 * r['combine_GBps'] / peak:.0f} |")
+    else:
+        for r in rows:
+            print(json.dumps(r))
+
+
+if __name__ == "__main__":
+    main()
