@@ -34,9 +34,10 @@ WORKLOADS = {"c1": inputs.C1, "c2": inputs.C2, "c3": inputs.C3, "c4": inputs.C4,
              # dispatch/combine-only sweep points (identity experts)
              "c5_8192": inputs.C5(8192), "c5_8192_zipf": inputs.C5(8192, 1.2), "c5_2048": inputs.C5(2048)}
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel,
-# from the ncu capture summarised under profiles/; None until a capture exists for that workload.
-NCU_TRAFFIC_BYTES = {}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
+# ncu capture summarised in profiles/ffn_tc_kernel_c2_small.md.  The capture ran the quarter-size case
+# (901.6 MB per launch); C2 proper does 4x its flops with 4x its weights, so the figure is scaled by 4.
+NCU_TRAFFIC_BYTES = {"mixtral_like_bf16_small": 901.6e6, "mixtral_like_bf16": 4 * 901.6e6}
 
 
 def load_peaks() -> tuple[dict, str]:
@@ -293,17 +294,21 @@ def run_cuda(args, w: inputs.Workload) -> None:
                     "unit": "GB/s", "frac": stages["dispatch"]["frac_hbm"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
                     "peak_source": f"{peak_kind} hbm_gbs"}
     else:
-        t1, t2 = sm["gemm1"], sm["gemm2"]
-        stages["ffn_gemm1"] = {"ms": t1, "TFLOPs": gemm1_flops / t1 / 1e9}
-        stages["ffn_gemm2"] = {"ms": t2, "TFLOPs": gemm2_flops / t2 / 1e9}
+        t_ffn = sm["gemm1"] + sm["gemm2"]
+        stages["ffn"] = {"ms": t_ffn, "TFLOPs": (gemm1_flops + gemm2_flops) / t_ffn / 1e9,
+                         "launches": 2 if args.ffn_split else 1}
+        if args.ffn_split:
+            stages["ffn_gemm1"] = {"ms": sm["gemm1"], "TFLOPs": gemm1_flops / sm["gemm1"] / 1e9}
+            stages["ffn_gemm2"] = {"ms": sm["gemm2"], "TFLOPs": gemm2_flops / sm["gemm2"] / 1e9}
         stages["worklist"] = {"ms": sm["worklist"]}
-        tensor_peak = peaks["bf16_tflops"]
-        ach = gemm1_flops / t1 / 1e9
-        roofline = {"kernel": "ffn_tc_kernel<SWIGLU> (GEMM1 + SwiGLU epilogue)", "bound": "tensor", "achieved": ach,
-                    "peak": tensor_peak, "unit": "TFLOP/s", "frac": ach / tensor_peak,
+        ach = stages["ffn"]["TFLOPs"]
+        roofline = {"kernel": "ffn_tc_kernel (expert GEMM1 + SwiGLU + GEMM2, tcgen05)", "bound": "tensor",
+                    "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
                     "traffic": NCU_TRAFFIC_BYTES.get(w.name),
-                    "peak_source": f"{peak_kind} bf16_tflops (burst)",
-                    "ffn_both_gemms_TFLOPs": (gemm1_flops + gemm2_flops) / (t1 + t2) / 1e9}
+                    "peak_source": f"{peak_kind} bf16_tflops (burst); the kernel runs power-capped at the clock in "
+                                   "clocks.ffn_kernel_sm_mhz",
+                    "frac_of_sustained_peak": ach / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                    "useful_flops_per_launch": gemm1_flops + gemm2_flops}
 
     # the CPU oracle on a bounded sample of the same batch (N = 1 only)
     cpu = None

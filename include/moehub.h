@@ -174,7 +174,8 @@ int moe_layer_host(moe_plan_t* plan, const void* h_x, const void* d_wr, const fl
 /* moe_layer with a CUDA event recorded after every kernel: runs the layer once, synchronises the
  * stream and writes the device time of each stage, in milliseconds, to h_stage_ms
  * [MOE_STAGE_COUNT] (host): route, dispatch (all its kernels and counter resets), FFN work list,
- * FFN GEMM1 (+SwiGLU), FFN GEMM2, combine.  For measurement only. */
+ * FFN GEMM1 (+SwiGLU), FFN GEMM2, combine.  With ffn_split = 0 both GEMMs are one launch: its
+ * time is reported under GEMM1 and GEMM2 reads 0.  For measurement only. */
 #define MOE_STAGE_ROUTE 0
 #define MOE_STAGE_DISPATCH 1
 #define MOE_STAGE_WORKLIST 2
