@@ -78,7 +78,9 @@ typedef struct {
                                    counters gate GEMM2); 1: one launch per GEMM                 */
   int64_t capacity_rows;        /* mode 1: rows per expert region, multiple of 128, 0 = T
                                    rounded up (overflow-free); modes 0/2: ignored            */
-  uint64_t spin_limit;          /* bound on every device-side wait, 0 = default (1<<22)      */
+  uint64_t spin_limit;          /* bound (iterations) on the dispatch kernels' waits, 0 = 1<<22 */
+  uint64_t wait_limit_ns;       /* bound (nanoseconds) on every wait inside the tensor-core
+                                   expert kernels, 0 = 2 s                                   */
 } moe_config_t;
 
 /* Number P of 128-row tiles in the receive pool for this configuration:
@@ -111,21 +113,31 @@ int moe_route(moe_plan_t* plan, const void* d_x, const void* d_wr, const float* 
  *      d_expert_count [E] rows per expert, d_tile_expert [P] owner of each tile or -1,
  *      d_src_info [P*128] = t*K+k of the row in that slot, -1 for an empty slot (the source
  *      information of Section IV-B, combine), d_slot_of [T,K] physical row of assignment
- *      (t,k), or -1 if it was dropped by an overflow (status MOE_ERR_OVERFLOW). */
+ *      (t,k), or -1 if it was dropped by an overflow (status MOE_ERR_OVERFLOW);
+ *      availability counters (Section IV-D, data availability manager), both or neither,
+ *      NULL = kept in the plan's workspace: d_tile_count [P] rows stored so far in each tile,
+ *      d_rows_done [1] assignments whose rows are stored; both raised with release semantics
+ *      after the rows they count are written, so a consumer that reads tile_count[p] >= 128
+ *      or rows_done == T*K with acquire semantics may read the tile. */
 int moe_dispatch(moe_plan_t* plan, const void* d_x, const int32_t* d_topk_idx, void* d_recv,
                  int32_t* d_expert_count, int32_t* d_tile_expert, int32_t* d_src_info,
-                 int32_t* d_slot_of, void* stream);
+                 int32_t* d_slot_of, int32_t* d_tile_count, int32_t* d_rows_done, void* stream);
 
 /* Step 3 (Section II-A, expert computation; "two GEMMs with an activation between", here
  * SwiGLU): for every used tile p of expert e = tile_expert[p]:
  *   S = silu(A*Wg[e]^T) .* (A*Wu[e]^T),  O = S*Wd[e]^T,  A = the tile's 128 rows of d_recv.
  * Unused tiles are skipped and their experts' weights never read (Section IV-D: thread
  * blocks whose counters stay zero are never scheduled).
- * in: d_recv [P*128,H], d_tile_expert [P], d_wg/d_wu [E,F,H], d_wd [E,H,F] (dtype).
+ * in: d_recv [P*128,H], d_tile_expert [P], d_wg/d_wu [E,F,H], d_wd [E,H,F] (dtype);
+ *     d_tile_count [P], d_rows_done [1]: the availability counters of moe_dispatch, both or
+ *     neither.  When given, the tensor-core kernel waits before it reads a tile until
+ *     tile_count[p] >= 128 or rows_done >= T*K (bounded by wait_limit_ns; on expiry the status
+ *     word reads MOE_ERR_TIMEOUT and the kernel returns).  NULL: the rows are complete when the
+ *     call is reached in stream order.  The SIMT kernel ignores them (stream order).
  * out: d_out_rows [P*128,H] (dtype); rows of empty slots hold unspecified values. */
 int moe_expert_ffn(moe_plan_t* plan, const void* d_recv, const int32_t* d_tile_expert,
                    const void* d_wg, const void* d_wu, const void* d_wd, void* d_out_rows,
-                   void* stream);
+                   const int32_t* d_tile_count, const int32_t* d_rows_done, void* stream);
 
 /* Dispatch without any allocation (the paper has no counterpart: this entry point exists for
  * the callers described here, not for a step of the method).  Some callers cannot give this

@@ -31,7 +31,7 @@ class MoeConfig(ctypes.Structure):
                 ("K", ctypes.c_int32), ("F", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("renormalize", ctypes.c_int32), ("dispatch_mode", ctypes.c_int32),
                 ("identity_experts", ctypes.c_int32), ("ffn_kernel", ctypes.c_int32), ("ffn_split", ctypes.c_int32),
-                ("capacity_rows", ctypes.c_int64), ("spin_limit", ctypes.c_uint64)]
+                ("capacity_rows", ctypes.c_int64), ("spin_limit", ctypes.c_uint64), ("wait_limit_ns", ctypes.c_uint64)]
 
 
 class MoeError(RuntimeError):
@@ -54,9 +54,9 @@ def lib() -> ctypes.CDLL:
         L.moe_plan_create.argtypes = [cfgp, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
         L.moe_plan_destroy.argtypes = [vp]
         L.moe_route.argtypes = [vp, vp, vp, fp, i32p, fp, vp]
-        L.moe_dispatch.argtypes = [vp, vp, i32p, vp, i32p, i32p, i32p, i32p, vp]
+        L.moe_dispatch.argtypes = [vp, vp, i32p, vp, i32p, i32p, i32p, i32p, i32p, i32p, vp]
         L.moe_dispatch_noalloc.argtypes = [cfgp, vp, i32p, vp, i32p, i32p, i32p, i32p, i32p, vp]
-        L.moe_expert_ffn.argtypes = [vp, vp, i32p, vp, vp, vp, vp, vp]
+        L.moe_expert_ffn.argtypes = [vp, vp, i32p, vp, vp, vp, vp, i32p, i32p, vp]
         L.moe_combine.argtypes = [vp, vp, i32p, fp, vp, vp]
         L.moe_layer.argtypes = [vp] * 9
         L.moe_layer_host.argtypes = [vp] * 9
@@ -99,9 +99,9 @@ def _stream(stream) -> int:
 
 
 def make_config(T, H, E, R, K, F, dtype, renormalize=0, dispatch_mode=DISPATCH_ATOMIC_PAGED, identity_experts=0,
-                ffn_kernel=0, capacity_rows=0, spin_limit=0, ffn_split=0) -> MoeConfig:
+                ffn_kernel=0, capacity_rows=0, spin_limit=0, ffn_split=0, wait_limit_ns=0) -> MoeConfig:
     return MoeConfig(T, H, E, R, K, F, dtype, int(renormalize), dispatch_mode, int(identity_experts), ffn_kernel, int(ffn_split),
-                     capacity_rows, spin_limit)
+                     capacity_rows, spin_limit, wait_limit_ns)
 
 
 def moe_pool_tiles(cfg: MoeConfig) -> int:
@@ -155,13 +155,16 @@ class Plan:
         _check(lib().moe_route(self.handle, _ptr(x), _ptr(wr), _ptr(bias), _ptr(topk_idx), _ptr(topk_w),
                                _stream(stream)), "moe_route")
 
-    def moe_dispatch(self, x, topk_idx, recv, expert_count, tile_expert, src_info, slot_of, stream=None):
+    def moe_dispatch(self, x, topk_idx, recv, expert_count, tile_expert, src_info, slot_of, tile_count=None,
+                     rows_done=None, stream=None):
         _check(lib().moe_dispatch(self.handle, _ptr(x), _ptr(topk_idx), _ptr(recv), _ptr(expert_count),
-                                  _ptr(tile_expert), _ptr(src_info), _ptr(slot_of), _stream(stream)), "moe_dispatch")
+                                  _ptr(tile_expert), _ptr(src_info), _ptr(slot_of), _ptr(tile_count), _ptr(rows_done),
+                                  _stream(stream)), "moe_dispatch")
 
-    def moe_expert_ffn(self, recv, tile_expert, wg, wu, wd, out_rows, stream=None):
+    def moe_expert_ffn(self, recv, tile_expert, wg, wu, wd, out_rows, tile_count=None, rows_done=None, stream=None):
         _check(lib().moe_expert_ffn(self.handle, _ptr(recv), _ptr(tile_expert), _ptr(wg), _ptr(wu), _ptr(wd),
-                                    _ptr(out_rows), _stream(stream)), "moe_expert_ffn")
+                                    _ptr(out_rows), _ptr(tile_count), _ptr(rows_done), _stream(stream)),
+               "moe_expert_ffn")
 
     def moe_combine(self, rows, slot_of, topk_w, y, stream=None):
         _check(lib().moe_combine(self.handle, _ptr(rows), _ptr(slot_of), _ptr(topk_w), _ptr(y), _stream(stream)),

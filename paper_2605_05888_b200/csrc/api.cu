@@ -176,30 +176,36 @@ int moe_route(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_b
 
 int moe_dispatch(moe_plan_t* p, const void* d_x, const int32_t* d_topk_idx, void* d_recv,
                  int32_t* d_expert_count, int32_t* d_tile_expert, int32_t* d_src_info, int32_t* d_slot_of,
-                 void* stream) {
+                 int32_t* d_tile_count, int32_t* d_rows_done, void* stream) {
   if (!p || !d_recv || !d_expert_count || !d_tile_expert || !d_src_info) return MOE_ERR_ARG;
   if (p->cfg.T > 0 && (!d_x || !d_topk_idx || !d_slot_of)) return MOE_ERR_ARG;
   if (misaligned(d_x) || misaligned(d_recv)) return MOE_ERR_ALIGN;
   p->launches = 0;
+  if ((d_tile_count == nullptr) != (d_rows_done == nullptr)) return MOE_ERR_ARG;
   return launch_dispatch(p, d_x, d_topk_idx, d_recv, d_expert_count, d_tile_expert, d_src_info, d_slot_of,
+                         d_tile_count ? d_tile_count : p->s.tile_count, d_rows_done ? d_rows_done : p->s.rows_done,
                          (cudaStream_t)stream) ? MOE_ERR_CUDA : MOE_OK;
 }
 
 static int ffn_dispatch(moe_plan* p, const void* recv, const int* tile_expert, const void* wg, const void* wu,
-                        const void* wd, void* out_rows, bool gate_on_dispatch, cudaStream_t st) {
+                        const void* wd, void* out_rows, const int* tile_count, const int* rows_done,
+                        cudaStream_t st) {
   if (p->cfg.dtype == MOE_DTYPE_BF16 && p->cfg.ffn_kernel != 1)
-    return launch_ffn_tc(p, recv, tile_expert, wg, wu, wd, out_rows, gate_on_dispatch, st);
+    return launch_ffn_tc(p, recv, tile_expert, wg, wu, wd, out_rows, tile_count, rows_done, st);
   return launch_ffn_simt(p, recv, tile_expert, wg, wu, wd, out_rows, st);
 }
 
 int moe_expert_ffn(moe_plan_t* p, const void* d_recv, const int32_t* d_tile_expert, const void* d_wg,
-                   const void* d_wu, const void* d_wd, void* d_out_rows, void* stream) {
+                   const void* d_wu, const void* d_wd, void* d_out_rows, const int32_t* d_tile_count,
+                   const int32_t* d_rows_done, void* stream) {
   if (!p || !d_recv || !d_tile_expert || !d_wg || !d_wu || !d_wd || !d_out_rows) return MOE_ERR_ARG;
   if (p->cfg.identity_experts) return MOE_ERR_ARG;
   if (misaligned(d_recv) || misaligned(d_wg) || misaligned(d_wu) || misaligned(d_wd) || misaligned(d_out_rows))
     return MOE_ERR_ALIGN;
   p->launches = 0;
-  int rc = ffn_dispatch(p, d_recv, d_tile_expert, d_wg, d_wu, d_wd, d_out_rows, false, (cudaStream_t)stream);
+  if ((d_tile_count == nullptr) != (d_rows_done == nullptr)) return MOE_ERR_ARG;
+  int rc = ffn_dispatch(p, d_recv, d_tile_expert, d_wg, d_wu, d_wd, d_out_rows, d_tile_count, d_rows_done,
+                        (cudaStream_t)stream);
   return rc == 0 ? MOE_OK : (rc < 0 ? rc : MOE_ERR_CUDA);
 }
 
@@ -226,11 +232,12 @@ int moe_layer(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_b
   mark(p, 0, st);
   if (launch_route(p, d_x, d_wr, d_bias, s.topk_idx, s.topk_w, st)) return MOE_ERR_CUDA;
   mark(p, 1, st);
-  if (launch_dispatch(p, d_x, s.topk_idx, s.recv, s.expert_count, s.tile_expert, s.src_info, s.slot_of, st))
+  if (launch_dispatch(p, d_x, s.topk_idx, s.recv, s.expert_count, s.tile_expert, s.src_info, s.slot_of, s.tile_count,
+                      s.rows_done, st))
     return MOE_ERR_CUDA;
   mark(p, 2, st);
   if (!p->cfg.identity_experts) {
-    int rc = ffn_dispatch(p, s.recv, s.tile_expert, d_wg, d_wu, d_wd, s.out_rows, true, st);
+    int rc = ffn_dispatch(p, s.recv, s.tile_expert, d_wg, d_wu, d_wd, s.out_rows, s.tile_count, s.rows_done, st);
     if (rc != 0) return rc < 0 ? rc : MOE_ERR_CUDA;
   } else {
     mark(p, 3, st);

@@ -109,15 +109,17 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
 int launch_route(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
                  float* topk_w, cudaStream_t st);
 int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv, int* expert_count,
-                    int* tile_expert, int* src_info, int* slot_of, cudaStream_t st);
+                    int* tile_expert, int* src_info, int* slot_of, int* tile_count, int* rows_done,
+                    cudaStream_t st);
 int launch_combine(moe_plan* p, const void* rows, const int* slot_of, const float* topk_w, void* y,
                    cudaStream_t st);
 int launch_ffn_simt(moe_plan* p, const void* recv, const int* tile_expert, const void* wg,
                     const void* wu, const void* wd, void* out_rows, cudaStream_t st);
-// gate_on_dispatch: the GEMM1 producer waits for the dispatch counters of this plan (tile_count,
-// rows_done) before it reads a tile; false when the rows come from somewhere else.
+// tile_count / rows_done: availability counters the GEMM1 producer waits on before it reads a tile
+// (nullptr: the rows are complete when the kernel starts).
 int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const void* wg,
-                  const void* wu, const void* wd, void* out_rows, bool gate_on_dispatch, cudaStream_t st);
+                  const void* wu, const void* wd, void* out_rows, const int* tile_count,
+                  const int* rows_done, cudaStream_t st);
 
 // ---- element helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ float to_float(float v) { return v; }

@@ -298,12 +298,14 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
 __global__ void __launch_bounds__(kDispThreads)
 reset_kernel(int* __restrict__ counters, int n_counters, int* __restrict__ expert_count, int E,
              int* __restrict__ tile_expert, int P, int* __restrict__ src_info, int n_src,
-             int* __restrict__ tile_table, int n_table, int* __restrict__ tile_count) {
+             int* __restrict__ tile_table, int n_table, int* __restrict__ tile_count,
+             int* __restrict__ rows_done) {
   const int stride = gridDim.x * kDispThreads;
   const int i0 = blockIdx.x * kDispThreads + threadIdx.x;
   pdl_wait();
   pdl_trigger();
   for (int i = i0; i < n_counters; i += stride) counters[i] = 0;
+  if (i0 == 0) *rows_done = 0;
   for (int i = i0; i < E; i += stride) expert_count[i] = 0;
   for (int i = i0; i < P; i += stride) {
     tile_expert[i] = -1;
@@ -315,7 +317,8 @@ reset_kernel(int* __restrict__ counters, int n_counters, int* __restrict__ exper
 
 // ------------------------------------------------------------------------------------------------
 int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv, int* expert_count,
-                    int* tile_expert, int* src_info, int* slot_of, cudaStream_t st) {
+                    int* tile_expert, int* src_info, int* slot_of, int* tile_count, int* rows_done,
+                    cudaStream_t st) {
   const moe_config_t& c = p->cfg;
   const int eb = c.dtype == MOE_DTYPE_BF16 ? 2 : 4;
   const int vec_per_row = c.H * eb / 16;
@@ -327,7 +330,7 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
     const int grid = (int)max(1ll, (most + 4 * kDispThreads - 1) / (4 * kDispThreads));
     launch_pdl(reset_kernel, dim3(grid), dim3(kDispThreads), 0, st, p->s.status,
                (int)(p->counters_bytes / sizeof(int)), expert_count, c.E, tile_expert, (int)p->P, src_info,
-               (int)(p->P * kTileRows), p->s.tile_table, table, p->s.tile_count);
+               (int)(p->P * kTileRows), p->s.tile_table, table, tile_count, rows_done);
     p->launches += 1;
   }
   if (c.T == 0) return 0;
@@ -339,8 +342,7 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
                expert_count, p->s.tile_base, tile_expert, p->s.scan_ticket);
     const size_t smem = sizeof(int) * ((kDispThreads / 32) * c.E + kMaxAssign);
     launch_maybe_pdl(false, scatter_kernel, dim3(nblk), dim3(kDispThreads), smem, st, (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb,
-               vec_per_row, p->s.cta_base, p->s.tile_base, (uint4*)recv, src_info, slot_of, p->s.tile_count,
-               p->s.rows_done);
+               vec_per_row, p->s.cta_base, p->s.tile_base, (uint4*)recv, src_info, slot_of, tile_count, rows_done);
     p->launches += 3;
   } else {
     const size_t smem = sizeof(int) * (2 * c.E + kMaxAssign);
@@ -348,7 +350,7 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
     auto kern = c.dispatch_mode == MOE_DISPATCH_ATOMIC_PAGED ? dispatch_atomic_kernel<true> : dispatch_atomic_kernel<false>;
     launch_pdl(kern, dim3(nblk), dim3(kDispThreads), smem, st, (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row,
                (int)p->cap_rows, (int)p->P, p->tiles_per_expert, spin, expert_count, p->s.tile_table, p->s.pool_next,
-               tile_expert, (uint4*)recv, src_info, slot_of, p->s.status, p->s.tile_count, p->s.rows_done);
+               tile_expert, (uint4*)recv, src_info, slot_of, p->s.status, tile_count, rows_done);
     p->launches += 1;
   }
   return (int)cudaGetLastError();

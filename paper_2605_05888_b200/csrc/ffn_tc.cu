@@ -165,6 +165,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   const uint32_t tmem_base = sh->tmem_base;
   volatile int* abort_flag = &sh->abort_flag;
   ClockProbe probe(prm.clock_probe);
+  const unsigned long long wait_ns = prm.wait_ns;
 
   const int NB1 = (F + 127) / 128, NB2 = (H + 255) / 256;
   const int KB1 = (H + kBK - 1) / kBK, KB2 = (F + kBK - 1) / kBK;
@@ -207,7 +208,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
           if (ld_acquire(&tile_count[it.tile]) < kTileRows && ld_acquire(rows_done) < total_rows) {
             const unsigned long long t0 = globaltimer();
             while (ld_acquire(&tile_count[it.tile]) < kTileRows && ld_acquire(rows_done) < total_rows) {
-              if (*abort_flag || globaltimer() - t0 > kWaitNs) { fail_site = kWaitTileReady; break; }
+              if (*abort_flag || globaltimer() - t0 > wait_ns) { fail_site = kWaitTileReady; break; }
               __nanosleep(64);
             }
             if (fail_site) break;
@@ -221,7 +222,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
           if (ld_acquire(&gemm1_done[it.tile]) < need) {
             const unsigned long long t0 = globaltimer();
             while (ld_acquire(&gemm1_done[it.tile]) < need) {
-              if (*abort_flag || globaltimer() - t0 > kWaitNs) { fail_site = kWaitTileReady; break; }
+              if (*abort_flag || globaltimer() - t0 > wait_ns) { fail_site = kWaitTileReady; break; }
               __nanosleep(64);
             }
             if (fail_site) break;
@@ -231,7 +232,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
         const CUtensorMap* ma = it.type == 0 ? &map_a1 : &map_a2;
         const int KB = it.type == 0 ? KB1 : KB2;
         for (int kb = 0; kb < KB; ++kb) {
-          if (!mbar_wait(smem_u32(&sh->empty[stage]), phase_bit ^ 1u, abort_flag)) { fail_site = kWaitMbarTma; break; }
+          if (!mbar_wait(smem_u32(&sh->empty[stage]), phase_bit ^ 1u, abort_flag, wait_ns)) { fail_site = kWaitMbarTma; break; }
           const uint32_t full = smem_u32(&sh->full[stage]);
           const uint32_t a_dst = smem_u32(stage_base + stage * kStageBytes);
           const uint32_t b_dst = a_dst + kABytes;
@@ -258,7 +259,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
           const uint32_t par = (uint32_t)((armed[s] - 1) & 1);
           const unsigned long long t0 = globaltimer();
           while (!mbar_try(smem_u32(&sh->full[s]), par))
-            if (globaltimer() - t0 > kWaitNs) break;
+            if (globaltimer() - t0 > wait_ns) break;
         }
       }
     }
@@ -273,11 +274,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
         const int KB = it.type == 0 ? KB1 : KB2;
         const int acc = local_item & 1;
         const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
-        if (!mbar_wait(smem_u32(&sh->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) { fail_site = kWaitMbarTmemFree; break; }
+        if (!mbar_wait(smem_u32(&sh->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, wait_ns)) { fail_site = kWaitMbarTmemFree; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kUmmaN);
         for (int kb = 0; kb < KB; ++kb) {
-          if (!mbar_wait(smem_u32(&sh->full[stage]), phase_bit, abort_flag)) { fail_site = kWaitMbarMma; break; }
+          if (!mbar_wait(smem_u32(&sh->full[stage]), phase_bit, abort_flag, wait_ns)) { fail_site = kWaitMbarMma; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(stage_base + stage * kStageBytes);
           const uint64_t adesc = smem_desc_sw128(a_addr);
@@ -302,7 +303,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       const Item it = decode(item);
       const int acc = local_item & 1;
       const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
-      if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag, 500)) { fail_site = kWaitMbarEpi; break; }
+      if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag, wait_ns, 500)) { fail_site = kWaitMbarEpi; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kUmmaN);
       const size_t row = (size_t)it.tile * kTileRows + row_in_tile;
@@ -411,7 +412,7 @@ static int make_map_3d(EncodeTiledFn enc, CUtensorMap* m, const void* base, uint
 }
 
 int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const void* wg, const void* wu,
-                  const void* wd, void* out_rows, bool gate_on_dispatch, cudaStream_t st) {
+                  const void* wd, void* out_rows, const int* tile_count, const int* rows_done, cudaStream_t st) {
   const moe_config_t& c = p->cfg;
   if (p->P == 0 || c.T == 0) return 0;
   EncodeTiledFn enc;
@@ -453,8 +454,9 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   prm.inter = (__nv_bfloat16*)p->s.inter;
   prm.out = (__nv_bfloat16*)out_rows;
   prm.gemm1_done = p->s.gemm1_done;
-  prm.tile_count = gate_on_dispatch ? p->s.tile_count : nullptr;
-  prm.rows_done = p->s.rows_done;
+  prm.tile_count = tile_count;
+  prm.rows_done = rows_done;
+  prm.wait_ns = c.wait_limit_ns ? c.wait_limit_ns : kDefaultWaitNs;
   prm.total_rows = c.T * c.K;
   prm.status = p->s.status;
   prm.clock_probe = reinterpret_cast<unsigned long long*>(p->s.clock_probe);

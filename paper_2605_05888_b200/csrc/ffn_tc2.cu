@@ -129,6 +129,7 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
   const uint32_t tmem_base = sh->tmem_base;
   volatile int* abort_flag = &sh->abort_flag;
   ClockProbe probe(prm.clock_probe);
+  const unsigned long long wait_ns = prm.wait_ns;
 
   const int NB1 = (F + 127) / 128, NB2 = (H + 255) / 256;
   const int KB1 = (H + kBK - 1) / kBK, KB2 = (F + kBK - 1) / kBK;
@@ -175,7 +176,7 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
           if (ld_acquire(&prm.tile_count[it.tile]) < kTileRows && ld_acquire(prm.rows_done) < prm.total_rows) {
             const unsigned long long t0 = globaltimer();
             while (ld_acquire(&prm.tile_count[it.tile]) < kTileRows && ld_acquire(prm.rows_done) < prm.total_rows) {
-              if (*abort_flag || globaltimer() - t0 > kWaitNs) { fail_site = kWaitTileReady; break; }
+              if (*abort_flag || globaltimer() - t0 > wait_ns) { fail_site = kWaitTileReady; break; }
               __nanosleep(64);
             }
             if (fail_site) break;
@@ -187,7 +188,7 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
           if (ld_acquire(&prm.gemm1_done[it.tile]) < need) {
             const unsigned long long t0 = globaltimer();
             while (ld_acquire(&prm.gemm1_done[it.tile]) < need) {
-              if (*abort_flag || globaltimer() - t0 > kWaitNs) { fail_site = kWaitTileReady; break; }
+              if (*abort_flag || globaltimer() - t0 > wait_ns) { fail_site = kWaitTileReady; break; }
               __nanosleep(64);
             }
             if (fail_site) break;
@@ -199,7 +200,7 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
         const int b_row = it.type == 0 ? it.nb * 128 : it.nb * 256 + (int)rank * 128;
         const int KB = it.type == 0 ? KB1 : KB2;
         for (int kb = 0; kb < KB; ++kb) {
-          if (!mbar_wait(smem_u32(&sh->empty[stage]), phase_bit ^ 1u, abort_flag)) { fail_site = kWaitMbarTma; break; }
+          if (!mbar_wait(smem_u32(&sh->empty[stage]), phase_bit ^ 1u, abort_flag, wait_ns)) { fail_site = kWaitMbarTma; break; }
           const uint32_t full_leader = map_to_cta(smem_u32(&sh->full[stage]), 0);
           const uint32_t a_dst = smem_u32(stage_base + stage * kStageBytes2);
           mbar_expect_tx_cluster(full_leader, kStageBytes2);
@@ -229,11 +230,11 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
         const int KB = it.type == 0 ? KB1 : KB2;
         const int acc = local_item & 1;
         const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
-        if (!mbar_wait(smem_u32(&sh->tmem_empty[acc]), acc_phase ^ 1u, abort_flag)) { fail_site = kWaitMbarTmemFree; break; }
+        if (!mbar_wait(smem_u32(&sh->tmem_empty[acc]), acc_phase ^ 1u, abort_flag, wait_ns)) { fail_site = kWaitMbarTmemFree; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * kUmmaN);
         for (int kb = 0; kb < KB; ++kb) {
-          if (!mbar_wait(smem_u32(&sh->full[stage]), phase_bit, abort_flag)) { fail_site = kWaitMbarMma; break; }
+          if (!mbar_wait(smem_u32(&sh->full[stage]), phase_bit, abort_flag, wait_ns)) { fail_site = kWaitMbarMma; break; }
           tc_fence_after();
           const uint32_t a_addr = smem_u32(stage_base + stage * kStageBytes2);
           const uint64_t adesc = smem_desc_sw128(a_addr);
@@ -259,7 +260,7 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
       const Item it = decode(item, fill);
       const int acc = local_item & 1;
       const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
-      if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag, 500)) { fail_site = kWaitMbarEpi; break; }
+      if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag, wait_ns, 500)) { fail_site = kWaitMbarEpi; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kUmmaN);
       if (it.tile >= 0) {

@@ -14,7 +14,7 @@ constexpr int kABytes = kTileRows * kBK * 2;  // 16 KB
 constexpr int kBBytes = kUmmaN * kBK * 2;     // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kTcSmem = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr unsigned long long kWaitNs = 2000000000ull;  // 2 s bound on any single wait
+constexpr unsigned long long kDefaultWaitNs = 2000000000ull;  // default bound on any single wait: 2 s
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -45,7 +45,7 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // sleep_ns > 0 backs off between polls: for waits that are long by design (an epilogue warp waiting
 // for a whole main loop) polling at full rate only burns power the tensor pipe could use.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          unsigned sleep_ns = 0) {
+                                          unsigned long long limit_ns, unsigned sleep_ns = 0) {
   if (mbar_try(bar, parity)) return true;
   const unsigned long long t0 = globaltimer();
   for (unsigned it = 1;; ++it) {
@@ -53,7 +53,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try(bar, parity)) return true;
     if ((it & 31u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer() - t0 > kWaitNs) return false;
+      if (globaltimer() - t0 > limit_ns) return false;
     }
   }
 }
@@ -126,6 +126,7 @@ struct FfnParams {
   const int* tile_count;
   const int* rows_done;
   int total_rows;
+  unsigned long long wait_ns;  // bound on every wait inside the kernel
   int* status;
   unsigned long long* clock_probe;  // [2]: SM cycles and nanoseconds CTA 0 spent in the kernel (accumulated)
 };

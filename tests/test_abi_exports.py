@@ -33,7 +33,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_config_struct_matches_header():
-    assert ctypes.sizeof(B.MoeConfig) == 12 * 4 + 8 + 8
+    assert ctypes.sizeof(B.MoeConfig) == 12 * 4 + 8 + 8 + 8
 
 
 def test_host_side_checks_without_gpu(lib):

@@ -224,3 +224,70 @@ def test_bad_arguments_are_refused_on_the_host():
         B.moe_workspace_bytes(B.make_config(16, 128, 8, 3, 2, 64, BF16))   # E % R != 0
     with pytest.raises(B.MoeError):
         B.moe_workspace_bytes(B.make_config(16, 128, 8, 2, 9, 64, BF16))   # K > E
+
+
+# ------------------------------------------------------------------ availability counters and the bounded wait
+def _dispatch_with_counters(w, plan, dx, didx):
+    rows = plan.P * 128
+    b = dict(recv=torch.zeros((rows, w.H), dtype=Hh.el_dtype(w), device="cuda"),
+             cnt=torch.empty(w.E, dtype=torch.int32, device="cuda"), te=torch.empty(plan.P, dtype=torch.int32, device="cuda"),
+             src=torch.empty(rows, dtype=torch.int32, device="cuda"),
+             slot=torch.empty((w.T, w.K), dtype=torch.int32, device="cuda"),
+             tile_count=torch.full((plan.P,), 77, dtype=torch.int32, device="cuda"),
+             rows_done=torch.full((1,), 77, dtype=torch.int32, device="cuda"))
+    plan.moe_dispatch(dx, didx, b["recv"], b["cnt"], b["te"], b["src"], b["slot"], b["tile_count"], b["rows_done"])
+    return b
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_dispatch_availability_counters_and_gated_consumer(mode):
+    """Section IV-D in software: after dispatch every tile's status counter equals the rows stored in it
+    and the global counter equals T*K; the tensor-core consumer gated on those counters gives the same
+    result as the ungated one."""
+    w = SMALL[3]
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    plan = Hh.make_plan(w, mode)
+    dx = Hh.to_dev(x)
+    b = _dispatch_with_counters(w, plan, dx, Hh.to_dev(ref["topk_idx"]))
+    torch.cuda.synchronize()
+    assert int(b["rows_done"][0]) == w.T * w.K
+    per_tile = torch.bincount(b["slot"].flatten().long() // 128, minlength=plan.P).int()
+    assert torch.equal(b["tile_count"], per_tile)
+    out = torch.zeros_like(b["recv"])
+    plan.moe_expert_ffn(b["recv"], b["te"], Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd), out, b["tile_count"], b["rows_done"])
+    y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
+    plan.moe_combine(out, b["slot"], Hh.to_dev(ref["topk_w"]), y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+
+
+@pytest.mark.parametrize("kernel", [0, 2])
+def test_consumer_wait_runs_out_and_reports_it(kernel):
+    """A flag that nothing sets: the consumer is given availability counters that stay at zero.  Its
+    bounded wait (50 ms here) runs out, the kernel returns on its own, the status word says timeout
+    and names the wait, and the same plan then runs a correct layer: nothing hangs, the context lives."""
+    w = SMALL[3]
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED, ffn_kernel=kernel, wait_limit_ns=50_000_000)
+    dx, dwg, dwu, dwd = Hh.to_dev(x), Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd)
+    b = _dispatch_with_counters(w, plan, dx, Hh.to_dev(ref["topk_idx"]))
+    never = torch.zeros(plan.P + 1, dtype=torch.int32, device="cuda")
+    out = torch.zeros_like(b["recv"])
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    plan.moe_expert_ffn(b["recv"], b["te"], dwg, dwu, dwd, out, never[:plan.P], never[plan.P:])
+    t1.record()
+    code, detail = plan.moe_last_status()
+    # MOE_ERR_TIMEOUT; the wait site is the producer's tile-availability wait (7) or, since every role's wait
+    # has the same bound, the MMA (4) or epilogue (5) wait that starved behind it: the first to expire is kept
+    assert code == -6 and detail in (7, 4, 5), (code, detail)
+    assert t0.elapsed_time(t1) < 2000.0
+    y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
+    plan.moe_layer(dx, Hh.to_dev(wr), Hh.to_dev(bias), dwg, dwu, dwd, y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
