@@ -15,7 +15,7 @@
 // An expert with an odd number of tiles leaves the peer of its last pair without a tile: that CTA
 // stages the pair's first tile again (valid memory) and stores nothing.
 //
-// No TMA multicast is used: every CTA loads its own bytes.  Synchronisation: per stage, a "full"
+// Every CTA loads its own bytes with plain per-CTA TMA loads.  Synchronisation: per stage, a "full"
 // barrier in the leader (two arrivals + 64 KB of transactions, both CTAs' TMA loads signal it) and an
 // "empty" barrier in each CTA (the leader's tcgen05.commit arrives on both); per accumulator, a "full"
 // barrier in each CTA (commit to both) and an "empty" barrier in the leader that all eight epilogue

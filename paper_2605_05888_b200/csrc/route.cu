@@ -25,7 +25,7 @@ __device__ __forceinline__ void select_topk(const float* ls, int tvalid, int t0,
                                             int* __restrict__ topk_idx, float* __restrict__ topk_w) {
   constexpr int NJ = (EP + 31) / 32;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  for (int tl = warp; tl < tvalid; tl += kRouteThreads / 32) {
+  for (int tl = warp; tl < tvalid; tl += blockDim.x / 32) {
     float v[NJ];
 #pragma unroll
     for (int j = 0; j < NJ; ++j) {
@@ -207,18 +207,18 @@ static int launch_wide(moe_plan* p, const void* x, const void* wr, const float* 
 // memory (fp32, converted while staging), so a lane reads four consecutive h of its token and of its
 // expert with two 16-byte loads and runs its chain over them.  The time is close to the latency of
 // the chain itself (4 cycles per h) once the chunk loads are overlapped.
-template <typename XT, int ROWS, int HC>
+template <typename XT, int ROWS, int HC, int THREADS>
 struct NaturalChunk {
   static constexpr int N = Vec16<XT>::N;
   static constexpr int PARTS = HC / N;
   static constexpr int NVEC = ROWS * PARTS;
-  static constexpr int PER_THREAD = (NVEC + kRouteThreads - 1) / kRouteThreads;
+  static constexpr int PER_THREAD = (NVEC + THREADS - 1) / THREADS;
   static constexpr int PITCH = HC + 4;  // floats; rows land on different banks
   uint4 v[PER_THREAD];
   __device__ __forceinline__ void load(const XT* base, int row0, int nrows_valid, int H, int h0) {
 #pragma unroll
     for (int i = 0; i < PER_THREAD; ++i) {
-      const int idx = threadIdx.x + i * kRouteThreads;
+      const int idx = threadIdx.x + i * THREADS;
       const int r = idx / PARTS, part = idx % PARTS;
       const int h = h0 + part * N;
       v[i] = make_uint4(0, 0, 0, 0);
@@ -229,7 +229,7 @@ struct NaturalChunk {
   __device__ __forceinline__ void store(float* s) const {  // s: [ROWS][PITCH]
 #pragma unroll
     for (int i = 0; i < PER_THREAD; ++i) {
-      const int idx = threadIdx.x + i * kRouteThreads;
+      const int idx = threadIdx.x + i * THREADS;
       if (idx < NVEC) {
         const int r = idx / PARTS, part = idx % PARTS;
         float f[N];
@@ -242,13 +242,13 @@ struct NaturalChunk {
   }
 };
 
-template <typename XT, int LE, int TE, int HC>
-__global__ void __launch_bounds__(kRouteThreads)
+template <typename XT, int LE, int TE, int HC, int THREADS>
+__global__ void __launch_bounds__(THREADS)
 route_narrow_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias, int T,
                     int H, int E, int K, int renorm, int* __restrict__ topk_idx, float* __restrict__ topk_w) {
   constexpr int EP = LE * TE;              // experts covered (padded)
   constexpr int TW = 32 / LE;              // tokens per warp
-  constexpr int TB = TW * (kRouteThreads / 32);
+  constexpr int TB = TW * (THREADS / 32);
   constexpr int PITCH = HC + 4;
   extern __shared__ __align__(16) float smem[];
   float* xs = smem;               // [TB][PITCH]
@@ -263,8 +263,8 @@ route_narrow_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const f
   float acc[TE];
 #pragma unroll
   for (int i = 0; i < TE; ++i) acc[i] = 0.0f;
-  NaturalChunk<XT, TB, HC> xr;
-  NaturalChunk<XT, EP, HC> wrg;
+  NaturalChunk<XT, TB, HC, THREADS> xr;
+  NaturalChunk<XT, EP, HC, THREADS> wrg;
   pdl_wait();
   pdl_trigger();
   xr.load(x, t0, tvalid, H, 0);
@@ -330,19 +330,19 @@ route_narrow_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const f
   select_topk<EP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w);
 }
 
-template <typename XT, int LE, int TE, int HC>
+template <typename XT, int LE, int TE, int HC, int THREADS>
 static int launch_narrow(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
                          float* topk_w, cudaStream_t st) {
-  constexpr int EP = LE * TE, TB = (32 / LE) * (kRouteThreads / 32);
+  constexpr int EP = LE * TE, TB = (32 / LE) * (THREADS / 32);
   const size_t smem = sizeof(float) * (TB + EP) * (HC + 4);
-  auto kern = route_narrow_kernel<XT, LE, TE, HC>;
+  auto kern = route_narrow_kernel<XT, LE, TE, HC, THREADS>;
   if (smem > 48 * 1024) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
   }
   const moe_config_t& c = p->cfg;
   p->launches += 1;
-  return (int)launch_maybe_pdl(false, kern, dim3((c.T + TB - 1) / TB), dim3(kRouteThreads), smem, st, (const XT*)x,
+  return (int)launch_maybe_pdl(false, kern, dim3((c.T + TB - 1) / TB), dim3(THREADS), smem, st, (const XT*)x,
                          (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w);
 }
 
@@ -350,11 +350,21 @@ template <typename XT>
 static int launch_typed(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
                         float* topk_w, cudaStream_t st) {
   const moe_config_t& c = p->cfg;
-  // Small E is bound by the latency of the chain: one lane per chain, long chunks.
-  if (c.E <= 8) return launch_narrow<XT, 8, 1, 512>(p, x, wr, bias, topk_idx, topk_w, st);
-  if (c.E <= 16) return launch_narrow<XT, 16, 1, 512>(p, x, wr, bias, topk_idx, topk_w, st);
-  if (c.E <= 32) return launch_narrow<XT, 32, 1, 512>(p, x, wr, bias, topk_idx, topk_w, st);
-  if (c.E <= 64) return launch_narrow<XT, 32, 2, 256>(p, x, wr, bias, topk_idx, topk_w, st);
+  // Small E is bound by the latency of the chain: one lane per chain, long chunks; small batches use
+  // 128-thread CTAs so that the blocks spread over more SMs.
+  const bool small = c.T <= 2048;
+  if (c.E <= 8)
+    return small ? launch_narrow<XT, 8, 1, 512, 128>(p, x, wr, bias, topk_idx, topk_w, st)
+                 : launch_narrow<XT, 8, 1, 512, 256>(p, x, wr, bias, topk_idx, topk_w, st);
+  if (c.E <= 16)
+    return small ? launch_narrow<XT, 16, 1, 512, 128>(p, x, wr, bias, topk_idx, topk_w, st)
+                 : launch_narrow<XT, 16, 1, 512, 256>(p, x, wr, bias, topk_idx, topk_w, st);
+  if (c.E <= 32)
+    return small ? launch_narrow<XT, 32, 1, 512, 128>(p, x, wr, bias, topk_idx, topk_w, st)
+                 : launch_narrow<XT, 32, 1, 512, 256>(p, x, wr, bias, topk_idx, topk_w, st);
+  if (c.E <= 64)
+    return small ? launch_narrow<XT, 32, 2, 256, 128>(p, x, wr, bias, topk_idx, topk_w, st)
+                 : launch_narrow<XT, 32, 2, 256, 256>(p, x, wr, bias, topk_idx, topk_w, st);
   return launch_wide<XT>(p, x, wr, bias, topk_idx, topk_w, st);
 }
 
