@@ -12,18 +12,12 @@ namespace moehub {
 constexpr int kTileRows = MOE_TILE_ROWS;
 
 // Device status word: [0] code, [1] detail.  First error wins.
-struct Status {
-  int code;
-  int detail;
-  int pad[2];
-};
-
 __device__ __forceinline__ void set_status(int* status, int code, int detail) {
   if (atomicCAS(status, 0, code) == 0) status[1] = detail;
 }
 
 // Wait sites reported in the detail word of MOE_ERR_TIMEOUT.
-enum WaitSite { kWaitTileTable = 1, kWaitScanTicket = 2, kWaitMbarTma = 3, kWaitMbarMma = 4,
+enum WaitSite { kWaitTileTable = 1, kWaitMbarTma = 3, kWaitMbarMma = 4,
                 kWaitMbarEpi = 5, kWaitMbarTmemFree = 6, kWaitTileReady = 7 };
 
 struct Scratch {          // device pointers carved out of the caller's workspace

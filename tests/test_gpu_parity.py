@@ -291,3 +291,37 @@ def test_consumer_wait_runs_out_and_reports_it(kernel):
     torch.cuda.synchronize()
     assert plan.moe_last_status() == (0, 0)
     Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+
+
+# ------------------------------------------------------------------ random small shapes
+def _random_workloads(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        dtype = BF16 if rng.random() < 0.7 else FP32
+        q = 8 if dtype == BF16 else 4                       # row pitch must be a multiple of 16 bytes
+        E = int(rng.choice([1, 2, 3, 5, 8, 12, 24, 40, 64, 100, 256]))
+        R = int(rng.choice([r for r in (1, 2, 3, 4, 5, 8) if E % r == 0]))
+        K = int(rng.integers(1, min(E, 8) + 1))
+        out.append(inputs.Workload(f"rand{i}", T=int(rng.integers(1, 400)), H=q * int(rng.integers(2, 40)), E=E, R=R,
+                                   K=K, F=q * int(rng.integers(2, 40)), dtype=dtype,
+                                   zipf_s=float(rng.choice([0.0, 1.0])), seed=int(rng.integers(0, 1000))))
+    return out
+
+
+@pytest.mark.parametrize("w", _random_workloads(24, 2024), ids=lambda w: f"{w.name}_T{w.T}_H{w.H}_E{w.E}_K{w.K}_F{w.F}_d{w.dtype}")
+def test_random_small_layers_match_oracle(w):
+    """Seeded random small shapes (ragged T, K = 1 ... 8, E from 1 to 256, odd H and F multiples, both
+    dtypes, biased and unbiased routers), every dispatch scheme, whole layer against the oracle."""
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    for mode in MODES:
+        plan = Hh.make_plan(w, mode)
+        y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
+        plan.moe_layer(Hh.to_dev(x), Hh.to_dev(wr), Hh.to_dev(bias), Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd), y)
+        torch.cuda.synchronize()
+        assert plan.moe_last_status() == (0, 0)
+        Hh.check_route(plan.layer_tensor(0), plan.layer_tensor(1), ref["topk_idx"], ref["topk_w"])
+        Hh.check_dispatch(w, plan.P, x, ref["topk_idx"], ref, plan.layer_tensor(2), plan.layer_tensor(3),
+                          plan.layer_tensor(4), plan.layer_tensor(5), plan.layer_tensor(6))
+        Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
