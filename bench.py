@@ -296,8 +296,8 @@ def run_cuda(args, w: inputs.Workload) -> None:
     else:
         t_ffn = sm["gemm1"] + sm["gemm2"]
         stages["ffn"] = {"ms": t_ffn, "TFLOPs": (gemm1_flops + gemm2_flops) / t_ffn / 1e9,
-                         "launches": 2 if args.ffn_split else 1}
-        if args.ffn_split:
+                         "launches": 2 if sm["gemm2"] > 0 else 1}
+        if sm["gemm2"] > 0:
             stages["ffn_gemm1"] = {"ms": sm["gemm1"], "TFLOPs": gemm1_flops / sm["gemm1"] / 1e9}
             stages["ffn_gemm2"] = {"ms": sm["gemm2"], "TFLOPs": gemm2_flops / sm["gemm2"] / 1e9}
         stages["worklist"] = {"ms": sm["worklist"]}
@@ -346,7 +346,8 @@ def main() -> None:
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ffn-kernel", type=int, default=0, choices=[0, 1, 2],
                     help="0: tcgen05 one CTA per tile (default), 2: tcgen05 CTA pairs, 1: SIMT check path")
-    ap.add_argument("--ffn-split", action="store_true", help="one launch per expert GEMM instead of one for both")
+    ap.add_argument("--ffn-split", type=int, default=0, choices=[0, 1, 2],
+                    help="expert GEMMs: 1 = one launch each, 2 = one launch for both, 0 = library default")
     args = ap.parse_args()
     w = WORKLOADS[args.workload]
     if args.impl == "reference":

@@ -81,16 +81,18 @@ def test_simt_ffn_matches_oracle_bf16(w):
     Hh.assert_output_close(Hh.to_host_f64(g["y"]), ref["y"], w.dtype)
 
 
-@pytest.mark.parametrize("split", [0, 1])
+@pytest.mark.parametrize("split", [1, 2])
 @pytest.mark.parametrize("w", [SMALL[3], SMALL[4], SMALL[5], SMALL[7],
                                inputs.Workload("three_tiles", T=700, H=320, E=4, R=2, K=2, F=392, dtype=BF16)],
                          ids=lambda w: w.name)
-def test_cta_pair_ffn_matches_oracle(w, split):
-    """The cta_group::2 form of the tensor-core expert kernel (two tiles of an expert per MMA; experts with
-    an odd number of tiles leave one CTA of the last pair without work), as one launch and as two."""
+@pytest.mark.parametrize("kernel", [0, 2])
+def test_tensor_core_ffn_forms_match_oracle(w, split, kernel):
+    """Both forms of the tensor-core expert kernel - one CTA per tile (0) and the cta_group::2 form (2: two
+    tiles of an expert per MMA; experts with an odd number of tiles leave one CTA of the last pair without
+    work) - each as one launch for both GEMMs (per-tile counters gate GEMM2) and as two launches."""
     x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
     ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
-    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED, ffn_kernel=2, ffn_split=split)
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED, ffn_kernel=kernel, ffn_split=split)
     y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
     plan.moe_layer(Hh.to_dev(x), Hh.to_dev(wr), Hh.to_dev(bias), Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd), y)
     torch.cuda.synchronize()
