@@ -185,6 +185,18 @@ int moe_layer(moe_plan_t* plan, const void* d_x, const void* d_wr, const float* 
 int moe_layer_host(moe_plan_t* plan, const void* h_x, const void* d_wr, const float* d_bias,
                    const void* d_wg, const void* d_wu, const void* d_wd, void* h_y, void* stream);
 
+/* Pipelined form of moe_layer_host for a stream of batches.  submit() enqueues one step and returns
+ * at once with a ticket: the copy of h_x goes to a copy-in stream, the layer to `stream`, the copy of
+ * y to a copy-out stream, chained by events, with two sets of staging buffers, so that step n+1's
+ * host-to-device copy and step n-1's device-to-host copy run under step n's kernels.  wait(ticket)
+ * blocks the host until that step's h_y is complete.  Keep at most two steps in flight (wait for
+ * ticket n-1 before submitting n+1), leave h_x and h_y alone until their step is waited for, and use
+ * pinned host memory: pageable memory makes the copies synchronous.  Device errors: moe_last_status. */
+int moe_layer_host_submit(moe_plan_t* plan, const void* h_x, const void* d_wr, const float* d_bias,
+                          const void* d_wg, const void* d_wu, const void* d_wd, void* h_y, void* stream,
+                          int64_t* ticket);
+int moe_layer_host_wait(moe_plan_t* plan, int64_t ticket);
+
 /* moe_layer with a CUDA event recorded after every kernel: runs the layer once, synchronises the
  * stream and writes the device time of each stage, in milliseconds, to h_stage_ms
  * [MOE_STAGE_COUNT] (host): route, dispatch (all its kernels and counter resets), FFN work list,

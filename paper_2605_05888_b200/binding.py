@@ -22,7 +22,8 @@ TILE_ROWS = 128
 STAGES = ["route", "dispatch", "worklist", "gemm1", "gemm2", "combine"]
 
 EXPORTS = ["moe_dispatch_noalloc", "moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
-           "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host", "moe_layer_timed", "moe_layer_buffer",
+           "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host", "moe_layer_host_submit", "moe_layer_host_wait", "moe_layer_timed",
+           "moe_layer_buffer",
            "moe_ffn_clock_mhz", "moe_last_launch_count", "moe_last_status", "moe_strerror"]
 
 
@@ -60,6 +61,8 @@ def lib() -> ctypes.CDLL:
         L.moe_combine.argtypes = [vp, vp, i32p, fp, vp, vp]
         L.moe_layer.argtypes = [vp] * 9
         L.moe_layer_host.argtypes = [vp] * 9
+        L.moe_layer_host_submit.argtypes = [vp] * 9 + [ctypes.POINTER(ctypes.c_int64)]
+        L.moe_layer_host_wait.argtypes = [vp, ctypes.c_int64]
         L.moe_layer_timed.argtypes = [vp] * 9 + [ctypes.POINTER(ctypes.c_float)]
         L.moe_layer_buffer.argtypes = [vp, ctypes.c_int, ctypes.POINTER(vp)]
         L.moe_ffn_clock_mhz.argtypes = [vp, vp, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
@@ -179,6 +182,18 @@ class Plan:
         assert not h_x.is_cuda and not h_y.is_cuda
         _check(lib().moe_layer_host(self.handle, _ptr(h_x), _ptr(wr), _ptr(bias), _ptr(wg), _ptr(wu), _ptr(wd),
                                     _ptr(h_y), _stream(stream)), "moe_layer_host")
+
+    def moe_layer_host_submit(self, h_x, wr, bias, wg, wu, wd, h_y, stream=None) -> int:
+        """Pipelined host-buffer step: returns a ticket at once; moe_layer_host_wait(ticket) blocks until h_y is
+        complete. At most two steps in flight; h_x, h_y pinned."""
+        assert not h_x.is_cuda and not h_y.is_cuda
+        t = ctypes.c_int64()
+        _check(lib().moe_layer_host_submit(self.handle, _ptr(h_x), _ptr(wr), _ptr(bias), _ptr(wg), _ptr(wu), _ptr(wd),
+                                           _ptr(h_y), _stream(stream), ctypes.byref(t)), "moe_layer_host_submit")
+        return t.value
+
+    def moe_layer_host_wait(self, ticket: int) -> None:
+        _check(lib().moe_layer_host_wait(self.handle, ticket), "moe_layer_host_wait")
 
     def moe_layer_timed(self, x, wr, bias, wg, wu, wd, y, stream=None) -> list[float]:
         """Runs the layer once with an event after every kernel; returns ms per stage (see STAGES)."""

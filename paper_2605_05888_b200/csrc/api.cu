@@ -91,8 +91,10 @@ size_t carve(const moe_config_t& c, const Geometry& g, char* base, Scratch* s, s
   t.tile_expert = (int*)take(sizeof(int) * (size_t)g.P);
   t.src_info = (int*)take(sizeof(int) * pool_rows);
   t.slot_of = (int*)take(sizeof(int) * (size_t)c.T * c.K);
-  t.x_stage = take((size_t)c.T * c.H * g.eb);
-  t.y_stage = take((size_t)c.T * c.H * g.eb);
+  for (int b = 0; b < 2; ++b) {
+    t.x_stage[b] = take((size_t)c.T * c.H * g.eb);
+    t.y_stage[b] = take((size_t)c.T * c.H * g.eb);
+  }
   if (s) *s = t;
   return off;
 }
@@ -142,6 +144,9 @@ int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, mo
   p->encode_tiled = nullptr;
   p->timing = 0;
   for (int i = 0; i <= MOE_STAGE_COUNT; ++i) p->tev[i] = nullptr;
+  p->copy_in = p->copy_out = nullptr;
+  p->submitted = 0;
+  for (int b = 0; b < 2; ++b) p->ev_in[b] = p->ev_done[b] = p->ev_out[b] = nullptr;
   carve(*cfg, g, (char*)d_workspace, &p->s, &p->counters_bytes);
   if (cudaGetDevice(&p->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device) != cudaSuccess) {
@@ -159,9 +164,17 @@ int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, mo
 }
 
 int moe_plan_destroy(moe_plan_t* plan) {
-  if (plan)
+  if (plan) {
     for (int i = 0; i <= MOE_STAGE_COUNT; ++i)
       if (plan->tev[i]) cudaEventDestroy(plan->tev[i]);
+    for (int b = 0; b < 2; ++b) {
+      if (plan->ev_in[b]) cudaEventDestroy(plan->ev_in[b]);
+      if (plan->ev_done[b]) cudaEventDestroy(plan->ev_done[b]);
+      if (plan->ev_out[b]) cudaEventDestroy(plan->ev_out[b]);
+    }
+    if (plan->copy_in) cudaStreamDestroy(plan->copy_in);
+    if (plan->copy_out) cudaStreamDestroy(plan->copy_out);
+  }
   delete plan;
   return MOE_OK;
 }
@@ -270,13 +283,57 @@ int moe_layer_host(moe_plan_t* p, const void* h_x, const void* d_wr, const float
   if (p->cfg.T > 0 && (!h_x || !h_y)) return MOE_ERR_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   const size_t bytes = (size_t)p->cfg.T * p->cfg.H * (p->cfg.dtype == MOE_DTYPE_BF16 ? 2 : 4);
-  if (bytes && cudaMemcpyAsync(p->s.x_stage, h_x, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+  if (bytes && cudaMemcpyAsync(p->s.x_stage[0], h_x, bytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return MOE_ERR_CUDA;
-  int rc = moe_layer(p, p->s.x_stage, d_wr, d_bias, d_wg, d_wu, d_wd, p->s.y_stage, stream);
+  int rc = moe_layer(p, p->s.x_stage[0], d_wr, d_bias, d_wg, d_wu, d_wd, p->s.y_stage[0], stream);
   if (rc != MOE_OK) return rc;
-  if (bytes && cudaMemcpyAsync(h_y, p->s.y_stage, bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+  if (bytes && cudaMemcpyAsync(h_y, p->s.y_stage[0], bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return MOE_ERR_CUDA;
   return cudaStreamSynchronize(st) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+int moe_layer_host_submit(moe_plan_t* p, const void* h_x, const void* d_wr, const float* d_bias, const void* d_wg,
+                          const void* d_wu, const void* d_wd, void* h_y, void* stream, int64_t* ticket) {
+  if (!p || !ticket) return MOE_ERR_ARG;
+  if (p->cfg.T > 0 && (!h_x || !h_y)) return MOE_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (!p->copy_in) {
+    if (cudaStreamCreateWithFlags(&p->copy_in, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&p->copy_out, cudaStreamNonBlocking) != cudaSuccess)
+      return MOE_ERR_CUDA;
+    for (int b = 0; b < 2; ++b)
+      if (cudaEventCreateWithFlags(&p->ev_in[b], cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&p->ev_done[b], cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&p->ev_out[b], cudaEventDisableTiming) != cudaSuccess)
+        return MOE_ERR_CUDA;
+  }
+  const int b = (int)(p->submitted & 1);
+  const bool reuse = p->submitted >= 2;  // buffer b was used by step n-2
+  const size_t bytes = (size_t)p->cfg.T * p->cfg.H * (p->cfg.dtype == MOE_DTYPE_BF16 ? 2 : 4);
+  // copy-in stream: x_stage[b] is free once step n-2's layer has run
+  if (reuse && cudaStreamWaitEvent(p->copy_in, p->ev_done[b], 0) != cudaSuccess) return MOE_ERR_CUDA;
+  if (bytes && cudaMemcpyAsync(p->s.x_stage[b], h_x, bytes, cudaMemcpyHostToDevice, p->copy_in) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (cudaEventRecord(p->ev_in[b], p->copy_in) != cudaSuccess) return MOE_ERR_CUDA;
+  // compute stream: needs this step's x, and y_stage[b] drained by step n-2's copy-out
+  if (cudaStreamWaitEvent(st, p->ev_in[b], 0) != cudaSuccess) return MOE_ERR_CUDA;
+  if (reuse && cudaStreamWaitEvent(st, p->ev_out[b], 0) != cudaSuccess) return MOE_ERR_CUDA;
+  int rc = moe_layer(p, p->s.x_stage[b], d_wr, d_bias, d_wg, d_wu, d_wd, p->s.y_stage[b], stream);
+  if (rc != MOE_OK) return rc;
+  if (cudaEventRecord(p->ev_done[b], st) != cudaSuccess) return MOE_ERR_CUDA;
+  // copy-out stream
+  if (cudaStreamWaitEvent(p->copy_out, p->ev_done[b], 0) != cudaSuccess) return MOE_ERR_CUDA;
+  if (bytes && cudaMemcpyAsync(h_y, p->s.y_stage[b], bytes, cudaMemcpyDeviceToHost, p->copy_out) != cudaSuccess)
+    return MOE_ERR_CUDA;
+  if (cudaEventRecord(p->ev_out[b], p->copy_out) != cudaSuccess) return MOE_ERR_CUDA;
+  *ticket = p->submitted++;
+  return MOE_OK;
+}
+
+int moe_layer_host_wait(moe_plan_t* p, int64_t ticket) {
+  if (!p || ticket < 0 || ticket >= p->submitted) return MOE_ERR_ARG;
+  if (ticket < p->submitted - 2) return MOE_OK;  // its buffer has been reused: that step finished long ago
+  return cudaEventSynchronize(p->ev_out[ticket & 1]) == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }
 
 int moe_layer_buffer(moe_plan_t* p, int which, void** out_ptr) {

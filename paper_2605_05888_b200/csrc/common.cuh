@@ -47,8 +47,8 @@ struct Scratch {          // device pointers carved out of the caller's workspac
   int* tile_expert;
   int* src_info;
   int* slot_of;
-  void* x_stage;          // [T,H] device copy of host x (moe_layer_host)
-  void* y_stage;          // [T,H]
+  void* x_stage[2];       // [T,H] device copies of host x (moe_layer_host; two for the pipelined form)
+  void* y_stage[2];       // [T,H]
 };
 
 }  // namespace moehub
@@ -66,6 +66,10 @@ struct moe_plan {
   size_t counters_bytes;     // leading part of the workspace cleared by dispatch
   moehub::Scratch s;
   void* encode_tiled;        // cuTensorMapEncodeTiled entry point (driver API), looked up once
+  // moe_layer_host_submit / _wait: copy streams and per-buffer events (host resources, made on first use)
+  cudaStream_t copy_in, copy_out;
+  cudaEvent_t ev_in[2], ev_done[2], ev_out[2];
+  long long submitted;       // steps submitted so far
   int timing;                // moe_layer_timed: record an event after every kernel of the layer
   cudaEvent_t tev[MOE_STAGE_COUNT + 1];
 };

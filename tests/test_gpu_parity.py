@@ -327,3 +327,27 @@ def test_random_small_layers_match_oracle(w):
         Hh.check_dispatch(w, plan.P, x, ref["topk_idx"], ref, plan.layer_tensor(2), plan.layer_tensor(3),
                           plan.layer_tensor(4), plan.layer_tensor(5), plan.layer_tensor(6))
         Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+
+
+def test_pipelined_host_steps_match_single_steps():
+    """moe_layer_host_submit / _wait with two steps in flight: five batches, each result identical to
+    the same batch run alone through moe_layer (bit for bit: same kernels, same order)."""
+    w = SMALL[3]
+    _, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    dwr, dbias, dwg, dwu, dwd = (Hh.to_dev(a) for a in (wr, bias, wg, wu, wd))
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED)
+    xs = [inputs.make_x(w.with_(seed=10 + i)) for i in range(5)]
+    hx = [torch.from_numpy(x.view(np.int16)).pin_memory() for x in xs]
+    hy = [torch.empty_like(h).pin_memory() for h in hx]
+    tickets = []
+    for i in range(5):
+        tickets.append(plan.moe_layer_host_submit(hx[i], dwr, dbias, dwg, dwu, dwd, hy[i]))
+        if i >= 1:
+            plan.moe_layer_host_wait(tickets[i - 1])
+    plan.moe_layer_host_wait(tickets[-1])
+    assert tickets == list(range(5)) and plan.moe_last_status() == (0, 0)
+    for i in range(5):
+        y = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+        plan.moe_layer(Hh.to_dev(xs[i]), dwr, dbias, dwg, dwu, dwd, y)
+        torch.cuda.synchronize()
+        assert np.array_equal(hy[i].numpy().view(np.uint16), Hh.to_host_bits(y)), f"step {i}"
