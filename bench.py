@@ -31,6 +31,8 @@ UNIT = "tokens/s"
 WORKLOADS = {"c1": inputs.C1, "c2": inputs.C2, "c3": inputs.C3, "c4": inputs.C4,
              # a quarter-size C2 (same kernels, 0.7 GB of weights) for ncu captures that must stay small
              "c2_small": inputs.C2.with_(name="mixtral_like_bf16_small", T=2048, E=4, R=4, F=7168),
+             # the other two shapes of the paper's Table II
+             "phi35": inputs.PHI35, "qwen64": inputs.QWEN64,
              # dispatch/combine-only sweep points (identity experts)
              "c5_8192": inputs.C5(8192), "c5_8192_zipf": inputs.C5(8192, 1.2), "c5_2048": inputs.C5(2048)}
 
@@ -299,12 +301,18 @@ def run_cuda(args, w: inputs.Workload) -> None:
     gemm2_flops = 2.0 * rows * w.H * w.F
     sm = dict(zip(B.STAGES, stage_ms.tolist()))
     hbm_peak = peaks["hbm_gbs"]
+    counts = plan.layer_tensor(3).cpu().numpy().astype(np.float64)
+    routing_stats = {"hottest_expert_rows_over_T": float(counts.max() / w.T), "experts_without_rows": int((counts == 0).sum()),
+                     "std_of_expert_share": float(np.std(counts / rows)), "tiles_used": int(np.sum((counts + 127) // 128)),
+                     "tiles_if_dense": int((rows + 127) // 128)}
     stages = {
         "route": {"ms": sm["route"], "GBps": route_bytes / sm["route"] / 1e6 if sm["route"] > 0 else None},
         "dispatch": {"ms": sm["dispatch"], "GBps": disp_bytes / sm["dispatch"] / 1e6,
-                     "frac_hbm": disp_bytes / sm["dispatch"] / 1e6 / hbm_peak, "mode": args.dispatch},
+                     "frac_hbm": disp_bytes / sm["dispatch"] / 1e6 / hbm_peak,
+                     "frac_hbm_nominal_8TBps": disp_bytes / sm["dispatch"] / 1e6 / 8000.0, "mode": args.dispatch},
         "combine": {"ms": sm["combine"], "GBps": comb_bytes / sm["combine"] / 1e6,
-                    "frac_hbm": comb_bytes / sm["combine"] / 1e6 / hbm_peak},
+                    "frac_hbm": comb_bytes / sm["combine"] / 1e6 / hbm_peak,
+                    "frac_hbm_nominal_8TBps": comb_bytes / sm["combine"] / 1e6 / 8000.0},
     }
     if w.identity_experts or w.dtype != inputs.BF16:
         dom = "dispatch"
@@ -326,6 +334,7 @@ def run_cuda(args, w: inputs.Workload) -> None:
                     "peak_source": f"{peak_kind} bf16_tflops (burst); the kernel runs power-capped at the clock in "
                                    "clocks.ffn_kernel_sm_mhz",
                     "frac_of_sustained_peak": ach / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                    "frac_of_nominal_2250": ach / 2250.0,
                     "useful_flops_per_launch": gemm1_flops + gemm2_flops}
 
     # the CPU oracle on a bounded sample of the same batch (N = 1 only)
@@ -349,7 +358,8 @@ def run_cuda(args, w: inputs.Workload) -> None:
                     "d2h_bytes_per_step": h2d,
                     "api": "moe_layer_host_submit/_wait: pinned host x and y, two steps in flight, host wall clock",
                     "one_step_at_a_time": whole_job_tokens_per_s(w.T, world, ms_e2e_sync / args.steps)},
-            "roofline": roofline, "cpu_baseline": cpu, "stages": stages, "dominant": roofline["kernel"]}
+            "roofline": roofline, "cpu_baseline": cpu, "stages": stages, "dominant": roofline["kernel"],
+            "routing": routing_stats}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

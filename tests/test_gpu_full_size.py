@@ -76,6 +76,16 @@ def test_c4_qwen_like_full_size(mode):
     Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
 
 
+@pytest.mark.parametrize("w", [inputs.PHI35, inputs.QWEN64], ids=lambda w: w.name)
+def test_other_table2_shapes(w):
+    """Phi-3.5-MoE and Qwen2-MoE (64 experts) shapes of the paper's Table II: routing and dispatch in full,
+    output on sampled tokens."""
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    plan, y = run_layer(w, B.DISPATCH_ATOMIC_PAGED, x, wr, bias, Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd))
+    check_full_routing_and_dispatch(w, plan, x, wr, bias)
+    check_sampled_output(w, y, x, wr, bias, wg, wu, wd, 32)
+
+
 @pytest.mark.parametrize("zipf", [0.0, 1.2])
 def test_c5_sweep_point_8192_against_oracle(zipf):
     w = inputs.C5(8192, zipf)
