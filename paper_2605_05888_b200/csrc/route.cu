@@ -194,8 +194,12 @@ static int launch_wide(moe_plan* p, const void* x, const void* wr, const float* 
                        float* topk_w, cudaStream_t st) {
   const size_t smem = sizeof(float) * kWideTB * kWideEP;  // the logits tile; the staging area is smaller
   auto kern = route_wide_kernel<XT>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return (int)e;
+  static bool attr_done = false;  // per instantiation and process, idempotent
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return (int)e;
+    attr_done = true;
+  }
   const moe_config_t& c = p->cfg;
   p->launches += 1;
   return (int)launch_maybe_pdl(false, kern, dim3((c.T + kWideTB - 1) / kWideTB), dim3(kRouteThreads), smem, st, (const XT*)x,
@@ -336,9 +340,11 @@ static int launch_narrow(moe_plan* p, const void* x, const void* wr, const float
   constexpr int EP = LE * TE, TB = (32 / LE) * (THREADS / 32);
   const size_t smem = sizeof(float) * (TB + EP) * (HC + 4);
   auto kern = route_narrow_kernel<XT, LE, TE, HC, THREADS>;
-  if (smem > 48 * 1024) {
+  static bool attr_done = false;  // per instantiation and process, idempotent
+  if (smem > 48 * 1024 && !attr_done) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return (int)e;
+    attr_done = true;
   }
   const moe_config_t& c = p->cfg;
   p->launches += 1;
