@@ -322,11 +322,10 @@ def run_cuda(args, w: inputs.Workload) -> None:
     else:
         t_ffn = sm["gemm1"] + sm["gemm2"]
         stages["ffn"] = {"ms": t_ffn, "TFLOPs": (gemm1_flops + gemm2_flops) / t_ffn / 1e9,
-                         "launches": 2 if sm["gemm2"] > 0 else 1}
-        if sm["gemm2"] > 0:
+                         "launches": 2 if sm["gemm2"] > 0.02 * sm["gemm1"] else 1}
+        if stages["ffn"]["launches"] == 2:
             stages["ffn_gemm1"] = {"ms": sm["gemm1"], "TFLOPs": gemm1_flops / sm["gemm1"] / 1e9}
             stages["ffn_gemm2"] = {"ms": sm["gemm2"], "TFLOPs": gemm2_flops / sm["gemm2"] / 1e9}
-        stages["worklist"] = {"ms": sm["worklist"]}
         ach = stages["ffn"]["TFLOPs"]
         roofline = {"kernel": "ffn_tc_kernel (expert GEMM1 + SwiGLU + GEMM2, tcgen05)", "bound": "tensor",
                     "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],

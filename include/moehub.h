@@ -136,7 +136,9 @@ int moe_dispatch(moe_plan_t* plan, const void* d_x, const int32_t* d_topk_idx, v
  *     tile_count[p] >= 128 or rows_done >= T*K (bounded by wait_limit_ns; on expiry the status
  *     word reads MOE_ERR_TIMEOUT and the kernel returns).  NULL: the rows are complete when the
  *     call is reached in stream order.  The SIMT kernel ignores them (stream order).
- * out: d_out_rows [P*128,H] (dtype); rows of empty slots hold unspecified values. */
+ * out: d_out_rows [P*128,H] (dtype); rows of empty slots hold unspecified values.
+ * The tensor-core kernels keep their work list in shared memory: P <= 4608 tiles (T*K <= 557 056 rows at
+ * E = 256), MOE_ERR_UNSUPPORTED beyond. */
 int moe_expert_ffn(moe_plan_t* plan, const void* d_recv, const int32_t* d_tile_expert,
                    const void* d_wg, const void* d_wu, const void* d_wd, void* d_out_rows,
                    const int32_t* d_tile_count, const int32_t* d_rows_done, void* stream);
@@ -199,8 +201,9 @@ int moe_layer_host_wait(moe_plan_t* plan, int64_t ticket);
 
 /* moe_layer with a CUDA event recorded after every kernel: runs the layer once, synchronises the
  * stream and writes the device time of each stage, in milliseconds, to h_stage_ms
- * [MOE_STAGE_COUNT] (host): route, dispatch (all its kernels and counter resets), FFN work list,
- * FFN GEMM1 (+SwiGLU), FFN GEMM2, combine.  With ffn_split = 0 both GEMMs are one launch: its
+ * [MOE_STAGE_COUNT] (host): route, dispatch (all its kernels and counter resets), FFN set-up (host-side
+ * descriptor encoding only: the work list is built inside the expert kernel), FFN GEMM1 (+SwiGLU), FFN GEMM2,
+ * combine.  With ffn_split = 0 both GEMMs are one launch: its
  * time is reported under GEMM1 and GEMM2 reads 0.  For measurement only. */
 #define MOE_STAGE_ROUTE 0
 #define MOE_STAGE_DISPATCH 1

@@ -74,11 +74,6 @@ size_t carve(const moe_config_t& c, const Geometry& g, char* base, Scratch* s, s
   t.cta_count = (int*)take(sizeof(int) * (size_t)(g.nblk > 0 ? g.nblk : 1) * c.E);
   t.cta_base = (int*)take(sizeof(int) * (size_t)(g.nblk > 0 ? g.nblk : 1) * c.E);
   t.tile_base = (int*)take(sizeof(int) * (size_t)(c.E + 1));
-  t.tile_list = (int*)take(sizeof(int) * (size_t)(g.P > 0 ? g.P : 1));
-  t.expert_start = (int*)take(sizeof(int) * (size_t)(c.E + 1));
-  t.seg_start = (int*)take(sizeof(int) * (size_t)(2 * c.E + 1));
-  t.seg_info = (int*)take(sizeof(int) * (size_t)(2 * c.E));
-  t.work_meta = (int*)take(sizeof(int) * 4);
   t.clock_probe = (unsigned long long*)take(sizeof(unsigned long long) * 2);
   t.gemm1_done = (int*)take(sizeof(int) * (size_t)(g.P > 0 ? g.P : 1));
   const size_t pool_rows = (size_t)g.P * kTileRows;

@@ -30,11 +30,6 @@ struct Scratch {          // device pointers carved out of the caller's workspac
   int* cta_count;         // [nblk * E] mode 0: per token-block histogram
   int* cta_base;          // [nblk * E] mode 0: exclusive prefix inside the expert
   int* tile_base;         // [E + 1]    mode 0: first pool tile of each expert
-  int* tile_list;         // [P]   used tiles grouped by expert (FFN work list)
-  int* expert_start;      // [E + 1] first work-list index of each expert
-  int* seg_start;         // [2E + 1] first item of each work segment
-  int* seg_info;          // [2E]   expert | type << 16 of each segment
-  int* work_meta;         // [4]    [0]: items before the first GEMM2 item (split launches)
   unsigned long long* clock_probe;  // [2] cycles, nanoseconds of CTA 0 inside the tensor-core kernels
   int* gemm1_done;        // [P]    per-tile status counter: GEMM1 blocks finished (x4 epilogue warps)
   void* inter;            // [P*128, F] SwiGLU intermediate

@@ -299,7 +299,7 @@ __global__ void __launch_bounds__(kDispThreads)
 reset_kernel(int* __restrict__ counters, int n_counters, int* __restrict__ expert_count, int E,
              int* __restrict__ tile_expert, int P, int* __restrict__ src_info, int n_src,
              int* __restrict__ tile_table, int n_table, int* __restrict__ tile_count,
-             int* __restrict__ rows_done) {
+             int* __restrict__ rows_done, int* __restrict__ gemm1_done) {
   const int stride = gridDim.x * kDispThreads;
   const int i0 = blockIdx.x * kDispThreads + threadIdx.x;
   pdl_wait();
@@ -310,6 +310,7 @@ reset_kernel(int* __restrict__ counters, int n_counters, int* __restrict__ exper
   for (int i = i0; i < P; i += stride) {
     tile_expert[i] = -1;
     tile_count[i] = 0;
+    gemm1_done[i] = 0;
   }
   for (int i = i0; i < n_table; i += stride) tile_table[i] = -1;
   for (int i = i0; i < n_src; i += stride) src_info[i] = -1;
@@ -330,7 +331,7 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
     const int grid = (int)max(1ll, (most + 4 * kDispThreads - 1) / (4 * kDispThreads));
     launch_pdl(reset_kernel, dim3(grid), dim3(kDispThreads), 0, st, p->s.status,
                (int)(p->counters_bytes / sizeof(int)), expert_count, c.E, tile_expert, (int)p->P, src_info,
-               (int)(p->P * kTileRows), p->s.tile_table, table, tile_count, rows_done);
+               (int)(p->P * kTileRows), p->s.tile_table, table, tile_count, rows_done, p->s.gemm1_done);
     p->launches += 1;
   }
   if (c.T == 0) return 0;

@@ -31,77 +31,6 @@
 
 namespace moehub {
 
-// ---- work list ------------------------------------------------------------------------------
-// tile_list: the used tiles grouped by expert; expert_start[e]: first index of expert e's tiles,
-// expert_start[E] = number of used tiles.  Segments: the item sequence is a list of at most 2E
-// segments, segment = all GEMM1 items or all GEMM2 items of one expert; seg_start[i] is the first
-// item of segment i (seg_start[2E] = number of items), seg_info[i] = expert | type << 16
-// (type 0: GEMM1, 1: GEMM2).  pair = 2 counts one item per PAIR of tiles (CTA-pair kernel).  meta[0] = number of items that precede the first GEMM2 item when the
-// launch is split in two phases.
-__global__ void __launch_bounds__(256)
-worklist_kernel(const int* __restrict__ tile_expert, int P, int E, int NB1, int NB2, int lag, int fused, int pair,
-                int* __restrict__ tile_list, int* __restrict__ expert_start, int* __restrict__ seg_start,
-                int* __restrict__ seg_info, int* __restrict__ meta, int* __restrict__ gemm1_done) {
-  __shared__ int s_cnt[kMaxExperts];
-  __shared__ int s_cur[kMaxExperts];
-  __shared__ int s_warp[8];
-  const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
-  s_cnt[threadIdx.x] = 0;
-  __syncthreads();
-  pdl_wait();
-  pdl_trigger();
-  for (int p = threadIdx.x; p < P; p += 256) {
-    gemm1_done[p] = 0;
-    const int e = tile_expert[p];
-    if (e >= 0 && e < E) atomicAdd(&s_cnt[e], 1);
-  }
-  __syncthreads();
-  const int c = s_cnt[threadIdx.x];
-  int incl = c;
-#pragma unroll
-  for (int off = 1; off < 32; off <<= 1) {
-    const int n = __shfl_up_sync(0xffffffffu, incl, off);
-    if (lane >= off) incl += n;
-  }
-  if (lane == 31) s_warp[warp] = incl;
-  __syncthreads();
-  int wbase = 0;
-  for (int w = 0; w < warp; ++w) wbase += s_warp[w];
-  const int first = wbase + incl - c;
-  s_cur[threadIdx.x] = first;
-  if (threadIdx.x < E) expert_start[threadIdx.x] = first;
-  if (threadIdx.x == E - 1) expert_start[E] = first + c;
-  __syncthreads();
-  for (int p = threadIdx.x; p < P; p += 256) {
-    const int e = tile_expert[p];
-    if (e >= 0 && e < E) tile_list[atomicAdd(&s_cur[e], 1)] = p;
-  }
-  if (threadIdx.x == 0) {
-    // Item order.  Split launches: all GEMM1 segments, then all GEMM2 segments.  One launch: the GEMM2
-    // segment of an expert follows once at least `lag` items were placed after its GEMM1 segment.
-    int pos = 0, nseg = 0, q = 0;
-    for (int e = 0; e < E; ++e) {
-      seg_start[nseg] = pos;
-      seg_info[nseg++] = e;
-      pos += (s_cnt[e] + pair - 1) / pair * NB1;
-      s_cur[e] = pos;  // end of this expert's GEMM1 items
-      while (fused && q < e && pos - s_cur[q] >= lag) {
-        seg_start[nseg] = pos;
-        seg_info[nseg++] = q | (1 << 16);
-        pos += (s_cnt[q] + pair - 1) / pair * NB2;
-        ++q;
-      }
-    }
-    meta[0] = fused ? 0 : pos;
-    for (; q < E; ++q) {
-      seg_start[nseg] = pos;
-      seg_info[nseg++] = q | (1 << 16);
-      pos += (s_cnt[q] + pair - 1) / pair * NB2;
-    }
-    seg_start[nseg] = pos;  // nseg == 2E
-  }
-}
-
 // ---- the grouped GEMM -----------------------------------------------------------------------
 struct TcShared {
   unsigned long long full[kStages];
@@ -116,11 +45,6 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_bg,
               const __grid_constant__ CUtensorMap map_bu, const __grid_constant__ CUtensorMap map_a2,
               const __grid_constant__ CUtensorMap map_bd, const FfnParams prm) {
-  const int* __restrict__ tile_list = prm.tile_list;
-  const int* __restrict__ expert_start = prm.expert_start;
-  const int* __restrict__ seg_start = prm.seg_start;
-  const int* __restrict__ seg_info = prm.seg_info;
-  const int* __restrict__ meta = prm.meta;
   const int phase = prm.phase, E = prm.E, F = prm.F, H = prm.H;
   __nv_bfloat16* __restrict__ inter = prm.inter;
   __nv_bfloat16* __restrict__ out = prm.out;
@@ -132,9 +56,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   uint8_t* stage_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   TcShared* sh = reinterpret_cast<TcShared*>(stage_base + kStages * kStageBytes);
-  __shared__ int s_estart[kMaxExperts + 1];
-  __shared__ int s_seg_start[2 * kMaxExperts + 1];
-  __shared__ int s_seg_info[2 * kMaxExperts];
+  __shared__ WorkList wl;
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int nseg = 2 * E;
@@ -156,9 +78,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   pdl_wait();  // everything above needs no global data and overlaps the predecessor's tail
-  for (int i = threadIdx.x; i <= E; i += kTcThreads) s_estart[i] = expert_start[i];
-  for (int i = threadIdx.x; i <= nseg; i += kTcThreads) s_seg_start[i] = seg_start[i];
-  for (int i = threadIdx.x; i < nseg; i += kTcThreads) s_seg_info[i] = seg_info[i];
+  build_worklist(wl, prm.tile_expert, prm.P, E, (F + 127) / 128, (H + 255) / 256, prm.lag, prm.fused, 1);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -169,24 +89,24 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
 
   const int NB1 = (F + 127) / 128, NB2 = (H + 255) / 256;
   const int KB1 = (H + kBK - 1) / kBK, KB2 = (F + kBK - 1) / kBK;
-  int item_begin = 0, item_end = s_seg_start[nseg];
-  if (phase == 1) item_end = meta[0];
-  if (phase == 2) item_begin = meta[0];
+  int item_begin = 0, item_end = wl.seg_start[nseg];
+  if (phase == 1) item_end = wl.n1;
+  if (phase == 2) item_begin = wl.n1;
 
   // item -> (type, expert, column block, tile); inside a segment column-block-major, tile-minor
   auto decode = [&](int item) {
     int lo = 0, hi = nseg;  // largest segment whose first item is <= item
     while (hi - lo > 1) {
       const int mid = (lo + hi) / 2;
-      if (s_seg_start[mid] <= item) lo = mid; else hi = mid;
+      if (wl.seg_start[mid] <= item) lo = mid; else hi = mid;
     }
     Item it;
-    it.type = s_seg_info[lo] >> 16;
-    it.e = s_seg_info[lo] & 0xffff;
-    const int m = s_estart[it.e + 1] - s_estart[it.e];
-    const int local = item - s_seg_start[lo];
+    it.type = wl.seg_info[lo] >> 16;
+    it.e = wl.seg_info[lo] & 0xffff;
+    const int m = wl.estart[it.e + 1] - wl.estart[it.e];
+    const int local = item - wl.seg_start[lo];
     it.nb = local / m;
-    it.tile = tile_list[s_estart[it.e] + local % m];
+    it.tile = wl.tiles[wl.estart[it.e] + local % m];
     return it;
   };
   const int first_item = item_begin + blockIdx.x;
@@ -440,16 +360,16 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   const int fused = c.ffn_split == 2 ? 1 : (c.ffn_split == 1 ? 0 : (c.E <= 64 ? 1 : 0));
   const bool pairs = c.ffn_kernel == 2;  // opt-in: the CTA-pair kernel
   const int workers = pairs ? grid / 2 : grid;
-  launch_pdl(worklist_kernel, dim3(1), dim3(256), 0, st, tile_expert, (int)p->P, c.E, NB1, NB2, 2 * workers, fused,
-             pairs ? 2 : 1, p->s.tile_list, p->s.expert_start, p->s.seg_start, p->s.seg_info, p->s.work_meta,
-             p->s.gemm1_done);
+  if (p->P > kMaxListTiles) return MOE_ERR_UNSUPPORTED;  // the work list lives in the kernel's shared memory
+  if (tile_count == nullptr &&  // a call outside moe_layer: the per-tile GEMM1 counters are not reset by a dispatch
+      cudaMemsetAsync(p->s.gemm1_done, 0, sizeof(int) * (size_t)p->P, st) != cudaSuccess)
+    return MOE_ERR_CUDA;
   mark(p, 3, st);
   FfnParams prm;
-  prm.tile_list = p->s.tile_list;
-  prm.expert_start = p->s.expert_start;
-  prm.seg_start = p->s.seg_start;
-  prm.seg_info = p->s.seg_info;
-  prm.meta = p->s.work_meta;
+  prm.tile_expert = tile_expert;
+  prm.P = (int)p->P;
+  prm.lag = 2 * workers;
+  prm.fused = fused;
   prm.E = c.E;
   prm.F = c.F;
   prm.H = c.H;
@@ -471,12 +391,12 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   if (fused) {
     if ((rc = launch(0)) != 0) return rc;
     mark(p, 4, st);  // timed runs: the whole launch is booked on the GEMM1 stage, the GEMM2 stage is empty
-    p->launches += 2;
+    p->launches += 1;
   } else {
     if ((rc = launch(1)) != 0) return rc;
     mark(p, 4, st);
     if ((rc = launch(2)) != 0) return rc;
-    p->launches += 3;
+    p->launches += 2;
   }
   return cudaGetLastError() == cudaSuccess ? 0 : MOE_ERR_CUDA;
 }

@@ -92,9 +92,7 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
   extern __shared__ uint8_t smem_raw[];
   uint8_t* stage_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   Tc2Shared* sh = reinterpret_cast<Tc2Shared*>(stage_base + kStages2 * kStageBytes2);
-  __shared__ int s_estart[kMaxExperts + 1];
-  __shared__ int s_seg_start[2 * kMaxExperts + 1];
-  __shared__ int s_seg_info[2 * kMaxExperts];
+  __shared__ WorkList wl;
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const uint32_t rank = cluster_ctarank();
@@ -119,9 +117,7 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   pdl_wait();  // everything above needs no global data and overlaps the predecessor's tail
-  for (int i = threadIdx.x; i <= E; i += kTcThreads) s_estart[i] = prm.expert_start[i];
-  for (int i = threadIdx.x; i <= nseg; i += kTcThreads) s_seg_start[i] = prm.seg_start[i];
-  for (int i = threadIdx.x; i < nseg; i += kTcThreads) s_seg_info[i] = prm.seg_info[i];
+  build_worklist(wl, prm.tile_expert, prm.P, E, (F + 127) / 128, (H + 255) / 256, prm.lag, prm.fused, 2);
   tc_fence_before();
   __syncthreads();
   cluster_sync_all();  // both CTAs' barriers exist before anything arrives on them
@@ -133,9 +129,9 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
 
   const int NB1 = (F + 127) / 128, NB2 = (H + 255) / 256;
   const int KB1 = (H + kBK - 1) / kBK, KB2 = (F + kBK - 1) / kBK;
-  int item_begin = 0, item_end = s_seg_start[nseg];
-  if (prm.phase == 1) item_end = prm.meta[0];
-  if (prm.phase == 2) item_begin = prm.meta[0];
+  int item_begin = 0, item_end = wl.seg_start[nseg];
+  if (prm.phase == 1) item_end = wl.n1;
+  if (prm.phase == 2) item_begin = wl.n1;
   const int n_clusters = gridDim.x / 2;
   const int first_item = item_begin + blockIdx.x / 2;
 
@@ -145,19 +141,19 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
     int lo = 0, hi = nseg;
     while (hi - lo > 1) {
       const int mid = (lo + hi) / 2;
-      if (s_seg_start[mid] <= item) lo = mid; else hi = mid;
+      if (wl.seg_start[mid] <= item) lo = mid; else hi = mid;
     }
     Item it;
-    it.type = s_seg_info[lo] >> 16;
-    it.e = s_seg_info[lo] & 0xffff;
-    const int m = s_estart[it.e + 1] - s_estart[it.e];  // tiles of the expert
+    it.type = wl.seg_info[lo] >> 16;
+    it.e = wl.seg_info[lo] & 0xffff;
+    const int m = wl.estart[it.e + 1] - wl.estart[it.e];  // tiles of the expert
     const int pairs = (m + 1) / 2;
-    const int local = item - s_seg_start[lo];
+    const int local = item - wl.seg_start[lo];
     it.nb = local / pairs;
     const int j = local % pairs;
-    const int base = s_estart[it.e] + 2 * j;
-    fill = prm.tile_list[base];
-    it.tile = (2 * j + (int)rank < m) ? prm.tile_list[base + rank] : -1;
+    const int base = wl.estart[it.e] + 2 * j;
+    fill = wl.tiles[base];
+    it.tile = (2 * j + (int)rank < m) ? wl.tiles[base + rank] : -1;
     if (it.tile >= 0) fill = it.tile;
     return it;
   };

@@ -112,13 +112,104 @@ struct Item {
   int e, nb, tile;
 };
 
+// The work list, built by every CTA for itself in shared memory from tile_expert[P] (the same
+// deterministic result in every CTA, so no launch and no global round trip is spent on it).
+//   tiles[estart[e] .. estart[e+1])  the used tiles of expert e, in ascending tile order;
+//   the item sequence is at most 2E segments, segment = all GEMM1 items or all GEMM2 items of one
+//   expert: seg_start[i] first item of segment i (seg_start[2E] = number of items), seg_info[i] =
+//   expert | type << 16 (type 0: GEMM1, 1: GEMM2); n1 = items before the first GEMM2 item when the
+//   two GEMMs are separate launches.
+constexpr int kMaxListTiles = 4608;
+struct WorkList {
+  int estart[kMaxExperts + 1];
+  int seg_start[2 * kMaxExperts + 1];
+  int seg_info[2 * kMaxExperts];
+  int cursor[kMaxExperts];
+  int n1;
+  int tiles[kMaxListTiles];
+};
+
+// All threads of the CTA call this (it synchronises the CTA).  pair = 2 counts one item per PAIR of
+// tiles.  fused: the GEMM2 segment of an expert follows once at least `lag` items were placed after its
+// GEMM1 segment; otherwise all GEMM1 segments come first.
+__device__ __forceinline__ void build_worklist(WorkList& wl, const int* __restrict__ tile_expert, int P, int E,
+                                               int NB1, int NB2, int lag, int fused, int pair) {
+  const int tid = threadIdx.x, nthr = blockDim.x, lane = tid % 32;
+  for (int e = tid; e < kMaxExperts; e += nthr) wl.cursor[e] = 0;
+  __syncthreads();
+  for (int p = tid; p < P; p += nthr) {
+    const int e = tile_expert[p];
+    if (e >= 0 && e < E) atomicAdd(&wl.cursor[e], 1);
+  }
+  __syncthreads();
+  if (tid < 32) {  // exclusive scan of the per-expert tile counts: 8 experts per lane
+    int c[kMaxExperts / 32], sum = 0;
+#pragma unroll
+    for (int i = 0; i < kMaxExperts / 32; ++i) {
+      const int e = lane * (kMaxExperts / 32) + i;
+      c[i] = e < E ? wl.cursor[e] : 0;
+      sum += c[i];
+    }
+    int incl = sum;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += n;
+    }
+    int run = incl - sum;
+#pragma unroll
+    for (int i = 0; i < kMaxExperts / 32; ++i) {
+      const int e = lane * (kMaxExperts / 32) + i;
+      if (e < E) {
+        wl.estart[e] = run;
+        wl.cursor[e] = run;
+      }
+      run += c[i];
+    }
+    if (lane == 31) wl.estart[E] = incl;
+    __syncwarp();
+    // stable scatter, 32 tiles at a time: the same list in every CTA
+    for (int p0 = 0; p0 < P; p0 += 32) {
+      const int p = p0 + lane;
+      int e = p < P ? tile_expert[p] : -1;
+      if (e >= E) e = -1;
+      const unsigned peers = __match_any_sync(0xffffffffu, e);
+      if (e >= 0) wl.tiles[wl.cursor[e] + __popc(peers & ((1u << lane) - 1u))] = p;
+      __syncwarp();
+      if (e >= 0 && lane == __ffs(peers) - 1) wl.cursor[e] += __popc(peers);
+      __syncwarp();
+    }
+    if (lane == 0) {
+      int pos = 0, nseg = 0, q = 0;
+      for (int e = 0; e < E; ++e) {
+        const int m = wl.estart[e + 1] - wl.estart[e];
+        wl.seg_start[nseg] = pos;
+        wl.seg_info[nseg++] = e;
+        pos += (m + pair - 1) / pair * NB1;
+        wl.cursor[e] = pos;  // end of this expert's GEMM1 items
+        while (fused && q < e && pos - wl.cursor[q] >= lag) {
+          wl.seg_start[nseg] = pos;
+          wl.seg_info[nseg++] = q | (1 << 16);
+          pos += (wl.estart[q + 1] - wl.estart[q] + pair - 1) / pair * NB2;
+          ++q;
+        }
+      }
+      wl.n1 = fused ? 0 : pos;
+      for (; q < E; ++q) {
+        wl.seg_start[nseg] = pos;
+        wl.seg_info[nseg++] = q | (1 << 16);
+        pos += (wl.estart[q + 1] - wl.estart[q] + pair - 1) / pair * NB2;
+      }
+      wl.seg_start[nseg] = pos;  // nseg == 2E
+    }
+  }
+  __syncthreads();
+}
+
 // Everything the expert-FFN kernels take.
 struct FfnParams {
-  const int* tile_list;
-  const int* expert_start;
-  const int* seg_start;
-  const int* seg_info;
-  const int* meta;
+  const int* tile_expert;  // [P]
+  int P, lag, fused;
   int phase, E, F, H;
   __nv_bfloat16* inter;
   __nv_bfloat16* out;
