@@ -240,7 +240,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             const float gv = __uint_as_float(g[i]);
-            s[i] = gv / (1.0f + __expf(-gv)) * __uint_as_float(u[i]);
+            s[i] = silu_mul(gv, __uint_as_float(u[i]));
           }
           if (c + 8 <= ncols) *reinterpret_cast<uint4*>(dst + c) = Vec16<__nv_bfloat16>::pack(s);
           if (c + 16 <= ncols) *reinterpret_cast<uint4*>(dst + c + 8) = Vec16<__nv_bfloat16>::pack(s + 8);
