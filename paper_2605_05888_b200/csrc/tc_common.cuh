@@ -138,7 +138,8 @@ struct WorkList {
 
 // All threads of the CTA call this (it synchronises the CTA).  pair = 2 counts one item per PAIR of
 // tiles.  fused: the GEMM2 segment of an expert follows once at least `lag` items were placed after its
-// GEMM1 segment; otherwise all GEMM1 segments come first.
+// GEMM1 segment, as long as `lag` GEMM2 items stay in reserve for the end of the list; otherwise all
+// GEMM1 segments come first.
 __device__ __forceinline__ void build_worklist(WorkList& wl, const int* __restrict__ tile_expert, int P, int E,
                                                int NB1, int NB2, int lag, int fused, int pair) {
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid % 32;
@@ -188,17 +189,24 @@ __device__ __forceinline__ void build_worklist(WorkList& wl, const int* __restri
     }
     if (lane == 0) {
       int pos = 0, nseg = 0, q = 0;
+      // GEMM2 items of experts q+1 .. E-2: what would still stand between the last expert's GEMM1 and
+      // its GEMM2 if expert q's GEMM2 segment were placed now.  Keeping `lag` items in that reserve
+      // gives the last experts the same distance as the first ones (without it their GEMM2 items
+      // waited up to half an item for the intermediate).
+      int reserve = 0;
+      for (int j = 1; j + 1 < E; ++j) reserve += (wl.estart[j + 1] - wl.estart[j] + pair - 1) / pair * NB2;
       for (int e = 0; e < E; ++e) {
         const int m = wl.estart[e + 1] - wl.estart[e];
         wl.seg_start[nseg] = pos;
         wl.seg_info[nseg++] = e;
         pos += (m + pair - 1) / pair * NB1;
         wl.cursor[e] = pos;  // end of this expert's GEMM1 items
-        while (fused && q < e && pos - wl.cursor[q] >= lag) {
+        while (fused && q < e && pos - wl.cursor[q] >= lag && reserve >= lag) {
           wl.seg_start[nseg] = pos;
           wl.seg_info[nseg++] = q | (1 << 16);
           pos += (wl.estart[q + 1] - wl.estart[q] + pair - 1) / pair * NB2;
           ++q;
+          if (q + 1 < E) reserve -= (wl.estart[q + 1] - wl.estart[q] + pair - 1) / pair * NB2;
         }
       }
       wl.n1 = fused ? 0 : pos;
