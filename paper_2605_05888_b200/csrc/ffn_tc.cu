@@ -94,12 +94,23 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   if (phase == 2) item_begin = wl.n1;
 
   // item -> (type, expert, column block, tile); inside a segment column-block-major, tile-minor
+  // Shared-memory reads are slow while the tensor pipe streams its operands from the same memory
+  // (a microsecond for the nine dependent reads of a binary search, measured), so only the first
+  // lookup is a search: a thread's items only move forward through the segment list.
+  int seg_cursor = -1;
   auto decode = [&](int item) {
-    int lo = 0, hi = nseg;  // largest segment whose first item is <= item
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) / 2;
-      if (wl.seg_start[mid] <= item) lo = mid; else hi = mid;
+    int lo = seg_cursor;
+    if (lo < 0) {  // largest segment whose first item is <= item
+      int hi = nseg;
+      lo = 0;
+      while (hi - lo > 1) {
+        const int mid = (lo + hi) / 2;
+        if (wl.seg_start[mid] <= item) lo = mid; else hi = mid;
+      }
+    } else {
+      while (wl.seg_start[lo + 1] <= item) ++lo;  // seg_start[nseg] is the item count, above every item
     }
+    seg_cursor = lo;
     Item it;
     it.type = wl.seg_info[lo] >> 16;
     it.e = wl.seg_info[lo] & 0xffff;
@@ -217,6 +228,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   } else {
     // ===================== epilogue =====================
     const int quarter = warp & 3;  // TMEM lanes this warp may read
+    // 32-byte stores need every row start on a 32-byte boundary
+    const bool wide1 = F % 16 == 0 && (reinterpret_cast<uintptr_t>(inter) & 31) == 0;
+    const bool wide2 = H % 16 == 0 && (reinterpret_cast<uintptr_t>(out) & 31) == 0;
     const int row_in_tile = quarter * 32 + lane;
     int local_item = 0;
     for (int item = first_item; item < item_end && !fail_site; item += gridDim.x, ++local_item) {
@@ -242,8 +256,12 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
             const float gv = __uint_as_float(g[i]);
             s[i] = silu_mul(gv, __uint_as_float(u[i]));
           }
-          if (c + 8 <= ncols) *reinterpret_cast<uint4*>(dst + c) = Vec16<__nv_bfloat16>::pack(s);
-          if (c + 16 <= ncols) *reinterpret_cast<uint4*>(dst + c + 8) = Vec16<__nv_bfloat16>::pack(s + 8);
+          if (wide1 && c + 16 <= ncols) {
+            st_global_32B(dst + c, Vec16<__nv_bfloat16>::pack(s), Vec16<__nv_bfloat16>::pack(s + 8));
+          } else {
+            if (c + 8 <= ncols) *reinterpret_cast<uint4*>(dst + c) = Vec16<__nv_bfloat16>::pack(s);
+            if (c + 16 <= ncols) *reinterpret_cast<uint4*>(dst + c + 8) = Vec16<__nv_bfloat16>::pack(s + 8);
+          }
         }
       } else {
         __nv_bfloat16* dst = out + row * H + (size_t)it.nb * 256;
@@ -257,9 +275,14 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
           float f[32];
 #pragma unroll
           for (int i = 0; i < 16; ++i) { f[i] = __uint_as_float(r0[i]); f[16 + i] = __uint_as_float(r1[i]); }
+          if (wide2 && c + 32 <= ncols) {
+            st_global_32B(dst + c, Vec16<__nv_bfloat16>::pack(f), Vec16<__nv_bfloat16>::pack(f + 8));
+            st_global_32B(dst + c + 16, Vec16<__nv_bfloat16>::pack(f + 16), Vec16<__nv_bfloat16>::pack(f + 24));
+          } else {
 #pragma unroll
-          for (int q = 0; q < 4; ++q)
-            if (c + 8 * q + 8 <= ncols) *reinterpret_cast<uint4*>(dst + c + 8 * q) = Vec16<__nv_bfloat16>::pack(f + 8 * q);
+            for (int q = 0; q < 4; ++q)
+              if (c + 8 * q + 8 <= ncols) *reinterpret_cast<uint4*>(dst + c + 8 * q) = Vec16<__nv_bfloat16>::pack(f + 8 * q);
+          }
         }
       }
       tc_fence_before();

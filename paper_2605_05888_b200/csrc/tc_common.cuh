@@ -90,6 +90,13 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t* r) {
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// One 32-byte store (a whole L2 sector) per lane.  The epilogues write a row per lane, so a 16-byte
+// store covers half a sector and the L2 has to merge the halves; whole sectors need no merge.
+__device__ __forceinline__ void st_global_32B(void* p, const uint4& lo, const uint4& hi) {
+  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(lo.x), "r"(lo.y), "r"(lo.z),
+               "r"(lo.w), "r"(hi.x), "r"(hi.y), "r"(hi.z), "r"(hi.w) : "memory");
+}
+
 // silu(g) * u in fp32.  The quotient is the approximate divide (2 ulp, far inside the bf16 rounding that
 // follows): the IEEE divide leaves its fast path for NaN, infinite and very large operands, and the
 // padding rows of a partly filled tile hold whatever the pool held before, so a single such lane
