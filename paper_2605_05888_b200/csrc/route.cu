@@ -5,8 +5,9 @@
 // logit decides which experts are picked and the pick has to be reproducible bit for bit.
 // The parallelism is across the T*E independent chains: x and Wr chunks are staged in shared
 // memory as fp32 (16-byte global loads, next chunk prefetched into registers).  Two shapes:
-// E <= 64 is bound by the latency of the chain itself - one lane per chain; 64 < E <= 256 is
-// bound by fp32 FMA issue - an 8 x 8 register tile of chains per thread.  Afterwards the logits
+// E <= 64 is bound by the latency of the chain itself and by the shared-memory pipe - one token and a
+// few experts per lane; 64 < E <= 256 is bound by fp32 FMA issue - an 8 x 8 register tile of chains
+// per thread.  Afterwards the logits
 // go through shared memory to one warp per token, which keeps them in registers (E/32 per lane)
 // and runs K rounds of a shuffle arg-max (ties: lowest expert index), then the softmax weights.
 #include <float.h>
@@ -118,11 +119,15 @@ route_wide_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const flo
   float* xs = smem;                      // [32][64]
   float* ws = smem + kWideHC * kWideTB;  // [32][256]
   float* ls = smem;                      // [64][256] after the h loop
-  // A warp is an 8 (token groups) x 4 (expert groups) grid of lanes and owns 32 experts for all 64
-  // tokens: per h it reads 256 B of x and 128 B of Wr from shared memory for 2048 FMAs.
+  // A warp is a 2 (token groups) x 16 (expert groups) grid of lanes: 16 tokens x 128 experts; the 8
+  // warps are 4 token quarters x 2 expert halves.  The lane grid is chosen for the shared-memory pipe:
+  // a 16-byte load costs 2 cycles when lanes that share an address are neighbours (lane / 2) or
+  // alternate (lane % 2), and 4 cycles for longer periods (lane % 4, lane % 8) or all-distinct
+  // addresses (measured), so per h a warp spends 8 pipe cycles on its four loads for 64 FMAs.
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int ly = lane / 4, lx = lane % 4;
-  const int ebase = 32 * warp + 4 * lx;  // experts ebase..ebase+3 and ebase+16..ebase+19
+  const int ly = lane % 2, lx = lane / 2;
+  const int tbase = 16 * (warp % 4) + 8 * ly;           // tokens tbase .. tbase+7
+  const int ebase = 128 * (warp / 4) + 4 * lx;          // experts ebase..ebase+3 and ebase+64..ebase+67
   const int t0 = blockIdx.x * kWideTB;
   const int tvalid = min(kWideTB, T - t0);
 
@@ -149,17 +154,17 @@ route_wide_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const flo
     }
     const int hmax = min(kWideHC, H - h0);
     // software pipeline: the operands of step hh+1 are loaded while step hh is computed
-    float4 xa = *reinterpret_cast<const float4*>(xs + 4 * ly);
-    float4 xb = *reinterpret_cast<const float4*>(xs + 32 + 4 * ly);
+    float4 xa = *reinterpret_cast<const float4*>(xs + tbase);
+    float4 xb = *reinterpret_cast<const float4*>(xs + tbase + 4);
     float4 wa = *reinterpret_cast<const float4*>(ws + ebase);
-    float4 wb = *reinterpret_cast<const float4*>(ws + ebase + 16);
+    float4 wb = *reinterpret_cast<const float4*>(ws + ebase + 64);
 #pragma unroll 2
     for (int hh = 0; hh < hmax; ++hh) {
       const int hn = min(hh + 1, kWideHC - 1);
-      const float4 nxa = *reinterpret_cast<const float4*>(xs + hn * kWideTB + 4 * ly);
-      const float4 nxb = *reinterpret_cast<const float4*>(xs + hn * kWideTB + 32 + 4 * ly);
+      const float4 nxa = *reinterpret_cast<const float4*>(xs + hn * kWideTB + tbase);
+      const float4 nxb = *reinterpret_cast<const float4*>(xs + hn * kWideTB + tbase + 4);
       const float4 nwa = *reinterpret_cast<const float4*>(ws + hn * kWideEP + ebase);
-      const float4 nwb = *reinterpret_cast<const float4*>(ws + hn * kWideEP + ebase + 16);
+      const float4 nwb = *reinterpret_cast<const float4*>(ws + hn * kWideEP + ebase + 64);
       const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
       const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
 #pragma unroll
@@ -172,10 +177,10 @@ route_wide_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const flo
   __syncthreads();
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    const int tl = (j < 4) ? 4 * ly + j : 32 + 4 * ly + (j - 4);
+    const int tl = tbase + j;
 #pragma unroll
     for (int g = 0; g < 2; ++g) {
-      const int e0 = ebase + 16 * g;
+      const int e0 = ebase + 64 * g;
       float l[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
@@ -206,140 +211,197 @@ static int launch_wide(moe_plan* p, const void* x, const void* wr, const float* 
                          (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w);
 }
 
-// The latency-bound shapes (E <= 64): one lane per chain (or two chains for 32 < E <= 64).  A token's
-// experts sit on LE consecutive lanes; x and Wr tiles stay in their natural [row][h] layout in shared
-// memory (fp32, converted while staging), so a lane reads four consecutive h of its token and of its
-// expert with two 16-byte loads and runs its chain over them.  The time is close to the latency of
-// the chain itself (4 cycles per h) once the chunk loads are overlapped.
-template <typename XT, int ROWS, int HC, int THREADS>
+// The latency-bound shapes (E <= 64).  x and Wr tiles stay in their natural [row][h] layout in shared
+// memory (fp32, converted while staging); a lane owns one token and two experts, reads four consecutive h
+// of its token and of each expert with 16-byte loads and runs its two chains over them.  What bounds the
+// kernel is the shared-memory pipe, not the chains (measured on this part): a 16-byte load costs the SM
+// 2 pipe cycles when the lanes that share an address are neighbours (lane / 2) or alternate (lane % 2)
+// and 4 cycles otherwise, and a warp that has the SM to itself still waits about 8 cycles per load.  So a
+// warp is 16 tokens x 2 expert groups (SWAP = false: token by lane / 2, group by lane % 2; 4 experts per
+// warp) or 2 tokens x 16 groups (SWAP = true: 32 experts per warp, for many experts), every load a 2-cycle
+// one, three loads per 8 FMAs, and enough warps per SM to keep the pipe busy.
+//
+// The compute warps only run chains.  Four more warps stage: while the compute warps work on one
+// shared-memory buffer, the staging warps convert the next chunk (already in their registers) into the
+// other buffer and fetch from global memory the chunks after it, so neither the global-memory latency nor
+// the conversion sits on the chains' critical path.  One __syncthreads per chunk.
+constexpr int kNarrowFillWarps = 4;
+
+// Four elements per staging load (16 bytes of fp32, 8 bytes of bf16): every thread then writes one 16-byte
+// vector and consecutive lanes write consecutive vectors, which is free of bank conflicts (eight bf16
+// per thread made two vectors 32 bytes apart per lane: a two-way conflict on every store).
+template <typename XT> struct Stage4;
+template <> struct Stage4<float> {
+  typedef uint4 V;
+  static __device__ __forceinline__ V zero() { return make_uint4(0, 0, 0, 0); }
+  static __device__ __forceinline__ V ld(const float* p) { return __ldg(reinterpret_cast<const uint4*>(p)); }
+  static __device__ __forceinline__ float4 cvt(const V& v) {
+    return make_float4(__uint_as_float(v.x), __uint_as_float(v.y), __uint_as_float(v.z), __uint_as_float(v.w));
+  }
+};
+template <> struct Stage4<__nv_bfloat16> {
+  typedef uint2 V;
+  static __device__ __forceinline__ V zero() { return make_uint2(0, 0); }
+  static __device__ __forceinline__ V ld(const __nv_bfloat16* p) { return __ldg(reinterpret_cast<const uint2*>(p)); }
+  static __device__ __forceinline__ float4 cvt(const V& v) {  // bf16 -> fp32 is a 16-bit shift
+    return make_float4(__uint_as_float(v.x << 16), __uint_as_float(v.x & 0xffff0000u), __uint_as_float(v.y << 16),
+                       __uint_as_float(v.y & 0xffff0000u));
+  }
+};
+
+template <typename XT, int ROWS, int HC>
 struct NaturalChunk {
-  static constexpr int N = Vec16<XT>::N;
+  static constexpr int FT = 32 * kNarrowFillWarps;  // staging threads
+  static constexpr int N = 4;
   static constexpr int PARTS = HC / N;
   static constexpr int NVEC = ROWS * PARTS;
-  static constexpr int PER_THREAD = (NVEC + THREADS - 1) / THREADS;
+  static constexpr int PER_THREAD = (NVEC + FT - 1) / FT;
   static constexpr int PITCH = HC + 4;  // floats; rows land on different banks
-  uint4 v[PER_THREAD];
-  __device__ __forceinline__ void load(const XT* base, int row0, int nrows_valid, int H, int h0) {
+  typename Stage4<XT>::V v[PER_THREAD];
+  // ft: index of the calling thread among the staging threads
+  __device__ __forceinline__ void load(int ft, const XT* base, int row0, int nrows_valid, int H, int h0) {
 #pragma unroll
     for (int i = 0; i < PER_THREAD; ++i) {
-      const int idx = threadIdx.x + i * THREADS;
+      const int idx = ft + i * FT;
       const int r = idx / PARTS, part = idx % PARTS;
       const int h = h0 + part * N;
-      v[i] = make_uint4(0, 0, 0, 0);
-      if (idx < NVEC && r < nrows_valid && h < H)
-        v[i] = __ldg(reinterpret_cast<const uint4*>(base + (size_t)(row0 + r) * H + h));
+      v[i] = Stage4<XT>::zero();
+      if (idx < NVEC && r < nrows_valid && h < H) v[i] = Stage4<XT>::ld(base + (size_t)(row0 + r) * H + h);
     }
   }
-  __device__ __forceinline__ void store(float* s) const {  // s: [ROWS][PITCH]
+  __device__ __forceinline__ void store(int ft, float* s) const {  // s: [ROWS][PITCH]
 #pragma unroll
     for (int i = 0; i < PER_THREAD; ++i) {
-      const int idx = threadIdx.x + i * THREADS;
+      const int idx = ft + i * FT;
       if (idx < NVEC) {
         const int r = idx / PARTS, part = idx % PARTS;
-        float f[N];
-        Vec16<XT>::unpack(v[i], f);
-        float4* dst = reinterpret_cast<float4*>(s + r * PITCH + part * N);
-#pragma unroll
-        for (int q = 0; q < N / 4; ++q) dst[q] = make_float4(f[4 * q], f[4 * q + 1], f[4 * q + 2], f[4 * q + 3]);
+        *reinterpret_cast<float4*>(s + r * PITCH + part * N) = Stage4<XT>::cvt(v[i]);
       }
     }
   }
 };
 
-template <typename XT, int LE, int TE, int HC, int THREADS>
-__global__ void __launch_bounds__(THREADS)
+// EW warps side by side cover the experts, TWP warps the tokens of the block.
+template <typename XT, bool SWAP, int EW, int TWP, int HC>
+__global__ void __launch_bounds__(32 * (EW * TWP + kNarrowFillWarps))
 route_narrow_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias, int T,
                     int H, int E, int K, int renorm, int* __restrict__ topk_idx, float* __restrict__ topk_w) {
-  constexpr int EP = LE * TE;              // experts covered (padded)
-  constexpr int TW = 32 / LE;              // tokens per warp
-  constexpr int TB = TW * (THREADS / 32);
+  constexpr int TN = 2;                    // experts per lane
+  constexpr int G = SWAP ? 16 : 2;         // expert groups per warp
+  constexpr int TW = 32 / G;               // tokens per warp
+  constexpr int EPW = G * TN;              // experts per warp
+  constexpr int EP = EW * EPW;             // experts covered (padded)
+  constexpr int TB = TW * TWP;             // tokens per block
+  constexpr int CW = EW * TWP;             // compute warps
   constexpr int PITCH = HC + 4;
+  constexpr int BUF = (TB + EP) * PITCH;   // floats per buffer: x tile [TB][PITCH], then Wr tile [EP][PITCH]
   extern __shared__ __align__(16) float smem[];
-  float* xs = smem;               // [TB][PITCH]
-  float* ws = smem + TB * PITCH;  // [EP][PITCH]
-  float* ls = smem;               // [TB][EP] after the h loop
+  float* ls = smem;                        // [TB][EP] after the h loop
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int tl = warp * TW + lane / LE;  // this lane's token inside the block
-  const int le = lane % LE;              // this lane's experts: le + LE*i
+  const bool computes = warp < CW;
+  const int ft = threadIdx.x - 32 * CW;
+  const int tl = (computes ? warp / EW : 0) * TW + (SWAP ? lane % 2 : lane / 2);   // this lane's token inside the block
+  const int le = (computes ? warp % EW : 0) * EPW + (SWAP ? lane / 2 : lane % 2);  // this lane's experts: le + G*i
   const int t0 = blockIdx.x * TB;
   const int tvalid = min(TB, T - t0);
+  const int nchunks = (H + HC - 1) / HC;
 
-  float acc[TE];
+  float acc[TN];
 #pragma unroll
-  for (int i = 0; i < TE; ++i) acc[i] = 0.0f;
-  NaturalChunk<XT, TB, HC, THREADS> xr;
-  NaturalChunk<XT, EP, HC, THREADS> wrg;
+  for (int i = 0; i < TN; ++i) acc[i] = 0.0f;
+  // The staging warps keep P chunks in flight in registers, so that global memory is not waited for.
+  constexpr int P = 2;
+  NaturalChunk<XT, TB, HC> xr[P];
+  NaturalChunk<XT, EP, HC> wrg[P];
   pdl_wait();
   pdl_trigger();
-  xr.load(x, t0, tvalid, H, 0);
-  wrg.load(wr, 0, E, H, 0);
-  for (int h0 = 0; h0 < H; h0 += HC) {
-    __syncthreads();
-    xr.store(xs);
-    wrg.store(ws);
-    __syncthreads();
-    if (h0 + HC < H) {
-      xr.load(x, t0, tvalid, H, h0 + HC);
-      wrg.load(wr, 0, E, H, h0 + HC);
+  if (!computes) {  // chunk 0 into buffer 0, chunks 1..P into the registers (slot = chunk % P)
+    xr[0].load(ft, x, t0, tvalid, H, 0);
+    wrg[0].load(ft, wr, 0, E, H, 0);
+    xr[0].store(ft, smem);
+    wrg[0].store(ft, smem + TB * PITCH);
+#pragma unroll
+    for (int j = 1; j <= P; ++j) {  // past H: zero-filled, never stored
+      xr[j % P].load(ft, x, t0, tvalid, H, j * HC);
+      wrg[j % P].load(ft, wr, 0, E, H, j * HC);
     }
-    const int hmax = min(HC, H - h0);
-    // Groups of 16 h: the next group's operands are loaded while this group's 16-step chain runs, so
-    // the shared-memory latency hides behind the chain.  The tail of a short last chunk is zero in
-    // shared memory (loads past H are zero-filled) and fma(0, 0, acc) leaves acc's value alone.
-    const float* xrow = xs + tl * PITCH;
-    const float* wrow = ws + le * PITCH;
-    constexpr int G = 4;
-    float4 xv[G], wv[TE][G];
+  }
+  for (int c0 = 0; c0 < nchunks; c0 += P) {
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-      xv[g] = *reinterpret_cast<const float4*>(xrow + 4 * g);
-#pragma unroll
-      for (int i = 0; i < TE; ++i) wv[i][g] = *reinterpret_cast<const float4*>(wrow + LE * i * PITCH + 4 * g);
-    }
-    for (int hh = 0; hh < hmax; hh += 4 * G) {
-      const int hn = min(hh + 4 * G, HC - 4 * G);
-      float4 nxv[G], nwv[TE][G];
-#pragma unroll
-      for (int g = 0; g < G; ++g) {
-        nxv[g] = *reinterpret_cast<const float4*>(xrow + hn + 4 * g);
-#pragma unroll
-        for (int i = 0; i < TE; ++i) nwv[i][g] = *reinterpret_cast<const float4*>(wrow + LE * i * PITCH + hn + 4 * g);
-      }
-#pragma unroll
-      for (int g = 0; g < G; ++g)
-#pragma unroll
-        for (int i = 0; i < TE; ++i) {
-          acc[i] = __fmaf_rn(xv[g].x, wv[i][g].x, acc[i]);
-          acc[i] = __fmaf_rn(xv[g].y, wv[i][g].y, acc[i]);
-          acc[i] = __fmaf_rn(xv[g].z, wv[i][g].z, acc[i]);
-          acc[i] = __fmaf_rn(xv[g].w, wv[i][g].w, acc[i]);
+    for (int p = 0; p < P; ++p) {
+      const int c = c0 + p;  // every thread runs the same number of barriers; chunks past the end do nothing
+      __syncthreads();       // buffer c&1 holds chunk c; buffer (c+1)&1 is no longer read
+      float* cur = smem + (c & 1) * BUF;
+      if (!computes) {
+        if (c + 1 < nchunks) {
+          float* nxt = smem + ((c + 1) & 1) * BUF;
+          xr[(p + 1) % P].store(ft, nxt);
+          wrg[(p + 1) % P].store(ft, nxt + TB * PITCH);
+          xr[(p + 1) % P].load(ft, x, t0, tvalid, H, (c + 1 + P) * HC);
+          wrg[(p + 1) % P].load(ft, wr, 0, E, H, (c + 1 + P) * HC);
         }
+        continue;
+      }
+      if (c >= nchunks) continue;
+      const float* xrow = cur + tl * PITCH;
+      const float* wrow = cur + TB * PITCH + le * PITCH;
+      // Four h at a time, the operands D steps ahead in flight.  The tail of a short last chunk is zero
+      // in shared memory (loads past H are zero-filled) and fma(0, 0, acc) leaves acc alone.
+      constexpr int D = 2;
+      float4 xv[D], wv[D][TN];
 #pragma unroll
-      for (int g = 0; g < G; ++g) {
-        xv[g] = nxv[g];
+      for (int d = 0; d < D; ++d) {
+        xv[d] = *reinterpret_cast<const float4*>(xrow + 4 * d);
 #pragma unroll
-        for (int i = 0; i < TE; ++i) wv[i][g] = nwv[i][g];
+        for (int i = 0; i < TN; ++i) wv[d][i] = *reinterpret_cast<const float4*>(wrow + G * i * PITCH + 4 * d);
+      }
+#pragma unroll 4
+      for (int hh = 0; hh < HC; hh += 4) {
+        const int hn = hh + 4 * D < HC ? hh + 4 * D : HC - 4;
+        const float4 nxv = *reinterpret_cast<const float4*>(xrow + hn);
+        float4 nwv[TN];
+#pragma unroll
+        for (int i = 0; i < TN; ++i) nwv[i] = *reinterpret_cast<const float4*>(wrow + G * i * PITCH + hn);
+#pragma unroll
+        for (int i = 0; i < TN; ++i) acc[i] = __fmaf_rn(xv[0].x, wv[0][i].x, acc[i]);
+#pragma unroll
+        for (int i = 0; i < TN; ++i) acc[i] = __fmaf_rn(xv[0].y, wv[0][i].y, acc[i]);
+#pragma unroll
+        for (int i = 0; i < TN; ++i) acc[i] = __fmaf_rn(xv[0].z, wv[0][i].z, acc[i]);
+#pragma unroll
+        for (int i = 0; i < TN; ++i) acc[i] = __fmaf_rn(xv[0].w, wv[0][i].w, acc[i]);
+#pragma unroll
+        for (int d = 0; d + 1 < D; ++d) {
+          xv[d] = xv[d + 1];
+#pragma unroll
+          for (int i = 0; i < TN; ++i) wv[d][i] = wv[d + 1][i];
+        }
+        xv[D - 1] = nxv;
+#pragma unroll
+        for (int i = 0; i < TN; ++i) wv[D - 1][i] = nwv[i];
       }
     }
   }
   __syncthreads();
+  if (computes) {
 #pragma unroll
-  for (int i = 0; i < TE; ++i) {
-    const int e = le + LE * i;
-    float l = acc[i];
-    if (bias != nullptr && e < E) l = l + bias[e];
-    ls[tl * EP + e] = l;
+    for (int i = 0; i < TN; ++i) {
+      const int e = le + G * i;
+      float l = acc[i];
+      if (bias != nullptr && e < E) l = l + bias[e];
+      ls[tl * EP + e] = l;
+    }
   }
   __syncthreads();
   select_topk<EP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w);
 }
 
-template <typename XT, int LE, int TE, int HC, int THREADS>
+template <typename XT, bool SWAP, int EW, int TWP, int HC>
 static int launch_narrow(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
                          float* topk_w, cudaStream_t st) {
-  constexpr int EP = LE * TE, TB = (32 / LE) * (THREADS / 32);
-  const size_t smem = sizeof(float) * (TB + EP) * (HC + 4);
-  auto kern = route_narrow_kernel<XT, LE, TE, HC, THREADS>;
+  constexpr int G = SWAP ? 16 : 2, EP = EW * G * 2, TB = (32 / G) * TWP;
+  constexpr size_t smem = sizeof(float) * (2 * (TB + EP) * (HC + 4) > TB * EP ? 2 * (TB + EP) * (HC + 4) : TB * EP);
+  auto kern = route_narrow_kernel<XT, SWAP, EW, TWP, HC>;
   static bool attr_done = false;  // per instantiation and process, idempotent
   if (smem > 48 * 1024 && !attr_done) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -348,29 +410,21 @@ static int launch_narrow(moe_plan* p, const void* x, const void* wr, const float
   }
   const moe_config_t& c = p->cfg;
   p->launches += 1;
-  return (int)launch_maybe_pdl(false, kern, dim3((c.T + TB - 1) / TB), dim3(THREADS), smem, st, (const XT*)x,
-                         (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w);
+  return (int)launch_maybe_pdl(false, kern, dim3((c.T + TB - 1) / TB), dim3(32 * (EW * TWP + kNarrowFillWarps)), smem, st,
+                               (const XT*)x, (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w);
 }
 
 template <typename XT>
 static int launch_typed(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
                         float* topk_w, cudaStream_t st) {
   const moe_config_t& c = p->cfg;
-  // Small E is bound by the latency of the chain: one lane per chain, long chunks; small batches use
-  // 128-thread CTAs so that the blocks spread over more SMs.
-  const bool small = c.T <= 2048;
-  if (c.E <= 8)
-    return small ? launch_narrow<XT, 8, 1, 512, 128>(p, x, wr, bias, topk_idx, topk_w, st)
-                 : launch_narrow<XT, 8, 1, 512, 256>(p, x, wr, bias, topk_idx, topk_w, st);
-  if (c.E <= 16)
-    return small ? launch_narrow<XT, 16, 1, 512, 128>(p, x, wr, bias, topk_idx, topk_w, st)
-                 : launch_narrow<XT, 16, 1, 512, 256>(p, x, wr, bias, topk_idx, topk_w, st);
-  if (c.E <= 32)
-    return small ? launch_narrow<XT, 32, 1, 512, 128>(p, x, wr, bias, topk_idx, topk_w, st)
-                 : launch_narrow<XT, 32, 1, 512, 256>(p, x, wr, bias, topk_idx, topk_w, st);
-  if (c.E <= 64)
-    return small ? launch_narrow<XT, 32, 2, 256, 128>(p, x, wr, bias, topk_idx, topk_w, st)
-                 : launch_narrow<XT, 32, 2, 256, 256>(p, x, wr, bias, topk_idx, topk_w, st);
+  // 16 tokens x 2 expert groups per warp, two compute warps per CTA (32 tokens: T = 4096 gives 128
+  // CTAs); with many experts 2 tokens x 16 groups, so that the chains still spread over the SMs.
+  constexpr int HL = sizeof(XT) == 2 ? 256 : 128;  // h per chunk
+  if (c.E <= 8) return launch_narrow<XT, false, 2, 2, HL>(p, x, wr, bias, topk_idx, topk_w, st);   // 32 tokens per CTA
+  if (c.E <= 16) return launch_narrow<XT, false, 4, 2, HL>(p, x, wr, bias, topk_idx, topk_w, st);  // 32 tokens per CTA
+  if (c.E <= 32) return launch_narrow<XT, true, 1, 4, HL / 2>(p, x, wr, bias, topk_idx, topk_w, st);  // 8 tokens per CTA
+  if (c.E <= 64) return launch_narrow<XT, true, 2, 2, HL / 2>(p, x, wr, bias, topk_idx, topk_w, st);  // 4 tokens per CTA
   return launch_wide<XT>(p, x, wr, bias, topk_idx, topk_w, st);
 }
 
