@@ -5,9 +5,9 @@
 // logit decides which experts are picked and the pick has to be reproducible bit for bit.
 // The parallelism is across the T*E independent chains: x and Wr chunks are staged in shared
 // memory as fp32 (16-byte global loads, next chunk prefetched into registers).  Two shapes:
-// E <= 64 is bound by the latency of the chain itself and by the shared-memory pipe - one token and a
-// few experts per lane; 64 < E <= 256 is bound by fp32 FMA issue - an 8 x 8 register tile of chains
-// per thread.  Afterwards the logits
+// E <= 64 is bound by the shared-memory pipe - one token and two experts per lane; 64 < E <= 256 is
+// bound by fp32 FMA issue - a register tile of up to 8 x 16 chains per thread.  In both, some warps only
+// stage the operands and the others only compute.  Afterwards the logits
 // go through shared memory to one warp per token, which keeps them in registers (E/32 per lane)
 // and runs K rounds of a shuffle arg-max (ties: lowest expert index), then the softmax weights.
 #include <float.h>
@@ -16,7 +16,6 @@
 
 namespace moehub {
 
-constexpr int kRouteThreads = 256;
 
 // One warp per token: the token's logits sit in registers (EP/32 per lane); K rounds of a shuffle
 // arg-max on (value, lowest index); then the softmax weights of the picks.  ls: [tokens][EP] logits
@@ -76,32 +75,43 @@ __device__ __forceinline__ void select_topk(const float* ls, int tvalid, int t0,
   }
 }
 
-// The compute-bound shape (64 < E <= 256): 64 tokens x 256 experts per CTA, 8 x 8 chains per thread,
-// every shared-memory read of the inner loop a 16-byte vector: 4 loads feed 64 FMAs.  The staging
-// stores are conflict-free because consecutive lanes handle consecutive rows of one 16-byte column
-// group.
-constexpr int kWideTB = 64, kWideEP = 256, kWideHC = 32;
+// The compute-bound shape (64 < E <= 256): up to 64 tokens x 256 experts per CTA.  Four compute warps
+// hold a TMT x 16 register tile of chains per thread (a warp: 2 token groups by lane % 2, 16 expert
+// groups by lane / 2, so that each of its six 16-byte shared-memory loads per h costs the 2-cycle
+// minimum) and do nothing but FMAs; four staging warps convert the next chunk of x and Wr into the other
+// shared-memory buffer (transposed to [h][token] and [h][expert], fp32) and keep the chunks after it in
+// flight from global memory.  One __syncthreads per chunk of 32 h.  TMT (tokens per thread, 4..8) is
+// picked at launch so that the CTAs fill the SMs evenly: T = 8192 runs 147 CTAs of 56 tokens.
+constexpr int kWideEP = 256, kWideHC = 32, kWideSlots = 64;
+constexpr int kWideComputeWarps = 4, kWideFillWarps = 4;
+constexpr int kWideThreads = 32 * (kWideComputeWarps + kWideFillWarps);
+constexpr int kWideBuf = kWideHC * (kWideSlots + kWideEP);  // floats per buffer
 
+// ROWS rows of the tile (x: token slots, Wr: experts) times kWideHC h, 16 bytes per staging load.
 template <typename XT, int ROWS>
 struct WideChunk {
+  static constexpr int FT = 32 * kWideFillWarps;
   static constexpr int N = Vec16<XT>::N;
   static constexpr int PARTS = kWideHC / N;
-  static constexpr int PER_THREAD = ROWS * PARTS / kRouteThreads;
+  static constexpr int PER_THREAD = ROWS * PARTS / FT;
   uint4 v[PER_THREAD];
-  __device__ __forceinline__ void load(const XT* base, int row0, int nrows_valid, int H, int h0) {
+  // row_of(r): global row of tile row r, or -1 for a padding row
+  template <typename RowOf>
+  __device__ __forceinline__ void load(int ft, const XT* base, RowOf row_of, int H, int h0) {
 #pragma unroll
     for (int i = 0; i < PER_THREAD; ++i) {
-      const int idx = threadIdx.x + i * kRouteThreads;
+      const int idx = ft + i * FT;
       const int r = idx % ROWS, part = idx / ROWS;
       const int h = h0 + part * N;
+      const int row = row_of(r);
       v[i] = make_uint4(0, 0, 0, 0);
-      if (r < nrows_valid && h < H) v[i] = __ldg(reinterpret_cast<const uint4*>(base + (size_t)(row0 + r) * H + h));
+      if (row >= 0 && h < H) v[i] = __ldg(reinterpret_cast<const uint4*>(base + (size_t)row * H + h));
     }
   }
-  __device__ __forceinline__ void store(float* s) const {  // s: [kWideHC][ROWS]
+  __device__ __forceinline__ void store(int ft, float* s) const {  // s: [kWideHC][ROWS]
 #pragma unroll
     for (int i = 0; i < PER_THREAD; ++i) {
-      const int idx = threadIdx.x + i * kRouteThreads;
+      const int idx = ft + i * FT;
       const int r = idx % ROWS, part = idx / ROWS;
       float f[N];
       Vec16<XT>::unpack(v[i], f);
@@ -111,94 +121,128 @@ struct WideChunk {
   }
 };
 
-template <typename XT>
-__global__ void __launch_bounds__(kRouteThreads)
+template <typename XT, int TMT>
+__global__ void __launch_bounds__(kWideThreads)
 route_wide_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias, int T,
                   int H, int E, int K, int renorm, int* __restrict__ topk_idx, float* __restrict__ topk_w) {
+  constexpr int TB = 8 * TMT;  // tokens per CTA: 4 warps x 2 lane groups x TMT
   extern __shared__ __align__(16) float smem[];
-  float* xs = smem;                      // [32][64]
-  float* ws = smem + kWideHC * kWideTB;  // [32][256]
-  float* ls = smem;                      // [64][256] after the h loop
-  // A warp is a 2 (token groups) x 16 (expert groups) grid of lanes: 16 tokens x 128 experts; the 8
-  // warps are 4 token quarters x 2 expert halves.  The lane grid is chosen for the shared-memory pipe:
-  // a 16-byte load costs 2 cycles when lanes that share an address are neighbours (lane / 2) or
-  // alternate (lane % 2), and 4 cycles for longer periods (lane % 4, lane % 8) or all-distinct
-  // addresses (measured), so per h a warp spends 8 pipe cycles on its four loads for 64 FMAs.
+  float* ls = smem;  // [TB][256] after the h loop
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-  const int ly = lane % 2, lx = lane / 2;
-  const int tbase = 16 * (warp % 4) + 8 * ly;           // tokens tbase .. tbase+7
-  const int ebase = 128 * (warp / 4) + 4 * lx;          // experts ebase..ebase+3 and ebase+64..ebase+67
-  const int t0 = blockIdx.x * kWideTB;
-  const int tvalid = min(kWideTB, T - t0);
+  const bool computes = warp < kWideComputeWarps;
+  const int ft = threadIdx.x - 32 * kWideComputeWarps;
+  const int grp = 2 * (computes ? warp : 0) + lane % 2;  // this thread's token group: tokens grp*TMT .. +TMT-1
+  const int ebase = 4 * (lane / 2);                       // experts ebase + 64*i + q, i < 4, q < 4
+  const int t0 = blockIdx.x * TB;
+  const int tvalid = min(TB, T - t0);
+  const int nchunks = (H + kWideHC - 1) / kWideHC;
+  // The x tile has 8 slots per token group (16-byte aligned for any TMT); slots past TMT stay zero.
+  auto x_row = [&](int slot) {
+    const int tl = (slot / 8) * TMT + slot % 8;
+    return (slot % 8 < TMT && tl < tvalid) ? t0 + tl : -1;
+  };
+  auto w_row = [&](int e) { return e < E ? e : -1; };
 
-  float acc[8][8];
+  float acc[TMT][16];
 #pragma unroll
-  for (int j = 0; j < 8; ++j)
+  for (int j = 0; j < TMT; ++j)
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc[j][i] = 0.0f;
+    for (int i = 0; i < 16; ++i) acc[j][i] = 0.0f;
 
-  WideChunk<XT, kWideTB> xr;
-  WideChunk<XT, kWideEP> wrg;
+  constexpr int P = sizeof(XT) == 2 ? 2 : 1;  // chunks kept in flight in the staging warps' registers
+  WideChunk<XT, kWideSlots> xr[P];
+  WideChunk<XT, kWideEP> wrg[P];
   pdl_wait();
   pdl_trigger();
-  xr.load(x, t0, tvalid, H, 0);
-  wrg.load(wr, 0, E, H, 0);
-  for (int h0 = 0; h0 < H; h0 += kWideHC) {
-    __syncthreads();
-    xr.store(xs);
-    wrg.store(ws);
-    __syncthreads();
-    if (h0 + kWideHC < H) {
-      xr.load(x, t0, tvalid, H, h0 + kWideHC);
-      wrg.load(wr, 0, E, H, h0 + kWideHC);
+  if (!computes) {  // chunk 0 into buffer 0, chunks 1..P into the registers (slot = chunk % P)
+    xr[0].load(ft, x, x_row, H, 0);
+    wrg[0].load(ft, wr, w_row, H, 0);
+    xr[0].store(ft, smem);
+    wrg[0].store(ft, smem + kWideHC * kWideSlots);
+#pragma unroll
+    for (int j = 1; j <= P; ++j) {  // past H: zero-filled, never stored
+      xr[j % P].load(ft, x, x_row, H, j * kWideHC);
+      wrg[j % P].load(ft, wr, w_row, H, j * kWideHC);
     }
-    const int hmax = min(kWideHC, H - h0);
-    // software pipeline: the operands of step hh+1 are loaded while step hh is computed
-    float4 xa = *reinterpret_cast<const float4*>(xs + tbase);
-    float4 xb = *reinterpret_cast<const float4*>(xs + tbase + 4);
-    float4 wa = *reinterpret_cast<const float4*>(ws + ebase);
-    float4 wb = *reinterpret_cast<const float4*>(ws + ebase + 64);
+  }
+  for (int c0 = 0; c0 < nchunks; c0 += P) {
+#pragma unroll
+    for (int p = 0; p < P; ++p) {
+      const int c = c0 + p;  // every thread runs the same number of barriers; chunks past the end do nothing
+      __syncthreads();       // buffer c&1 holds chunk c; buffer (c+1)&1 is no longer read
+      if (!computes) {
+        if (c + 1 < nchunks) {
+          float* nxt = smem + ((c + 1) & 1) * kWideBuf;
+          xr[(p + 1) % P].store(ft, nxt);
+          wrg[(p + 1) % P].store(ft, nxt + kWideHC * kWideSlots);
+          xr[(p + 1) % P].load(ft, x, x_row, H, (c + 1 + P) * kWideHC);
+          wrg[(p + 1) % P].load(ft, wr, w_row, H, (c + 1 + P) * kWideHC);
+        }
+        continue;
+      }
+      if (c >= nchunks) continue;
+      const float* xs = smem + (c & 1) * kWideBuf + 8 * grp;              // [h][slot]
+      const float* ws = smem + (c & 1) * kWideBuf + kWideHC * kWideSlots + ebase;  // [h][expert]
+      // software pipeline: the operands of step hh+1 are loaded while step hh is computed.  The tail of
+      // a short last chunk is zero in shared memory and fma(0, 0, acc) leaves acc alone.
+      float4 xa = *reinterpret_cast<const float4*>(xs);
+      float4 xb = *reinterpret_cast<const float4*>(xs + 4);
+      float4 wv[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) wv[i] = *reinterpret_cast<const float4*>(ws + 64 * i);
 #pragma unroll 2
-    for (int hh = 0; hh < hmax; ++hh) {
-      const int hn = min(hh + 1, kWideHC - 1);
-      const float4 nxa = *reinterpret_cast<const float4*>(xs + hn * kWideTB + tbase);
-      const float4 nxb = *reinterpret_cast<const float4*>(xs + hn * kWideTB + tbase + 4);
-      const float4 nwa = *reinterpret_cast<const float4*>(ws + hn * kWideEP + ebase);
-      const float4 nwb = *reinterpret_cast<const float4*>(ws + hn * kWideEP + ebase + 64);
-      const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
-      const float wv[8] = {wa.x, wa.y, wa.z, wa.w, wb.x, wb.y, wb.z, wb.w};
+      for (int hh = 0; hh < kWideHC; ++hh) {
+        const int hn = hh + 1 < kWideHC ? hh + 1 : hh;
+        const float4 nxa = *reinterpret_cast<const float4*>(xs + hn * kWideSlots);
+        const float4 nxb = *reinterpret_cast<const float4*>(xs + hn * kWideSlots + 4);
+        float4 nwv[4];
 #pragma unroll
-      for (int j = 0; j < 8; ++j)
+        for (int i = 0; i < 4; ++i) nwv[i] = *reinterpret_cast<const float4*>(ws + hn * kWideEP + 64 * i);
+        const float xv[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
 #pragma unroll
-        for (int i = 0; i < 8; ++i) acc[j][i] = __fmaf_rn(xv[j], wv[i], acc[j][i]);
-      xa = nxa; xb = nxb; wa = nwa; wb = nwb;
+        for (int j = 0; j < TMT; ++j)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            acc[j][4 * i + 0] = __fmaf_rn(xv[j], wv[i].x, acc[j][4 * i + 0]);
+            acc[j][4 * i + 1] = __fmaf_rn(xv[j], wv[i].y, acc[j][4 * i + 1]);
+            acc[j][4 * i + 2] = __fmaf_rn(xv[j], wv[i].z, acc[j][4 * i + 2]);
+            acc[j][4 * i + 3] = __fmaf_rn(xv[j], wv[i].w, acc[j][4 * i + 3]);
+          }
+        xa = nxa;
+        xb = nxb;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) wv[i] = nwv[i];
+      }
     }
   }
   __syncthreads();
+  if (computes) {
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    const int tl = tbase + j;
-#pragma unroll
-    for (int g = 0; g < 2; ++g) {
-      const int e0 = ebase + 64 * g;
-      float l[4];
+    for (int j = 0; j < TMT; ++j) {
+      const int tl = grp * TMT + j;
 #pragma unroll
       for (int i = 0; i < 4; ++i) {
-        l[i] = acc[j][g * 4 + i];
-        if (bias != nullptr && e0 + i < E) l[i] = l[i] + bias[e0 + i];
+        const int e0 = ebase + 64 * i;
+        float l[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          l[q] = acc[j][4 * i + q];
+          if (bias != nullptr && e0 + q < E) l[q] = l[q] + bias[e0 + q];
+        }
+        *reinterpret_cast<float4*>(ls + tl * kWideEP + e0) = make_float4(l[0], l[1], l[2], l[3]);
       }
-      *reinterpret_cast<float4*>(ls + tl * kWideEP + e0) = make_float4(l[0], l[1], l[2], l[3]);
     }
   }
   __syncthreads();
   select_topk<kWideEP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w);
 }
 
-template <typename XT>
-static int launch_wide(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
-                       float* topk_w, cudaStream_t st) {
-  const size_t smem = sizeof(float) * kWideTB * kWideEP;  // the logits tile; the staging area is smaller
-  auto kern = route_wide_kernel<XT>;
+template <typename XT, int TMT>
+static int launch_wide_tmt(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
+                           float* topk_w, cudaStream_t st) {
+  constexpr size_t stage = sizeof(float) * 2 * kWideBuf, logits = sizeof(float) * 8 * TMT * kWideEP;
+  constexpr size_t smem = stage > logits ? stage : logits;
+  auto kern = route_wide_kernel<XT, TMT>;
   static bool attr_done = false;  // per instantiation and process, idempotent
   if (!attr_done) {
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -207,8 +251,28 @@ static int launch_wide(moe_plan* p, const void* x, const void* wr, const float* 
   }
   const moe_config_t& c = p->cfg;
   p->launches += 1;
-  return (int)launch_maybe_pdl(false, kern, dim3((c.T + kWideTB - 1) / kWideTB), dim3(kRouteThreads), smem, st, (const XT*)x,
-                         (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w);
+  return (int)launch_maybe_pdl(false, kern, dim3((c.T + 8 * TMT - 1) / (8 * TMT)), dim3(kWideThreads), smem, st,
+                               (const XT*)x, (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w);
+}
+
+template <typename XT>
+static int launch_wide(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
+                       float* topk_w, cudaStream_t st) {
+  // Tokens per thread: the time is (waves of CTAs over the SMs) x TMT; ties go to the larger tile.
+  const int T = p->cfg.T, sms = p->sm_count > 0 ? p->sm_count : 148;
+  int best = 8, best_cost = 1 << 30;
+  for (int tmt = 8; tmt >= 4; --tmt) {
+    const int ctas = (T + 8 * tmt - 1) / (8 * tmt);
+    const int cost = (ctas + sms - 1) / sms * tmt;
+    if (cost < best_cost) { best_cost = cost; best = tmt; }
+  }
+  switch (best) {
+    case 4: return launch_wide_tmt<XT, 4>(p, x, wr, bias, topk_idx, topk_w, st);
+    case 5: return launch_wide_tmt<XT, 5>(p, x, wr, bias, topk_idx, topk_w, st);
+    case 6: return launch_wide_tmt<XT, 6>(p, x, wr, bias, topk_idx, topk_w, st);
+    case 7: return launch_wide_tmt<XT, 7>(p, x, wr, bias, topk_idx, topk_w, st);
+    default: return launch_wide_tmt<XT, 8>(p, x, wr, bias, topk_idx, topk_w, st);
+  }
 }
 
 // The latency-bound shapes (E <= 64).  x and Wr tiles stay in their natural [row][h] layout in shared
