@@ -75,7 +75,7 @@ size_t carve(const moe_config_t& c, const Geometry& g, char* base, Scratch* s, s
   t.cta_base = (int*)take(sizeof(int) * (size_t)(g.nblk > 0 ? g.nblk : 1) * c.E);
   t.tile_base = (int*)take(sizeof(int) * (size_t)(c.E + 1));
   t.clock_probe = (unsigned long long*)take(sizeof(unsigned long long) * 2);
-  t.gemm1_done = (int*)take(sizeof(int) * (size_t)(g.P > 0 ? g.P : 1));
+  t.gemm1_done = (int*)take(sizeof(int) * (size_t)((g.P > 0 ? g.P : 1) + 4));  // + the expert kernel's item and exit counters
   const size_t pool_rows = (size_t)g.P * kTileRows;
   if (!c.identity_experts) t.inter = take(pool_rows * c.F * g.eb);
   t.topk_idx = (int*)take(sizeof(int) * (size_t)c.T * c.K);

@@ -18,7 +18,7 @@ __device__ __forceinline__ void set_status(int* status, int code, int detail) {
 
 // Wait sites reported in the detail word of MOE_ERR_TIMEOUT.
 enum WaitSite { kWaitTileTable = 1, kWaitMbarTma = 3, kWaitMbarMma = 4,
-                kWaitMbarEpi = 5, kWaitMbarTmemFree = 6, kWaitTileReady = 7 };
+                kWaitMbarEpi = 5, kWaitMbarTmemFree = 6, kWaitTileReady = 7, kWaitItem = 8 };
 
 struct Scratch {          // device pointers carved out of the caller's workspace
   int* status;            // [4]
@@ -31,7 +31,7 @@ struct Scratch {          // device pointers carved out of the caller's workspac
   int* cta_base;          // [nblk * E] mode 0: exclusive prefix inside the expert
   int* tile_base;         // [E + 1]    mode 0: first pool tile of each expert
   unsigned long long* clock_probe;  // [2] cycles, nanoseconds of CTA 0 inside the tensor-core kernels
-  int* gemm1_done;        // [P]    per-tile status counter: GEMM1 blocks finished (x4 epilogue warps)
+  int* gemm1_done;        // [P+4]  per-tile status counter: GEMM1 blocks finished (x4 epilogue warps); [P..P+1] item counters, [P+2..P+3] exit counters of the expert kernel's launches
   void* inter;            // [P*128, F] SwiGLU intermediate
   // moe_layer's internal buffers
   int* topk_idx;

@@ -306,6 +306,7 @@ reset_kernel(int* __restrict__ counters, int n_counters, int* __restrict__ exper
   pdl_trigger();
   for (int i = i0; i < n_counters; i += stride) counters[i] = 0;
   if (i0 == 0) *rows_done = 0;
+  if (i0 < 4) gemm1_done[P + i0] = 0;  // the expert kernel's item and exit counters
   for (int i = i0; i < E; i += stride) expert_count[i] = 0;
   for (int i = i0; i < P; i += stride) {
     tile_expert[i] = -1;

@@ -32,11 +32,21 @@
 namespace moehub {
 
 // ---- the grouped GEMM -----------------------------------------------------------------------
+// Items are handed out dynamically: every CTA starts with item blockIdx.x and then takes the next
+// unclaimed item of the list (one global atomicAdd per item, issued by the producer thread while the
+// previous item's loads run), so CTAs whose items were short take more of them.  The producer
+// publishes each item index (-1: no more) to the other roles through a ring in shared memory with one
+// mbarrier per slot.  The producer is at most 4 items (one per pipeline stage) ahead of the MMA
+// thread and that at most 2 (the accumulators) ahead of the epilogue, so 16 slots never wrap onto an
+// unread one.
+constexpr int kItemRing = 16;
 struct TcShared {
   unsigned long long full[kStages];
   unsigned long long empty[kStages];
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
+  unsigned long long item_bar[kItemRing];
+  int item_ring[kItemRing];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -69,6 +79,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       mbar_init(smem_u32(&sh->tmem_full[a]), 1);
       mbar_init(smem_u32(&sh->tmem_empty[a]), 4);
     }
+    for (int i = 0; i < kItemRing; ++i) mbar_init(smem_u32(&sh->item_bar[i]), 1);
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -121,6 +132,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     return it;
   };
   const int first_item = item_begin + blockIdx.x;
+  int* work_counter = prm.work_counter + (phase == 2 ? 1 : 0);
+  volatile int* item_ring = sh->item_ring;
 
   int fail_site = 0;
   if (warp == 0) {
@@ -131,7 +144,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       int armed[kStages];
 #pragma unroll
       for (int s = 0; s < kStages; ++s) armed[s] = 0;
-      for (int item = first_item; item < item_end && !fail_site; item += gridDim.x) {
+      int item = first_item;
+      for (int local_item = 0; !fail_site; ++local_item) {
+        const int slot = local_item & (kItemRing - 1);
+        item_ring[slot] = item < item_end ? item : -1;
+        mbar_arrive(smem_u32(&sh->item_bar[slot]));  // release: the slot is written before the phase completes
+        if (item >= item_end) break;
+        const int next_item = item_begin + (int)gridDim.x + atomicAdd(work_counter, 1);  // used after this item's loads
         const Item it = decode(item);
         if (it.type == 0 && tile_count != nullptr) {
           // Availability of this tile's rows (dispatch side): 128 rows stored, or every assignment of
@@ -180,6 +199,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
             if (s == stage) armed[s] += 1;
           if (++stage == kStages) { stage = 0; phase_bit ^= 1u; }
         }
+        item = next_item;
       }
       if (fail_site || *abort_flag) {
         // Leave no copy in flight: wait (bounded) for the last fill of every stage.
@@ -199,8 +219,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     if (lane == 0) {
       int stage = 0;
       uint32_t phase_bit = 0;
-      int local_item = 0;
-      for (int item = first_item; item < item_end && !fail_site; item += gridDim.x, ++local_item) {
+      for (int local_item = 0; !fail_site; ++local_item) {
+        const int slot = local_item & (kItemRing - 1);
+        if (!mbar_wait(smem_u32(&sh->item_bar[slot]), (uint32_t)(local_item / kItemRing) & 1u, abort_flag, wait_ns)) { fail_site = kWaitItem; break; }
+        const int item = item_ring[slot];
+        if (item < 0) break;
         const Item it = decode(item);
         const int KB = it.type == 0 ? KB1 : KB2;
         const int acc = local_item & 1;
@@ -232,8 +255,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     const bool wide1 = F % 16 == 0 && (reinterpret_cast<uintptr_t>(inter) & 31) == 0;
     const bool wide2 = H % 16 == 0 && (reinterpret_cast<uintptr_t>(out) & 31) == 0;
     const int row_in_tile = quarter * 32 + lane;
-    int local_item = 0;
-    for (int item = first_item; item < item_end && !fail_site; item += gridDim.x, ++local_item) {
+    for (int local_item = 0; !fail_site; ++local_item) {
+      const int slot = local_item & (kItemRing - 1);
+      if (!mbar_wait(smem_u32(&sh->item_bar[slot]), (uint32_t)(local_item / kItemRing) & 1u, abort_flag, wait_ns)) { fail_site = kWaitItem; break; }
+      const int item = item_ring[slot];
+      if (item < 0) break;
       const Item it = decode(item);
       const int acc = local_item & 1;
       const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
@@ -307,6 +333,15 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   tc_fence_after();
   pdl_trigger();
   probe.finish();
+  if (threadIdx.x == 0) {
+    // Every CTA has taken its last item index by now; the last one to leave puts the counters back to
+    // zero, so a launch never depends on the host having cleared them.
+    int* exit_counter = work_counter + 2;
+    if (atomicAdd(exit_counter, 1) == (int)gridDim.x - 1) {
+      *work_counter = 0;
+      *exit_counter = 0;
+    }
+  }
   if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
 }
@@ -377,15 +412,15 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   }
   const int grid = p->sm_count;
   const int NB1 = (c.F + 127) / 128, NB2 = (c.H + 255) / 256;
-  // One launch for both GEMMs, or one per GEMM.  In one launch the items of the two GEMMs differ in
-  // length and are dealt round-robin; with many small experts that deal gets uneven (5 % at E = 256
-  // under Zipf routing, measured and reproduced by counting), so the default splits there.
+  // One launch for both GEMMs, or one per GEMM.  With many small experts (E = 256 under Zipf routing)
+  // the single launch measures 2-3 % slower than two, also with items handed out dynamically, so the
+  // default splits there.
   const int fused = c.ffn_split == 2 ? 1 : (c.ffn_split == 1 ? 0 : (c.E <= 64 ? 1 : 0));
   const bool pairs = c.ffn_kernel == 2;  // opt-in: the CTA-pair kernel
   const int workers = pairs ? grid / 2 : grid;
   if (p->P > kMaxListTiles) return MOE_ERR_UNSUPPORTED;  // the work list lives in the kernel's shared memory
-  if (tile_count == nullptr &&  // a call outside moe_layer: the per-tile GEMM1 counters are not reset by a dispatch
-      cudaMemsetAsync(p->s.gemm1_done, 0, sizeof(int) * (size_t)p->P, st) != cudaSuccess)
+  if (tile_count == nullptr &&  // a call outside moe_layer: the GEMM1 and item counters are not reset by a dispatch
+      cudaMemsetAsync(p->s.gemm1_done, 0, sizeof(int) * (size_t)(p->P + 4), st) != cudaSuccess)
     return MOE_ERR_CUDA;
   mark(p, 3, st);
   FfnParams prm;
@@ -399,6 +434,7 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   prm.inter = (__nv_bfloat16*)p->s.inter;
   prm.out = (__nv_bfloat16*)out_rows;
   prm.gemm1_done = p->s.gemm1_done;
+  prm.work_counter = p->s.gemm1_done + p->P;
   prm.tile_count = tile_count;
   prm.rows_done = rows_done;
   prm.wait_ns = c.wait_limit_ns ? c.wait_limit_ns : kDefaultWaitNs;

@@ -13,7 +13,7 @@ constexpr int kUmmaN = 256;
 constexpr int kABytes = kTileRows * kBK * 2;  // 16 KB
 constexpr int kBBytes = kUmmaN * kBK * 2;     // 32 KB
 constexpr int kStageBytes = kABytes + kBBytes;
-constexpr int kTcSmem = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kTcSmem = kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers, item ring*/;
 constexpr unsigned long long kDefaultWaitNs = 2000000000ull;  // default bound on any single wait: 2 s
 
 // ---- PTX wrappers ---------------------------------------------------------------------------
@@ -236,6 +236,8 @@ struct FfnParams {
   __nv_bfloat16* inter;
   __nv_bfloat16* out;
   int* gemm1_done;
+  int* work_counter;  // [4] items handed out beyond the first one per CTA: [0] phases 0 and 1, [1] phase 2 (zero at launch; the
+                      // last CTA to leave zeroes it again); [2], [3]: CTAs that left
   const int* tile_count;
   const int* rows_done;
   int total_rows;
