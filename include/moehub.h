@@ -76,8 +76,8 @@ typedef struct {
                                    (cta_group::2, two tiles per MMA; bf16)                    */
   int32_t ffn_split;            /* 1: one launch per expert GEMM; 2: both GEMMs in one persistent
                                    launch (per-tile status counters gate GEMM2); 0: choose
-                                   (one launch when E <= 64, where its round-robin deal of the
-                                   two item kinds stays even)                                 */
+                                   (one launch when E <= 64; with more, smaller experts two
+                                   launches measure faster)                                   */
   int64_t capacity_rows;        /* mode 1: rows per expert region, multiple of 128, 0 = T
                                    rounded up (overflow-free); modes 0/2: ignored            */
   uint64_t spin_limit;          /* bound (iterations) on the dispatch kernels' waits, 0 = 1<<22 */
