@@ -173,6 +173,37 @@ def test_router_renormalize_and_bias(renorm):
     Hh.check_route(idx, tw, ridx, rw)
 
 
+# Every shape of the two router kernels: the narrow kernel's four lane layouts (E <= 8, 16, 32, 64), each
+# with a block boundary inside T and an h range that ends inside a chunk, in both dtypes; the wide kernel
+# with every register-tile height it picks (4 to 8 tokens per thread follows from T on a 148-SM part:
+# T <= 4736 -> 4, <= 5920 -> 5, <= 7104 -> 6, <= 8288 -> 7, <= 9472 -> 8) and E below and at 256.
+ROUTER_SHAPES = [
+    # (T, H, E, K, dtype, zipf_s)
+    (77, 264, 7, 2, BF16, 0.0), (1100, 520, 8, 3, BF16, 1.0), (45, 132, 5, 5, FP32, 0.0),
+    (333, 1032, 16, 2, BF16, 0.0), (90, 260, 13, 4, FP32, 1.0),
+    (70, 520, 32, 6, BF16, 0.0), (1500, 264, 24, 2, BF16, 1.0), (33, 68, 17, 3, FP32, 0.0),
+    (130, 776, 60, 4, BF16, 0.0), (1030, 136, 64, 8, BF16, 1.0), (21, 132, 33, 2, FP32, 0.0),
+    (200, 72, 65, 8, BF16, 0.0), (4000, 40, 256, 8, BF16, 1.0), (5000, 40, 200, 4, BF16, 0.0),
+    (6500, 40, 256, 8, BF16, 1.0), (8000, 40, 129, 2, BF16, 0.0), (9000, 40, 256, 8, BF16, 1.0),
+    (300, 36, 100, 5, FP32, 1.0), (5100, 20, 256, 3, FP32, 0.0),
+]
+
+
+@pytest.mark.parametrize("shape", ROUTER_SHAPES, ids=lambda s: f"T{s[0]}_H{s[1]}_E{s[2]}_K{s[3]}_d{s[4]}_z{s[5]}")
+def test_router_every_kernel_shape(shape):
+    T, H, E, K, dtype, zipf = shape
+    w = inputs.Workload("router_shape", T=T, H=H, E=E, R=1, K=K, F=8, dtype=dtype, zipf_s=zipf, seed=11,
+                        identity_experts=True)
+    x, wr, bias, *_ = Hh.oracle_inputs(w, with_experts=False)
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED)
+    idx = torch.empty((T, K), dtype=torch.int32, device="cuda")
+    tw = torch.empty((T, K), dtype=torch.float32, device="cuda")
+    plan.moe_route(Hh.to_dev(x), Hh.to_dev(wr), Hh.to_dev(bias), idx, tw)
+    torch.cuda.synchronize()
+    ridx, rw, _ = oracle.route(x, wr, bias, K, dtype)
+    Hh.check_route(idx, tw, ridx, rw)
+
+
 # ------------------------------------------------------------------ dispatch edge cases
 @pytest.mark.parametrize("mode", MODES)
 def test_dispatch_all_tokens_to_one_expert_and_empty_experts(mode):
