@@ -4,6 +4,12 @@ dispatch stage (baseline scan scheme and the destination-agnostic paged scheme) 
 with CUDA events and prints algorithmic GB/s and the fraction of the measured HBM copy bandwidth.
 
     python -m paper_2605_05888_b200.sweep [--max-t 65536] [--iters 20] [--markdown]
+    python -m paper_2605_05888_b200.sweep --imbalance [--iters 20] [--markdown]
+
+The second form is the imbalance study (Section VI-B of the paper varies the standard deviation of the
+experts' load shares): the Mixtral-like layer (T 4096, H 4096, 8 experts, top-2, F 14336, bf16, real expert
+GEMMs) with the router bias -s*ln(1+pi(e)) for s from 0 to 3; per point the measured standard deviation of
+the experts' shares of the T*K rows, the hottest expert's share, the tiles used, and the layer time.
 
 Algorithmic bytes: dispatch T*H*b*(1+K) + 12*T*K (row read once, written K times; indices in, slot and
 source info out); combine T*H*b*(K+1) + 8*T*K.  Below T = 2048 the stages take a few microseconds and are
@@ -52,13 +58,64 @@ def time_point(w: inputs.Workload, mode: int, iters: int) -> dict:
             "imbalance_std": float(np.std(cnt / (w.T * w.K)))}
 
 
+def imbalance_point(w: inputs.Workload, weights, iters: int) -> dict:
+    x = inputs.make_x(w)
+    wr, bias = inputs.make_router(w)
+    bf = lambda a: torch.from_numpy(a).view(torch.int16).cuda().view(torch.bfloat16)
+    dx, dwr = bf(x), bf(wr)
+    dbias = None if bias is None else torch.from_numpy(bias).cuda()
+    plan = B.Plan(B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype))
+    y = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+    for _ in range(5):
+        plan.moe_layer(dx, dwr, dbias, *weights, y)
+    torch.cuda.synchronize()
+    code, detail = plan.moe_last_status()
+    assert code == 0, (code, detail)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        plan.moe_layer(dx, dwr, dbias, *weights, y)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / iters
+    cnt = plan.layer_tensor(3).cpu().numpy().astype(np.float64)
+    rows = w.T * w.K
+    return {"zipf_s": w.zipf_s, "std_of_expert_share": float(np.std(cnt / rows)), "hottest_share_of_rows": float(cnt.max() / rows),
+            "tiles_used": int(np.sum((cnt + 127) // 128)), "tiles_if_dense": (rows + 127) // 128, "layer_ms": ms,
+            "tokens_per_s": w.T / ms * 1e3}
+
+
+def imbalance_sweep(iters: int, markdown: bool) -> None:
+    base = inputs.C2
+    wg, wu, wd = inputs.make_all_expert_weights(base)
+    bf = lambda a: torch.from_numpy(a).view(torch.int16).cuda().view(torch.bfloat16)
+    weights = (bf(wg), bf(wu), bf(wd))
+    del wg, wu, wd
+    rows = [imbalance_point(base.with_(zipf_s=s), weights, iters) for s in (0.0, 0.25, 0.5, 1.0, 1.5, 2.0, 3.0)]
+    if not markdown:
+        for r in rows:
+            print(json.dumps(r))
+        return
+    print(f"Layer time = {iters} back-to-back `moe_layer` calls between two CUDA events, after 5 warm-ups.")
+    print()
+    print("| bias strength s | std of expert shares | hottest expert's share of rows | tiles used / dense | layer ms | tokens/s |")
+    print("|---|---|---|---|---|---|")
+    for r in rows:
+        print(f"| {r['zipf_s']:.2f} | {r['std_of_expert_share']:.4f} | {r['hottest_share_of_rows']:.3f} | {r['tiles_used']} / {r['tiles_if_dense']} | "
+              f"{r['layer_ms']:.3f} | {r['tokens_per_s']:.3e} |")
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--min-t", type=int, default=128)
     ap.add_argument("--max-t", type=int, default=65536)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--markdown", action="store_true")
+    ap.add_argument("--imbalance", action="store_true", help="the imbalance study on the Mixtral-like layer instead of the T sweep")
     args = ap.parse_args()
+    if args.imbalance:
+        imbalance_sweep(args.iters, args.markdown)
+        return
     peak, kind = hbm_peak_gbs()
     rows = []
     T = args.min_t
