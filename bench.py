@@ -38,8 +38,8 @@ WORKLOADS = {"c1": inputs.C1, "c2": inputs.C2, "c3": inputs.C3, "c4": inputs.C4,
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
 # ncu capture summarised in profiles/ffn_tc_kernel_c2_small.md.  The capture ran the quarter-size case
-# (901.6 MB per launch); C2 proper does 4x its flops with 4x its weights, so the figure is scaled by 4.
-NCU_TRAFFIC_BYTES = {"mixtral_like_bf16_small": 901.6e6, "mixtral_like_bf16": 4 * 901.6e6}
+# (898.9 MB per launch); C2 proper does 4x its flops with 4x its weights, so the figure is scaled by 4.
+NCU_TRAFFIC_BYTES = {"mixtral_like_bf16_small": 898.9e6, "mixtral_like_bf16": 4 * 898.9e6}
 
 
 def load_peaks() -> tuple[dict, str]:
