@@ -296,6 +296,33 @@ def test_dispatch_availability_counters_and_gated_consumer(mode):
     Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
 
 
+@pytest.mark.parametrize("split", [1, 2])
+def test_expert_kernel_can_be_called_again_without_a_dispatch_in_between(split):
+    """The expert kernel hands its items out through device counters and puts them back to zero itself:
+    three calls in a row on one dispatch result (the counter-gated form, where the host clears nothing)
+    give bit-identical rows, and those rows match the oracle."""
+    w = inputs.Workload("many_items", T=700, H=520, E=12, R=3, K=3, F=1032, dtype=BF16, seed=5)  # 288 items for 148 CTAs
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED, ffn_split=split)
+    dx = Hh.to_dev(x)
+    b = _dispatch_with_counters(w, plan, dx, Hh.to_dev(ref["topk_idx"]))
+    dwg, dwu, dwd = Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd)
+    outs = []
+    for _ in range(3):
+        out = torch.zeros_like(b["recv"])
+        plan.moe_expert_ffn(b["recv"], b["te"], dwg, dwu, dwd, out, b["tile_count"], b["rows_done"])
+        outs.append(out)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    used = (b["src"] >= 0)
+    assert torch.equal(outs[0][used], outs[1][used]) and torch.equal(outs[0][used], outs[2][used])
+    y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
+    plan.moe_combine(outs[2], b["slot"], Hh.to_dev(ref["topk_w"]), y)
+    torch.cuda.synchronize()
+    Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+
+
 @pytest.mark.parametrize("kernel", [0, 2])
 def test_consumer_wait_runs_out_and_reports_it(kernel):
     """A flag that nothing sets: the consumer is given availability counters that stay at zero.  Its
