@@ -12,6 +12,10 @@
 //                   inter[:, f0:f0+128] = bf16( silu(D[:, 0:128]) * D[:, 128:256] )
 //   GEMM2         : D[128, 256] = inter[128, F] * Wd[e, h0:h0+256, :]^T ; out = bf16(D)
 //
+// A tile that is its expert's only one and holds at most 64 rows runs both GEMMs the other way
+// round (D^T: 128 weight rows x the tile's rows rounded up to 16, two MMAs per 16 k for the two
+// halves of the weight block; the epilogue stores transposed).
+//
 // Work order is expert-major, then column block, then tile, so that CTAs running at the same time
 // share the weight block through L2 and an expert's rows stay L2-resident across its column blocks.
 //
@@ -54,7 +58,8 @@ struct TcShared {
 __global__ void __launch_bounds__(kTcThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_bg,
               const __grid_constant__ CUtensorMap map_bu, const __grid_constant__ CUtensorMap map_a2,
-              const __grid_constant__ CUtensorMap map_bd, const FfnParams prm) {
+              const __grid_constant__ CUtensorMap map_bd, const __grid_constant__ CUtensorMap map_a1t,
+              const __grid_constant__ CUtensorMap map_a2t, const FfnParams prm) {
   const int phase = prm.phase, E = prm.E, F = prm.F, H = prm.H;
   __nv_bfloat16* __restrict__ inter = prm.inter;
   __nv_bfloat16* __restrict__ out = prm.out;
@@ -98,7 +103,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   ClockProbe probe(prm.clock_probe);
   const unsigned long long wait_ns = prm.wait_ns;
 
-  const int NB1 = (F + 127) / 128, NB2 = (H + 255) / 256;
+  const int NB1 = (F + 127) / 128;
   const int KB1 = (H + kBK - 1) / kBK, KB2 = (F + kBK - 1) / kBK;
   int item_begin = 0, item_end = wl.seg_start[nseg];
   if (phase == 1) item_end = wl.n1;
@@ -126,6 +131,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     it.type = wl.seg_info[lo] >> 16;
     it.e = wl.seg_info[lo] & 0xffff;
     const int m = wl.estart[it.e + 1] - wl.estart[it.e];
+    it.m = m;
     const int local = item - wl.seg_start[lo];
     it.nb = local / m;
     it.tile = wl.tiles[wl.estart[it.e] + local % m];
@@ -147,9 +153,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       int item = first_item;
       for (int local_item = 0; !fail_site; ++local_item) {
         const int slot = local_item & (kItemRing - 1);
-        item_ring[slot] = item < item_end ? item : -1;
-        mbar_arrive(smem_u32(&sh->item_bar[slot]));  // release: the slot is written before the phase completes
-        if (item >= item_end) break;
+        if (item >= item_end) {
+          item_ring[slot] = -1;
+          mbar_arrive(smem_u32(&sh->item_bar[slot]));
+          break;
+        }
         const int next_item = item_begin + (int)gridDim.x + atomicAdd(work_counter, 1);  // used after this item's loads
         const Item it = decode(item);
         if (it.type == 0 && tile_count != nullptr) {
@@ -179,14 +187,30 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
           }
           asm volatile("fence.proxy.async.global;" ::: "memory");
         }
-        const CUtensorMap* ma = it.type == 0 ? &map_a1 : &map_a2;
+        // The only tile of an expert with at most 64 rows is computed the other way round: the weight rows
+        // are the M side of the MMA and the tile's rows, rounded up to 16, the N side, so the MMA work and
+        // the row operand shrink with the rows instead of staying those of 128.  Such an expert's weights
+        // are used once, so its items are bound by streaming them, and the narrow form helps (C3 -3.6 %,
+        // C4 -4 %); the short last tile of an expert with several tiles stays in the normal form: its
+        // weights come from L2, and eight small MMAs per k-block took as long as four full ones
+        // (measured: the clock rose 6 %, the step time did not fall).  The row count is final here: the
+        // tile was declared ready above (GEMM1) or long ago (GEMM2).
+        int n16 = 0;
+        if (tile_count != nullptr) {
+          const int r = tile_count[it.tile];
+          if (r <= kThinRows && it.m == 1) n16 = max(1, (r + 15) / 16);
+        }
+        item_ring[slot] = item | (n16 << kThinShift);
+        mbar_arrive(smem_u32(&sh->item_bar[slot]));  // release: the slot is written before the phase completes
+        const CUtensorMap* ma = it.type == 0 ? (n16 ? &map_a1t : &map_a1) : (n16 ? &map_a2t : &map_a2);
+        const uint32_t stage_tx = n16 ? (uint32_t)(kThinRows * kBK * 2 + kBBytes) : (uint32_t)kStageBytes;
         const int KB = it.type == 0 ? KB1 : KB2;
         for (int kb = 0; kb < KB; ++kb) {
           if (!mbar_wait(smem_u32(&sh->empty[stage]), phase_bit ^ 1u, abort_flag, wait_ns)) { fail_site = kWaitMbarTma; break; }
           const uint32_t full = smem_u32(&sh->full[stage]);
           const uint32_t a_dst = smem_u32(stage_base + stage * kStageBytes);
           const uint32_t b_dst = a_dst + kABytes;
-          mbar_expect_tx(full, kStageBytes);
+          mbar_expect_tx(full, stage_tx);
           tma_load_2d(a_dst, ma, full, kb * kBK, it.tile * kTileRows);
           if (it.type == 0) {
             tma_load_3d(b_dst, &map_bg, full, kb * kBK, it.nb * 128, it.e);
@@ -222,8 +246,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       for (int local_item = 0; !fail_site; ++local_item) {
         const int slot = local_item & (kItemRing - 1);
         if (!mbar_wait(smem_u32(&sh->item_bar[slot]), (uint32_t)(local_item / kItemRing) & 1u, abort_flag, wait_ns)) { fail_site = kWaitItem; break; }
-        const int item = item_ring[slot];
-        if (item < 0) break;
+        const int entry = item_ring[slot];
+        if (entry < 0) break;
+        const int item = entry & ((1 << kThinShift) - 1), n16 = entry >> kThinShift;
         const Item it = decode(item);
         const int KB = it.type == 0 ? KB1 : KB2;
         const int acc = local_item & 1;
@@ -237,9 +262,21 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
           const uint32_t a_addr = smem_u32(stage_base + stage * kStageBytes);
           const uint64_t adesc = smem_desc_sw128(a_addr);
           const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
+          if (n16 == 0) {
 #pragma unroll
-          for (int k = 0; k < kBK / 16; ++k)  // 16 k-elements = 32 bytes = 2 descriptor units per step
-            tc_mma(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
+            for (int k = 0; k < kBK / 16; ++k)  // 16 k-elements = 32 bytes = 2 descriptor units per step
+              tc_mma(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
+          } else {
+            // thin tile: D[128 weight rows, 16*n16 tile rows], once per half of the weight block (gate / up,
+            // or the two 128-row halves of the Wd block), into accumulator columns 0.. and 128..
+            const uint32_t idesc = thin_idesc(n16);
+            const uint64_t wdesc2 = smem_desc_sw128(a_addr + kABytes + kBBytes / 2);
+#pragma unroll
+            for (int k = 0; k < kBK / 16; ++k) {
+              tc_mma(d_tmem, bdesc + 2 * k, adesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+              tc_mma(d_tmem + 128, wdesc2 + 2 * k, adesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+          }
           tc_commit(smem_u32(&sh->empty[stage]));  // the stage is free once these MMAs have read it
           if (++stage == kStages) { stage = 0; phase_bit ^= 1u; }
         }
@@ -258,8 +295,9 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     for (int local_item = 0; !fail_site; ++local_item) {
       const int slot = local_item & (kItemRing - 1);
       if (!mbar_wait(smem_u32(&sh->item_bar[slot]), (uint32_t)(local_item / kItemRing) & 1u, abort_flag, wait_ns)) { fail_site = kWaitItem; break; }
-      const int item = item_ring[slot];
-      if (item < 0) break;
+      const int entry = item_ring[slot];
+      if (entry < 0) break;
+      const int item = entry & ((1 << kThinShift) - 1), n16 = entry >> kThinShift;
       const Item it = decode(item);
       const int acc = local_item & 1;
       const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
@@ -267,7 +305,41 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kUmmaN);
       const size_t row = (size_t)it.tile * kTileRows + row_in_tile;
-      if (it.type == 0) {
+      if (n16 != 0) {
+        // thin tile: this lane owns a weight row (an F or H column of the result), the accumulator's
+        // columns are the tile's rows; a warp's 32 lanes write 64 contiguous bytes of one output row.
+        const size_t row0 = (size_t)it.tile * kTileRows;
+        if (it.type == 0) {
+          const int f = it.nb * 128 + row_in_tile;
+#pragma unroll 1
+          for (int c = 0; c < 16 * n16; c += 16) {
+            uint32_t g[16], u[16];
+            tc_ld16(t_row + c, g);
+            tc_ld16(t_row + 128 + c, u);
+            tc_wait_ld();
+            if (f < F) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                inter[(row0 + c + i) * F + f] = __float2bfloat16_rn(silu_mul(__uint_as_float(g[i]), __uint_as_float(u[i])));
+            }
+          }
+        } else {
+#pragma unroll 1
+          for (int half = 0; half < 2; ++half) {
+            const int h = it.nb * 256 + half * 128 + row_in_tile;
+#pragma unroll 1
+            for (int c = 0; c < 16 * n16; c += 16) {
+              uint32_t v[16];
+              tc_ld16(t_row + half * 128 + c, v);
+              tc_wait_ld();
+              if (h < H) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) out[(row0 + c + i) * H + h] = __float2bfloat16_rn(__uint_as_float(v[i]));
+              }
+            }
+          }
+        }
+      } else if (it.type == 0) {
         __nv_bfloat16* dst = inter + row * F + (size_t)it.nb * 128;
         const int ncols = min(128, F - it.nb * 128);
 #pragma unroll 1
@@ -403,6 +475,9 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   if ((rc = make_map_3d(enc, &bu, wu, c.E, c.F, c.H, 128)) != MOE_OK) return rc;
   if ((rc = make_map_2d(enc, &a2, p->s.inter, pool_rows, c.F, kTileRows)) != MOE_OK) return rc;
   if ((rc = make_map_3d(enc, &bd, wd, c.E, c.H, c.F, c.ffn_kernel == 2 ? 128 : 256)) != MOE_OK) return rc;
+  CUtensorMap a1t, a2t;  // the first kThinRows rows of a tile, for tiles computed the other way round
+  if ((rc = make_map_2d(enc, &a1t, recv, pool_rows, c.H, kThinRows)) != MOE_OK) return rc;
+  if ((rc = make_map_2d(enc, &a2t, p->s.inter, pool_rows, c.F, kThinRows)) != MOE_OK) return rc;
 
   static bool attr_done = false;  // per-process, idempotent
   if (!attr_done) {
@@ -419,6 +494,7 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   const bool pairs = c.ffn_kernel == 2;  // opt-in: the CTA-pair kernel
   const int workers = pairs ? grid / 2 : grid;
   if (p->P > kMaxListTiles) return MOE_ERR_UNSUPPORTED;  // the work list lives in the kernel's shared memory
+  if ((long long)p->P * (NB1 + NB2) >= (1ll << kThinShift)) return MOE_ERR_UNSUPPORTED;  // item index field of the ring
   if (tile_count == nullptr &&  // a call outside moe_layer: the GEMM1 and item counters are not reset by a dispatch
       cudaMemsetAsync(p->s.gemm1_done, 0, sizeof(int) * (size_t)(p->P + 4), st) != cudaSuccess)
     return MOE_ERR_CUDA;
@@ -444,7 +520,7 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   auto launch = [&](int phase) -> int {
     prm.phase = phase;
     if (pairs) return launch_ffn_tc2_kernel(a1, bg, bu, a2, bd, prm, grid, st);
-    return launch_pdl(ffn_tc_kernel, dim3(grid), dim3(kTcThreads), kTcSmem, st, a1, bg, bu, a2, bd, prm) == cudaSuccess
+    return launch_pdl(ffn_tc_kernel, dim3(grid), dim3(kTcThreads), kTcSmem, st, a1, bg, bu, a2, bd, a1t, a2t, prm) == cudaSuccess
                ? 0 : MOE_ERR_CUDA;
   };
   if (fused) {

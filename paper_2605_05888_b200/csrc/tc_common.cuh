@@ -119,11 +119,19 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kUmmaN >> 3) << 17) |
                             ((uint32_t)(kTileRows >> 4) << 24);
 
+// Thin tiles (at most kThinRows rows): the MMA is M = 128 weight rows x N = 16*n16 tile rows.
+constexpr int kThinRows = 64;
+constexpr int kThinShift = 24;  // an item-ring entry is item | n16 << kThinShift
+__host__ __device__ constexpr uint32_t thin_idesc(int n16) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n16 * 16 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
 constexpr int kMaxExperts = 256;
 
 struct Item {
   int type;   // 0: GEMM1 (+SwiGLU), 1: GEMM2
   int e, nb, tile;
+  int m;      // tiles of expert e
 };
 
 // The work list, built by every CTA for itself in shared memory from tile_expert[P] (the same
