@@ -135,7 +135,10 @@ int moe_dispatch(moe_plan_t* plan, const void* d_x, const int32_t* d_topk_idx, v
  *     neither.  When given, the tensor-core kernel waits before it reads a tile until
  *     tile_count[p] >= 128 or rows_done >= T*K (bounded by wait_limit_ns; on expiry the status
  *     word reads MOE_ERR_TIMEOUT and the kernel returns).  NULL: the rows are complete when the
- *     call is reached in stream order.  The SIMT kernel ignores them (stream order).
+ *     call is reached in stream order.  The SIMT kernel ignores them (stream order).  The
+ *     counters also tell the kernel how many rows a tile holds: with them, an expert whose only
+ *     tile holds at most 64 rows is computed in a narrower form (same result, less work);
+ *     without them every tile is computed as 128 rows.
  * out: d_out_rows [P*128,H] (dtype); rows of empty slots hold unspecified values.
  * The tensor-core kernels keep their work list in shared memory: P <= 4608 tiles (T*K <= 557 056 rows at
  * E = 256), MOE_ERR_UNSUPPORTED beyond. */
