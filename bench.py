@@ -327,12 +327,16 @@ def run_cuda(args, w: inputs.Workload) -> None:
             stages["ffn_gemm1"] = {"ms": sm["gemm1"], "TFLOPs": gemm1_flops / sm["gemm1"] / 1e9}
             stages["ffn_gemm2"] = {"ms": sm["gemm2"], "TFLOPs": gemm2_flops / sm["gemm2"] / 1e9}
         ach = stages["ffn"]["TFLOPs"]
+        # The kernel is timed inside a loop of whole layers that runs for hundreds of milliseconds under the
+        # power cap, so the denominator is the sustained cuBLAS figure; the burst figure is given beside it.
+        peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
         roofline = {"kernel": "ffn_tc_kernel (expert GEMM1 + SwiGLU + GEMM2, tcgen05)", "bound": "tensor",
-                    "achieved": ach, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": ach / peaks["bf16_tflops"],
+                    "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
                     "traffic": NCU_TRAFFIC_BYTES.get(w.name),
-                    "peak_source": f"{peak_kind} bf16_tflops (burst); the kernel runs power-capped at the clock in "
-                                   "clocks.ffn_kernel_sm_mhz",
-                    "frac_of_sustained_peak": ach / peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"]),
+                    "peak_source": f"{peak_kind} bf16_tflops_sustained (the kernel is timed inside a long, power-capped "
+                                   "loop; its clock is in clocks.ffn_kernel_sm_mhz)",
+                    "frac_of_burst_peak": ach / peaks["bf16_tflops"],
+                    "frac_of_sustained_peak": ach / peak,
                     "frac_of_nominal_2250": ach / 2250.0,
                     "useful_flops_per_launch": gemm1_flops + gemm2_flops}
 
