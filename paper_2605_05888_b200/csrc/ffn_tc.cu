@@ -193,12 +193,15 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
         // are used once, so its items are bound by streaming them, and the narrow form helps (C3 -3.6 %,
         // C4 -4 %); the short last tile of an expert with several tiles stays in the normal form: its
         // weights come from L2, and eight small MMAs per k-block took as long as four full ones
-        // (measured: the clock rose 6 %, the step time did not fall).  The row count is final here: the
-        // tile was declared ready above (GEMM1) or long ago (GEMM2).
+        // (measured: the clock rose 6 %, the step time did not fall).  Such a tile runs the normal form on
+        // its first 64 rows only (M = 64 MMAs, the same count of instructions at half the work each: under the
+        // power cap the Phi-like layer and C3 gain 1.5 %).  The row count is final here: the tile was
+        // declared ready above (GEMM1) or long ago (GEMM2).
         int n16 = 0;
         if (tile_count != nullptr) {
           const int r = tile_count[it.tile];
           if (r <= kThinRows && it.m == 1) n16 = max(1, (r + 15) / 16);
+          else if (r <= kThinRows) n16 = kHalfForm;  // the short last tile of a larger expert: M = 64 MMAs
         }
         item_ring[slot] = item | (n16 << kThinShift);
         mbar_arrive(smem_u32(&sh->item_bar[slot]));  // release: the slot is written before the phase completes
@@ -262,10 +265,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
           const uint32_t a_addr = smem_u32(stage_base + stage * kStageBytes);
           const uint64_t adesc = smem_desc_sw128(a_addr);
           const uint64_t bdesc = smem_desc_sw128(a_addr + kABytes);
-          if (n16 == 0) {
+          if (n16 == 0 || n16 == kHalfForm) {
+            const uint32_t idesc = n16 == 0 ? kIdesc : kIdescHalf;  // 128 or 64 rows of the tile
 #pragma unroll
             for (int k = 0; k < kBK / 16; ++k)  // 16 k-elements = 32 bytes = 2 descriptor units per step
-              tc_mma(d_tmem, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
+              tc_mma(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
           } else {
             // thin tile: D[128 weight rows, 16*n16 tile rows], once per half of the weight block (gate / up,
             // or the two 128-row halves of the Wd block), into accumulator columns 0.. and 128..
@@ -304,8 +308,15 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag, wait_ns, 500)) { fail_site = kWaitMbarEpi; break; }
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kUmmaN);
-      const size_t row = (size_t)it.tile * kTileRows + row_in_tile;
-      if (n16 != 0) {
+      size_t row = (size_t)it.tile * kTileRows + row_in_tile;
+      bool row_live = true;
+      if (n16 == kHalfForm) {
+        // An M = 64 accumulator keeps 16 rows in each quadrant of the 128 lanes: row r sits in lane
+        // 32 * (r / 16) + r % 16 (checked against the oracle; rows in lanes 0-63 is not the layout).
+        row_live = lane < 16;
+        row = (size_t)it.tile * kTileRows + quarter * 16 + lane;
+      }
+      if (n16 != 0 && n16 != kHalfForm) {
         // thin tile: this lane owns a weight row (an F or H column of the result), the accumulator's
         // columns are the tile's rows; a warp's 32 lanes write 64 contiguous bytes of one output row.
         const size_t row0 = (size_t)it.tile * kTileRows;
@@ -354,6 +365,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
             const float gv = __uint_as_float(g[i]);
             s[i] = silu_mul(gv, __uint_as_float(u[i]));
           }
+          if (!row_live) continue;
           if (wide1 && c + 16 <= ncols) {
             st_global_32B(dst + c, Vec16<__nv_bfloat16>::pack(s), Vec16<__nv_bfloat16>::pack(s + 8));
           } else {
@@ -373,6 +385,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
           float f[32];
 #pragma unroll
           for (int i = 0; i < 16; ++i) { f[i] = __uint_as_float(r0[i]); f[16 + i] = __uint_as_float(r1[i]); }
+          if (!row_live) continue;
           if (wide2 && c + 32 <= ncols) {
             st_global_32B(dst + c, Vec16<__nv_bfloat16>::pack(f), Vec16<__nv_bfloat16>::pack(f + 8));
             st_global_32B(dst + c + 16, Vec16<__nv_bfloat16>::pack(f + 16), Vec16<__nv_bfloat16>::pack(f + 24));

@@ -126,6 +126,10 @@ __host__ __device__ constexpr uint32_t thin_idesc(int n16) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n16 * 16 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 }
 
+// Short last tile of an expert with several tiles: M = 64 MMAs on the tile's first 64 rows.
+constexpr int kHalfForm = 8;  // value of the n16 field for this form (thin tiles use 1..4)
+constexpr uint32_t kIdescHalf = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kUmmaN >> 3) << 17) | ((uint32_t)(64 >> 4) << 24);
+
 constexpr int kMaxExperts = 256;
 
 struct Item {
