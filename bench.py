@@ -39,7 +39,8 @@ WORKLOADS = {"c1": inputs.C1, "c2": inputs.C2, "c3": inputs.C3, "c4": inputs.C4,
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
 # ncu capture summarised in profiles/ffn_tc_kernel_c2_small.md.  The capture ran the quarter-size case
 # (898.9 MB per launch); C2 proper does 4x its flops with 4x its weights, so the figure is scaled by 4.
-NCU_TRAFFIC_BYTES = {"mixtral_like_bf16_small": 898.9e6, "mixtral_like_bf16": 4 * 898.9e6}
+# C4: profiles/ffn_tc_kernel_c4.md, the full-size workload itself (1.065 GB read + 17.3 MB written per launch).
+NCU_TRAFFIC_BYTES = {"mixtral_like_bf16_small": 898.9e6, "mixtral_like_bf16": 4 * 898.9e6, "qwen_moe_like_bf16": 1082.6e6}
 
 
 def load_peaks() -> tuple[dict, str]:
@@ -327,6 +328,11 @@ def run_cuda(args, w: inputs.Workload) -> None:
             stages["ffn_gemm1"] = {"ms": sm["gemm1"], "TFLOPs": gemm1_flops / sm["gemm1"] / 1e9}
             stages["ffn_gemm2"] = {"ms": sm["gemm2"], "TFLOPs": gemm2_flops / sm["gemm2"] / 1e9}
         ach = stages["ffn"]["TFLOPs"]
+        # Algorithmic bytes of the two GEMMs: the weights of every expert that has rows, once; the rows in
+        # and out; the intermediate written and read back.
+        active = int((counts > 0).sum())
+        ffn_bytes = 3.0 * active * w.F * w.H * eb + 2.0 * rows * w.H * eb + 2.0 * rows * w.F * eb
+        stages["ffn"]["GBps"] = ffn_bytes / t_ffn / 1e6
         # The kernel is timed inside a loop of whole layers that runs for hundreds of milliseconds under the
         # power cap, so the denominator is the sustained cuBLAS figure; the burst figure is given beside it.
         peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
@@ -339,6 +345,12 @@ def run_cuda(args, w: inputs.Workload) -> None:
                     "frac_of_sustained_peak": ach / peak,
                     "frac_of_nominal_2250": ach / 2250.0,
                     "useful_flops_per_launch": gemm1_flops + gemm2_flops}
+        if ffn_bytes / (hbm_peak * 1e9) > (gemm1_flops + gemm2_flops) / (peak * 1e12):
+            # About a tile per expert: streaming the weights takes longer than the MMAs could, so the same
+            # kernel is graded against the copy rate.
+            roofline.update({"bound": "hbm", "achieved": stages["ffn"]["GBps"], "peak": hbm_peak, "unit": "GB/s",
+                             "frac": stages["ffn"]["GBps"] / hbm_peak, "peak_source": f"{peak_kind} hbm_gbs",
+                             "algorithmic_bytes_per_launch": ffn_bytes, "tensor_TFLOPs": ach})
 
     # the CPU oracle on a bounded sample of the same batch (N = 1 only)
     cpu = None
