@@ -250,6 +250,20 @@ def run_cuda(args, w: inputs.Workload) -> None:
         stage_ms += np.array(plan.moe_layer_timed(dx, dwr, dbias, dwg, dwu, dwd, y))
     stage_ms /= args.steps
 
+    # ---- availability timeline of the dispatch (when does each 128-row tile become ready): 5 traced layers ----
+    plan.moe_availability_trace(True)
+    for _ in range(5):
+        step()
+    torch.cuda.synchronize()
+    trace = plan.layer_tensor(8).cpu().numpy().astype(np.float64)
+    plan.moe_availability_trace(False)
+    ready = trace[2:][trace[2:] > 0] - trace[0]
+    availability = {"full_tiles": int(ready.size), "all_ready_us": (trace[1] - trace[0]) / 1e3,
+                    "first_full_tile_us": float(ready.min() / 1e3) if ready.size else None,
+                    "median_full_tile_us": float(np.median(ready) / 1e3) if ready.size else None,
+                    "last_full_tile_us": float(ready.max() / 1e3) if ready.size else None,
+                    "what": "microseconds after the first dispatch CTA started (device %globaltimer), one traced layer"}
+
     # ---- end to end through the host-buffer entry point: H2D of x and D2H of y inside the timing ----
     hx = torch.from_numpy(x.view(np.int16) if x.dtype == np.uint16 else x).pin_memory()
     hy = torch.empty_like(hx).pin_memory()
@@ -374,7 +388,7 @@ def run_cuda(args, w: inputs.Workload) -> None:
                     "api": "moe_layer_host_submit/_wait: pinned host x and y, two steps in flight, host wall clock",
                     "one_step_at_a_time": whole_job_tokens_per_s(w.T, world, ms_e2e_sync / args.steps)},
             "roofline": roofline, "cpu_baseline": cpu, "stages": stages, "dominant": roofline["kernel"],
-            "routing": routing_stats}
+            "routing": routing_stats, "availability": availability}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

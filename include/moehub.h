@@ -221,8 +221,17 @@ int moe_layer_timed(moe_plan_t* plan, const void* d_x, const void* d_wr, const f
 
 /* Device pointers of moe_layer's intermediate results inside the workspace (valid after a
  * moe_layer call completes): which = 0 topk_idx, 1 topk_w, 2 recv, 3 expert_count,
- * 4 tile_expert, 5 src_info, 6 slot_of, 7 out_rows. */
+ * 4 tile_expert, 5 src_info, 6 slot_of, 7 out_rows, 8 the availability trace (below). */
 int moe_layer_buffer(moe_plan_t* plan, int which, void** out_ptr);
+
+/* Availability trace (Section IV-D: when does a consumer learn that a tile is ready), for
+ * measurement.  While enabled, the dispatch kernels of this plan (moe_dispatch, moe_layer) raise the
+ * availability counters with value-returning atomics and write %globaltimer nanoseconds into a
+ * uint64 array [P + 2] in the workspace (moe_layer_buffer, which = 8): [0] the earliest start of a
+ * dispatch CTA, [1] the moment the global counter reached all T*K assignments, [2 + p] the moment
+ * tile p's counter reached 128 rows (0: the tile never filled).  Disabled (the default) the kernels
+ * are unchanged.  The flag is host-side state of the plan. */
+int moe_availability_trace(moe_plan_t* plan, int enable);
 
 /* Effective SM clock inside the tensor-core expert kernels since the last reset: one CTA of every
  * launch accumulates its elapsed SM cycles and nanoseconds; *out_mhz = cycles / time (0 if none ran).

@@ -23,7 +23,7 @@ STAGES = ["route", "dispatch", "worklist", "gemm1", "gemm2", "combine"]
 
 EXPORTS = ["moe_dispatch_noalloc", "moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
            "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host", "moe_layer_host_submit", "moe_layer_host_wait", "moe_layer_timed",
-           "moe_layer_buffer",
+           "moe_layer_buffer", "moe_availability_trace",
            "moe_ffn_clock_mhz", "moe_last_launch_count", "moe_last_status", "moe_strerror"]
 
 
@@ -65,6 +65,7 @@ def lib() -> ctypes.CDLL:
         L.moe_layer_host_wait.argtypes = [vp, ctypes.c_int64]
         L.moe_layer_timed.argtypes = [vp] * 9 + [ctypes.POINTER(ctypes.c_float)]
         L.moe_layer_buffer.argtypes = [vp, ctypes.c_int, ctypes.POINTER(vp)]
+        L.moe_availability_trace.argtypes = [vp, ctypes.c_int]
         L.moe_ffn_clock_mhz.argtypes = [vp, vp, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
         L.moe_last_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
         L.moe_last_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
@@ -207,6 +208,9 @@ class Plan:
         _check(lib().moe_layer_buffer(self.handle, which, ctypes.byref(out)), "moe_layer_buffer")
         return out.value
 
+    def moe_availability_trace(self, enable: bool) -> None:
+        _check(lib().moe_availability_trace(self.handle, int(enable)), "moe_availability_trace")
+
     def moe_ffn_clock_mhz(self, reset: bool = True, stream=None) -> float:
         out = ctypes.c_float()
         _check(lib().moe_ffn_clock_mhz(self.handle, _stream(stream), int(reset), ctypes.byref(out)), "moe_ffn_clock_mhz")
@@ -230,7 +234,7 @@ class Plan:
         el = torch.bfloat16 if c.dtype == DTYPE_BF16 else torch.float32
         shapes = {0: ((c.T, c.K), torch.int32), 1: ((c.T, c.K), torch.float32), 2: ((rows, c.H), el),
                   3: ((c.E,), torch.int32), 4: ((self.P,), torch.int32), 5: ((rows,), torch.int32),
-                  6: ((c.T, c.K), torch.int32), 7: ((rows, c.H), el)}
+                  6: ((c.T, c.K), torch.int32), 7: ((rows, c.H), el), 8: ((self.P + 2,), torch.int64)}
         shape, dt = shapes[which]
         ptr = self.moe_layer_buffer(which)
         off = ptr - self.workspace.data_ptr()

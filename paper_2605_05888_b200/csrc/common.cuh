@@ -31,6 +31,7 @@ struct Scratch {          // device pointers carved out of the caller's workspac
   int* cta_base;          // [nblk * E] mode 0: exclusive prefix inside the expert
   int* tile_base;         // [E + 1]    mode 0: first pool tile of each expert
   unsigned long long* clock_probe;  // [2] cycles, nanoseconds of CTA 0 inside the tensor-core kernels
+  unsigned long long* avail_ns;  // [P+2] availability trace (measurement): dispatch start, all-ready time, per-tile ready time
   int* gemm1_done;        // [P+4]  per-tile status counter: GEMM1 blocks finished (x4 epilogue warps); [P..P+1] item counters, [P+2..P+3] exit counters of the expert kernel's launches
   void* inter;            // [P*128, F] SwiGLU intermediate
   // moe_layer's internal buffers
@@ -66,6 +67,7 @@ struct moe_plan {
   cudaEvent_t ev_in[2], ev_done[2], ev_out[2];
   long long submitted;       // steps submitted so far
   int timing;                // moe_layer_timed: record an event after every kernel of the layer
+  int trace;                 // moe_availability_trace: the dispatch kernels write avail_ns
   cudaEvent_t tev[MOE_STAGE_COUNT + 1];
 };
 

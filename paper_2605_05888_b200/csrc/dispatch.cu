@@ -63,8 +63,18 @@ __device__ __forceinline__ void copy_rows(const uint4* __restrict__ x, uint4* __
 // raised by the number of rows (release), and the global counter by the block's assignments.  A
 // consumer may read a tile once its counter shows 128 rows, or once the global counter shows all
 // T*K assignments (partly filled last tiles are then final; tiles at zero never become work).
+// With avail_ns given (measurement only) the counters are raised with atomics that return the old value,
+// and the thread that completes a tile, or the batch, writes the time: avail_ns[0] earliest start of a
+// dispatch CTA, [1] the moment the global counter reached all T*K assignments, [2 + tile] the moment the
+// tile's counter reached 128 (0: the tile never filled).
+__device__ __forceinline__ unsigned long long now_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 __device__ __forceinline__ void signal_rows(const int* s_slot, int na, int* __restrict__ tile_count,
-                                            int* __restrict__ rows_done) {
+                                            int* __restrict__ rows_done, unsigned long long* __restrict__ avail_ns,
+                                            int total_rows) {
   asm volatile("fence.proxy.async.global;" ::: "memory");  // consumers read the rows through TMA
   __threadfence();
   __syncthreads();
@@ -72,21 +82,37 @@ __device__ __forceinline__ void signal_rows(const int* s_slot, int na, int* __re
   const int slot = a < na ? s_slot[a] : -1;
   const int tile = slot >= 0 ? slot / kTileRows : -1;
   const unsigned peers = __match_any_sync(0xffffffffu, tile);
-  if (tile >= 0 && (threadIdx.x % 32) == __ffs(peers) - 1)
-    asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(tile_count + tile), "r"(__popc(peers)) : "memory");
-  if (threadIdx.x == 0) asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(rows_done), "r"(na) : "memory");
+  const bool first = tile >= 0 && (threadIdx.x % 32) == __ffs(peers) - 1;
+  if (avail_ns == nullptr) {
+    if (first)
+      asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(tile_count + tile), "r"(__popc(peers)) : "memory");
+    if (threadIdx.x == 0) asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(rows_done), "r"(na) : "memory");
+    return;
+  }
+  if (first) {
+    int old;
+    const int n = __popc(peers);
+    asm volatile("atom.release.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(tile_count + tile), "r"(n) : "memory");
+    if (old < kTileRows && old + n >= kTileRows) avail_ns[2 + tile] = now_ns();
+  }
+  if (threadIdx.x == 0) {
+    int old;
+    asm volatile("atom.release.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(rows_done), "r"(na) : "memory");
+    if (old < total_rows && old + na >= total_rows) avail_ns[1] = now_ns();
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
 // Mode 0, kernel 1: histogram of one token block.  cta_count[blk][e].
 __global__ void __launch_bounds__(kDispThreads)
 hist_kernel(const int* __restrict__ topk_idx, int T, int E, int K, int tok_per_blk,
-            int* __restrict__ cta_count) {
+            int* __restrict__ cta_count, unsigned long long* __restrict__ avail_ns) {
   extern __shared__ int s_cnt[];  // [E]
   for (int e = threadIdx.x; e < E; e += kDispThreads) s_cnt[e] = 0;
   __syncthreads();
   pdl_wait();
   pdl_trigger();
+  if (avail_ns != nullptr && threadIdx.x == 0) atomicMin(avail_ns, now_ns());
   const int t0 = blockIdx.x * tok_per_blk;
   const int na = min(tok_per_blk, T - t0) * K;
   for (int a = threadIdx.x; a < na; a += kDispThreads) atomicAdd(&s_cnt[topk_idx[(size_t)t0 * K + a]], 1);
@@ -165,7 +191,8 @@ __global__ void __launch_bounds__(kDispThreads)
 scatter_kernel(const uint4* __restrict__ x, const int* __restrict__ topk_idx, int T, int E, int K,
                int tok_per_blk, int vec_per_row, const int* __restrict__ cta_base,
                const int* __restrict__ tile_base, uint4* __restrict__ recv, int* __restrict__ src_info,
-               int* __restrict__ slot_of, int* __restrict__ tile_count, int* __restrict__ rows_done) {
+               int* __restrict__ slot_of, int* __restrict__ tile_count, int* __restrict__ rows_done,
+               unsigned long long* __restrict__ avail_ns) {
   extern __shared__ int smem_i[];
   int* s_wcnt = smem_i;                          // [8][E] per-warp counts
   int* s_slot = smem_i + (kDispThreads / 32) * E;  // [kMaxAssign]
@@ -177,6 +204,7 @@ scatter_kernel(const uint4* __restrict__ x, const int* __restrict__ topk_idx, in
   __syncthreads();
   pdl_wait();
   pdl_trigger();
+  if (avail_ns != nullptr && threadIdx.x == 0) atomicMin(avail_ns, now_ns());
   const int a = threadIdx.x;  // one assignment per thread, na <= 256
   int e = -1, wrank = 0;
   if (a < na) e = topk_idx[(size_t)t0 * K + a];
@@ -196,7 +224,7 @@ scatter_kernel(const uint4* __restrict__ x, const int* __restrict__ topk_idx, in
   }
   __syncthreads();
   copy_rows<4>(x, recv, s_slot, t0, ntok, K, vec_per_row);
-  signal_rows(s_slot, na, tile_count, rows_done);
+  signal_rows(s_slot, na, tile_count, rows_done, avail_ns, T * K);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -209,7 +237,7 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
                        int* __restrict__ tile_table, int* __restrict__ pool_next,
                        int* __restrict__ tile_expert, uint4* __restrict__ recv, int* __restrict__ src_info,
                        int* __restrict__ slot_of, int* __restrict__ status, int* __restrict__ tile_count,
-                       int* __restrict__ rows_done) {
+                       int* __restrict__ rows_done, unsigned long long* __restrict__ avail_ns) {
   extern __shared__ int smem_i[];
   int* s_cnt = smem_i;        // [E] rows this block sends to expert e
   int* s_base = smem_i + E;   // [E] first LocalRowID this block got from expert e's row pointer
@@ -222,6 +250,7 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
   __syncthreads();
   pdl_wait();
   pdl_trigger();
+  if (avail_ns != nullptr && threadIdx.x == 0) atomicMin(avail_ns, now_ns());
 
   // (a) rank inside the block: warp-aggregated shared-memory atomics
   const int a = threadIdx.x;
@@ -290,7 +319,7 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
   }
   __syncthreads();
   copy_rows<4>(x, recv, s_slot, t0, ntok, K, vec_per_row);
-  if (tile_count != nullptr) signal_rows(s_slot, na, tile_count, rows_done);
+  if (tile_count != nullptr) signal_rows(s_slot, na, tile_count, rows_done, avail_ns, T * K);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -299,7 +328,7 @@ __global__ void __launch_bounds__(kDispThreads)
 reset_kernel(int* __restrict__ counters, int n_counters, int* __restrict__ expert_count, int E,
              int* __restrict__ tile_expert, int P, int* __restrict__ src_info, int n_src,
              int* __restrict__ tile_table, int n_table, int* __restrict__ tile_count,
-             int* __restrict__ rows_done, int* __restrict__ gemm1_done) {
+             int* __restrict__ rows_done, int* __restrict__ gemm1_done, unsigned long long* __restrict__ avail_ns) {
   const int stride = gridDim.x * kDispThreads;
   const int i0 = blockIdx.x * kDispThreads + threadIdx.x;
   pdl_wait();
@@ -307,6 +336,8 @@ reset_kernel(int* __restrict__ counters, int n_counters, int* __restrict__ exper
   for (int i = i0; i < n_counters; i += stride) counters[i] = 0;
   if (i0 == 0) *rows_done = 0;
   if (i0 < 4) gemm1_done[P + i0] = 0;  // the expert kernel's item and exit counters
+  if (avail_ns != nullptr)
+    for (int i = i0; i < P + 2; i += stride) avail_ns[i] = i == 0 ? ~0ull : 0ull;
   for (int i = i0; i < E; i += stride) expert_count[i] = 0;
   for (int i = i0; i < P; i += stride) {
     tile_expert[i] = -1;
@@ -332,19 +363,20 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
     const int grid = (int)max(1ll, (most + 4 * kDispThreads - 1) / (4 * kDispThreads));
     launch_pdl(reset_kernel, dim3(grid), dim3(kDispThreads), 0, st, p->s.status,
                (int)(p->counters_bytes / sizeof(int)), expert_count, c.E, tile_expert, (int)p->P, src_info,
-               (int)(p->P * kTileRows), p->s.tile_table, table, tile_count, rows_done, p->s.gemm1_done);
+               (int)(p->P * kTileRows), p->s.tile_table, table, tile_count, rows_done, p->s.gemm1_done, p->trace ? p->s.avail_ns : nullptr);
     p->launches += 1;
   }
   if (c.T == 0) return 0;
   const int nblk = p->nblk, tpb = p->dispatch_tokens;
   if (c.dispatch_mode == MOE_DISPATCH_SCAN) {
     launch_maybe_pdl(false, hist_kernel, dim3(nblk), dim3(kDispThreads), sizeof(int) * c.E, st, topk_idx, c.T, c.E, c.K, tpb,
-               p->s.cta_count);
+               p->s.cta_count, p->trace ? p->s.avail_ns : nullptr);
     launch_maybe_pdl(false, scan_kernel, dim3(c.E), dim3(kDispThreads), 0, st, p->s.cta_count, nblk, c.E, (int)p->P, p->s.cta_base,
                expert_count, p->s.tile_base, tile_expert, p->s.scan_ticket);
     const size_t smem = sizeof(int) * ((kDispThreads / 32) * c.E + kMaxAssign);
     launch_maybe_pdl(false, scatter_kernel, dim3(nblk), dim3(kDispThreads), smem, st, (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb,
-               vec_per_row, p->s.cta_base, p->s.tile_base, (uint4*)recv, src_info, slot_of, tile_count, rows_done);
+               vec_per_row, p->s.cta_base, p->s.tile_base, (uint4*)recv, src_info, slot_of, tile_count, rows_done,
+               p->trace ? p->s.avail_ns : nullptr);
     p->launches += 3;
   } else {
     const size_t smem = sizeof(int) * (2 * c.E + kMaxAssign);
@@ -352,7 +384,8 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
     auto kern = c.dispatch_mode == MOE_DISPATCH_ATOMIC_PAGED ? dispatch_atomic_kernel<true> : dispatch_atomic_kernel<false>;
     launch_pdl(kern, dim3(nblk), dim3(kDispThreads), smem, st, (const uint4*)x, topk_idx, c.T, c.E, c.K, tpb, vec_per_row,
                (int)p->cap_rows, (int)p->P, p->tiles_per_expert, spin, expert_count, p->s.tile_table, p->s.pool_next,
-               tile_expert, (uint4*)recv, src_info, slot_of, p->s.status, tile_count, rows_done);
+               tile_expert, (uint4*)recv, src_info, slot_of, p->s.status, tile_count, rows_done,
+               p->trace ? p->s.avail_ns : nullptr);
     p->launches += 1;
   }
   return (int)cudaGetLastError();
@@ -444,6 +477,6 @@ extern "C" int moe_dispatch_noalloc(const moe_config_t* cfg, const void* d_x, co
   dispatch_atomic_kernel<true><<<nblk, kDispThreads, smem, st>>>(
       (const uint4*)d_x, d_topk_idx, c.T, c.E, c.K, tpb, c.H * eb / 16, 0, (int)P, tiles_per_expert, spin,
       d_expert_count, tile_table, pool_next, d_tile_expert, (uint4*)d_recv, d_src_info, d_slot_of, d_status,
-      nullptr, nullptr);
+      nullptr, nullptr, nullptr);
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
 }

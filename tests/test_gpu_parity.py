@@ -296,6 +296,37 @@ def test_dispatch_availability_counters_and_gated_consumer(mode):
     Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
 
 
+@pytest.mark.parametrize("mode", MODES)
+def test_availability_trace_orders_the_events(mode):
+    """With the trace on, every tile that holds 128 rows has a ready time between the dispatch start and
+    the all-ready time, tiles with fewer rows have none, and the layer's result is unchanged."""
+    w = inputs.Workload("trace", T=900, H=264, E=12, R=3, K=3, F=136, dtype=BF16, zipf_s=1.0, seed=9)
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    plan = Hh.make_plan(w, mode)
+    y0 = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
+    plan.moe_layer(*args, y0)
+    plan.moe_availability_trace(True)
+    y1 = torch.empty_like(y0)
+    plan.moe_layer(*args, y1)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    tr = plan.layer_tensor(8).cpu().numpy()
+    cnt = plan.layer_tensor(3).cpu().numpy()
+    te = plan.layer_tensor(4).cpu().numpy()
+    slot = plan.layer_tensor(6).cpu().numpy()
+    per_tile = np.bincount(slot.ravel() // 128, minlength=plan.P)
+    t0, t_all, ready = tr[0], tr[1], tr[2:]
+    assert t0 > 0 and t_all >= t0
+    full = per_tile == 128
+    assert full.any() and (~full & (te >= 0)).any()
+    assert (ready[full] >= t0).all() and (ready[full] <= t_all).all()
+    assert (ready[~full] == 0).all()
+    assert cnt.sum() == w.T * w.K
+    assert torch.equal(y0, y1)
+    plan.moe_availability_trace(False)
+
+
 @pytest.mark.parametrize("split", [1, 2])
 def test_expert_kernel_can_be_called_again_without_a_dispatch_in_between(split):
     """The expert kernel hands its items out through device counters and puts them back to zero itself:
