@@ -206,7 +206,7 @@ def run_cuda(args, w: inputs.Workload) -> None:
     mode = {"scan": B.DISPATCH_SCAN, "static": B.DISPATCH_ATOMIC_STATIC, "paged": B.DISPATCH_ATOMIC_PAGED}[args.dispatch]
     plan = B.Plan(B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype, dispatch_mode=mode,
                                 identity_experts=int(w.identity_experts), ffn_split=int(args.ffn_split),
-                                ffn_kernel=args.ffn_kernel))
+                                ffn_kernel=args.ffn_kernel, ffn_hot_min_tiles=args.ffn_hot_min_tiles, ffn_thin_tiles=args.ffn_thin_tiles))
     y = torch.empty((w.T, w.H), dtype=el, device="cuda")
     stream = torch.cuda.current_stream()
 
@@ -407,6 +407,10 @@ def main() -> None:
                     help="0: tcgen05 one CTA per tile (default), 2: tcgen05 CTA pairs, 1: SIMT check path")
     ap.add_argument("--ffn-split", type=int, default=0, choices=[0, 1, 2],
                     help="expert GEMMs: 1 = one launch each, 2 = one launch for both, 0 = library default")
+    ap.add_argument("--ffn-hot-min-tiles", type=int, default=0,
+                    help="two-launch expert GEMMs: experts with at least this many tiles are walked as tensor-bound "
+                         "work, interleaved with the weight-streaming-bound rest (0: library default, -1: off)")
+    ap.add_argument("--ffn-thin-tiles", type=int, default=0, help="-1: no transposed narrow form for small single tiles")
     args = ap.parse_args()
     w = WORKLOADS[args.workload]
     if args.impl == "reference":

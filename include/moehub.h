@@ -15,7 +15,9 @@
  * General rules
  *  - Every pointer named d_* is DEVICE memory owned by the caller; h_* is HOST memory.  The
  *    library allocates no device memory: its scratch is the caller's workspace (see
- *    moe_workspace_bytes / moe_plan_create).  A plan owns host-side metadata only.
+ *    moe_workspace_bytes / moe_plan_create).  A plan owns host-side metadata only.  The one
+ *    exception to this rule and to "no global state" below is moe_dispatch_noalloc, which keeps
+ *    its scratch in a device array that is part of the library image (see its declaration).
  *  - dtype 0: fp32, dtype 1: bf16.  It is the type of x, the router weight, the expert
  *    weights, the receive buffers, the expert outputs and y.  Routing weights are fp32,
  *    indices int32.  All matrices are row-major and dense.
@@ -23,8 +25,9 @@
  *    16-byte aligned (cudaMalloc / torch allocations are).
  *  - Calls are asynchronous on `stream` (a cudaStream_t passed as void*, NULL = default
  *    stream).  Return value: 0 = MOE_OK, negative = error found on the host before anything
- *    was launched.  Errors found on the device (region overflow, a bounded wait that ran out)
- *    are left in a device status word: read it with moe_last_status.
+ *    was launched.  Errors found on the device (region overflow, a bounded wait that ran out,
+ *    an expert id outside [0, E) in a caller-supplied topk_idx) are left in a device status
+ *    word: read it with moe_last_status.
  *  - A plan is used by one host thread / one stream at a time.  No global state.
  *  - Receive-buffer geometry: rows live in a pool of P tiles of 128 rows
  *    (moe_pool_tiles).  tile_expert[p] names the expert that owns tile p (-1: unused).  An
@@ -78,6 +81,15 @@ typedef struct {
                                    launch (per-tile status counters gate GEMM2); 0: choose
                                    (one launch when E <= 64; with more, smaller experts two
                                    launches measure faster)                                   */
+  int32_t ffn_hot_min_tiles;    /* two-launch form of the tensor-core kernel: > 0 = experts with at
+                                   least this many tiles count as tensor-bound, the others as
+                                   bound by streaming their weights, and the kernel walks the two
+                                   kinds of work interleaved; 0 (default) = one expert after the
+                                   other                                                       */
+  int32_t ffn_thin_tiles;       /* tensor-core kernel: 0 = an expert's only tile, if it holds at
+                                   most 64 rows, is computed in the transposed narrow form;
+                                   negative = never (such a tile runs M = 64 MMAs instead)      */
+  int32_t reserved_[2];         /* must be 0                                                  */
   int64_t capacity_rows;        /* mode 1: rows per expert region, multiple of 128, 0 = T
                                    rounded up (overflow-free); modes 0/2: ignored            */
   uint64_t spin_limit;          /* bound (iterations) on the dispatch kernels' waits, 0 = 1<<22 */
@@ -115,7 +127,9 @@ int moe_route(moe_plan_t* plan, const void* d_x, const void* d_wr, const float* 
  *      d_expert_count [E] rows per expert, d_tile_expert [P] owner of each tile or -1,
  *      d_src_info [P*128] = t*K+k of the row in that slot, -1 for an empty slot (the source
  *      information of Section IV-B, combine), d_slot_of [T,K] physical row of assignment
- *      (t,k), or -1 if it was dropped by an overflow (status MOE_ERR_OVERFLOW);
+ *      (t,k), or -1 if it was dropped by an overflow (status MOE_ERR_OVERFLOW) or because
+ *      topk_idx[t,k] is not in [0, E) (status MOE_ERR_ARG, detail = the token; no table is
+ *      indexed with such an id and the assignment's row is not stored);
  *      availability counters (Section IV-D, data availability manager), both or neither,
  *      NULL = kept in the plan's workspace: d_tile_count [P] rows stored so far in each tile,
  *      d_rows_done [1] assignments whose rows are stored; both raised with release semantics
@@ -125,7 +139,7 @@ int moe_dispatch(moe_plan_t* plan, const void* d_x, const int32_t* d_topk_idx, v
                  int32_t* d_expert_count, int32_t* d_tile_expert, int32_t* d_src_info,
                  int32_t* d_slot_of, int32_t* d_tile_count, int32_t* d_rows_done, void* stream);
 
-/* Step 3 (Section II-A, expert computation; "two GEMMs with an activation between", here
+/* Step 3 (Section II-A, expert computation: two GEMMs with an activation between them, here
  * SwiGLU): for every used tile p of expert e = tile_expert[p]:
  *   S = silu(A*Wg[e]^T) .* (A*Wu[e]^T),  O = S*Wd[e]^T,  A = the tile's 128 rows of d_recv.
  * Unused tiles are skipped and their experts' weights never read (Section IV-D: thread
@@ -163,7 +177,10 @@ int moe_expert_ffn(moe_plan_t* plan, const void* d_recv, const int32_t* d_tile_e
  * receives the device status (code, detail) that moe_last_status would report.
  *
  * The first call on each device looks up the array's device address (that device must be
- * current); make that first call outside any stream capture.  All calls on a device share the
+ * current); make that first call outside any stream capture.  With the CUDA runtime's lazy module
+ * loading, that first call (or the first kernel of this library on the device) is also when the
+ * driver loads the library's device image and places the array, so "allocates nothing" holds from
+ * the second call on: issue one warm-up call at start-up, while allocation is still permitted.  All calls on a device share the
  * one array, which still holds the previous call's contents: each call clears what it needs on
  * `stream` before its kernel, so calls issued to the same stream are safe back to back, but two
  * calls that can overlap on the GPU (different streams, no dependency) race on it. */
@@ -221,7 +238,8 @@ int moe_layer_timed(moe_plan_t* plan, const void* d_x, const void* d_wr, const f
 
 /* Device pointers of moe_layer's intermediate results inside the workspace (valid after a
  * moe_layer call completes): which = 0 topk_idx, 1 topk_w, 2 recv, 3 expert_count,
- * 4 tile_expert, 5 src_info, 6 slot_of, 7 out_rows, 8 the availability trace (below). */
+ * 4 tile_expert, 5 src_info, 6 slot_of, 7 out_rows, 8 the availability trace, 9 the work-item
+ * timeline (both below). */
 int moe_layer_buffer(moe_plan_t* plan, int which, void** out_ptr);
 
 /* Availability trace (Section IV-D: when does a consumer learn that a tile is ready), for
@@ -230,7 +248,15 @@ int moe_layer_buffer(moe_plan_t* plan, int which, void** out_ptr);
  * uint64 array [P + 2] in the workspace (moe_layer_buffer, which = 8): [0] the earliest start of a
  * dispatch CTA, [1] the moment the global counter reached all T*K assignments, [2 + p] the moment
  * tile p's counter reached 128 rows (0: the tile never filled).  Disabled (the default) the kernels
- * are unchanged.  The flag is host-side state of the plan. */
+ * are unchanged.  The flag is host-side state of the plan.
+ * While enabled, the tensor-core expert kernel (one CTA per tile, bf16) also writes a timeline of its
+ * work items: uint64 [P * (ceil(F/128) + ceil(H/256))][4] (moe_layer_buffer, which = 9), one entry
+ * per position of its item list in the order the items were claimed: [0] the moment the item's
+ * producer had seen its tile ready and began to load, [1] the moment its MMAs were complete, [2] what
+ * it was (bit 0: 0 = GEMM1 block, 1 = GEMM2 block; bit 1: an expert bound by streaming its weights;
+ * bits 2-5 the narrow form used; bits 8-23 expert, 24-31 column block, 32-51 tile, 52-63 SM),
+ * [3] the moment its last load was issued.  Entries of positions that were not claimed keep their
+ * old contents. */
 int moe_availability_trace(moe_plan_t* plan, int enable);
 
 /* Effective SM clock inside the tensor-core expert kernels since the last reset: one CTA of every
@@ -242,9 +268,9 @@ int moe_ffn_clock_mhz(moe_plan_t* plan, void* stream, int reset, float* out_mhz)
 /* Number of kernels the last stage call (or moe_layer) launched. */
 int moe_last_launch_count(moe_plan_t* plan, int32_t* out);
 
-/* Synchronises `stream` and reads the device status word: *code is MOE_OK, MOE_ERR_OVERFLOW
- * or MOE_ERR_TIMEOUT; *detail says where (expert id for an overflow, wait site for a
- * timeout). */
+/* Synchronises `stream` and reads the device status word: *code is MOE_OK, MOE_ERR_OVERFLOW,
+ * MOE_ERR_TIMEOUT or MOE_ERR_ARG; *detail says where (expert id for an overflow, wait site for
+ * a timeout, token index for an expert id outside [0, E)).  The first error of a call wins. */
 int moe_last_status(moe_plan_t* plan, void* stream, int32_t* code, int32_t* detail);
 
 const char* moe_strerror(int code);

@@ -108,8 +108,18 @@ def dispatch(x, topk_idx, E, R, dtype, want_rows=True):
     return dict(count=count, offset=offset, rank_count=rank_count, recv=recv, src=src, slot_of=slot_of)
 
 
-def expert_ffn(recv, offset, wg, wu, wd, dtype):
+def round_bf16(a):
+    """Nearest bf16 value (ties to even) of every element of an fp64 array, as fp64."""
+    a = np.ascontiguousarray(a, np.float64)
+    f = lib().oracle_round_bf16
+    f.restype, f.argtypes = ctypes.c_double, [ctypes.c_double]
+    return np.array([f(float(v)) for v in a.ravel()], np.float64).reshape(a.shape)
+
+
+def expert_ffn(recv, offset, wg, wu, wd, dtype, bf16_storage=False):
     """wg/wu/wd: sequences of E per-expert arrays ([F,H],[F,H],[H,F]); None allowed for empty experts.
+    bf16_storage: the diagnostic restatement that rounds the SwiGLU intermediate and the output rows to
+    bf16 (what the CUDA path stores), sums still in fp64.
 
     Returns out[rows,H] fp64."""
     rows, H = recv.shape
@@ -131,8 +141,8 @@ def expert_ffn(recv, offset, wg, wu, wd, dtype):
         return arr
 
     out = np.empty((rows, H), np.float64)
-    _check(lib().oracle_expert_ffn(H, F, E, dtype, _p(recv), _p(offset), ptrs(wg), ptrs(wu), ptrs(wd),
-                                   _p(out)), "oracle_expert_ffn")
+    fn = lib().oracle_expert_ffn_stored if bf16_storage else lib().oracle_expert_ffn
+    _check(fn(H, F, E, dtype, _p(recv), _p(offset), ptrs(wg), ptrs(wu), ptrs(wd), _p(out)), "oracle_expert_ffn")
     return out
 
 
@@ -146,24 +156,27 @@ def identity_ffn(recv, dtype):
     return out
 
 
-def combine(rows, slot_of, topk_w):
+def combine(rows, slot_of, topk_w, bf16_storage=False):
+    """bf16_storage: the diagnostic restatement that rounds y to bf16."""
     rows = np.ascontiguousarray(rows, np.float64)
     T, K = slot_of.shape
     H = rows.shape[1]
     slot_of = np.ascontiguousarray(slot_of, np.int32)
     topk_w = np.ascontiguousarray(topk_w, np.float32)
     y = np.empty((T, H), np.float64)
-    _check(lib().oracle_combine(T, H, K, _p(rows), _p(slot_of), _p(topk_w), _p(y)), "oracle_combine")
+    fn = lib().oracle_combine_stored if bf16_storage else lib().oracle_combine
+    _check(fn(T, H, K, _p(rows), _p(slot_of), _p(topk_w), _p(y)), "oracle_combine")
     return y
 
 
-def layer(x, wr, bias, wg, wu, wd, E, R, K, dtype, renormalize=0, identity_experts=False):
-    """The whole layer: route -> dispatch -> experts -> combine. Returns dict with every stage's output."""
+def layer(x, wr, bias, wg, wu, wd, E, R, K, dtype, renormalize=0, identity_experts=False, bf16_storage=False):
+    """The whole layer: route -> dispatch -> experts -> combine. Returns dict with every stage's output.
+    bf16_storage: the diagnostic restatement (intermediate, expert rows and y rounded to bf16)."""
     idx, w, lg = route(x, wr, bias, K, dtype, renormalize)
     d = dispatch(x, idx, E, R, dtype)
     if identity_experts:
         rows = identity_ffn(d["recv"], dtype)
     else:
-        rows = expert_ffn(d["recv"], d["offset"], wg, wu, wd, dtype)
-    y = combine(rows, d["slot_of"], w)
+        rows = expert_ffn(d["recv"], d["offset"], wg, wu, wd, dtype, bf16_storage=bf16_storage)
+    y = combine(rows, d["slot_of"], w, bf16_storage=bf16_storage)
     return dict(topk_idx=idx, topk_w=w, logits=lg, out_rows=rows, y=y, **d)

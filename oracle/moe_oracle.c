@@ -23,6 +23,13 @@
  * ascending, starting from 0.  Everything else (softmax weights, FFN, combine) is fp64.
  * bf16 inputs are widened exactly.
  *
+ * Diagnostic mode (bf16 storage).  The CUDA path keeps three tensors in bf16: the SwiGLU
+ * intermediate, the expert output rows and y.  oracle_expert_ffn_stored and oracle_combine_stored
+ * restate steps 3-5 with exactly those three values rounded to bf16 (nearest, ties to even) and
+ * every sum still in fp64: the best any implementation with bf16 storage can do.  The distance
+ * between this restatement and the exact functions is the rounding a tolerance has to leave room
+ * for; the distance between the CUDA path and this restatement is what the kernels add to it.
+ *
  * Every function is pinned by tests that do not go through this file (brute force, closed
  * forms, invariants, library routines); see tests/test_oracle_*.py.
  *
@@ -47,6 +54,21 @@ static inline float widen(const void *base, int dtype, int64_t i) {
 }
 
 static inline size_t elem_bytes(int dtype) { return dtype == ORACLE_FP32 ? 4 : 2; }
+
+/*
+ * Nearest bf16 value of a double (ties to even), returned as a double.  bf16 keeps 8 significant
+ * bits, a double 53: round away the low 45 bits of the significand.  Finite inputs in bf16's
+ * normal range only (everything this file feeds it is); zero stays zero.
+ */
+double oracle_round_bf16(double v) {
+  uint64_t b;
+  memcpy(&b, &v, sizeof b);
+  const uint64_t lsb = (b >> 45) & 1u;
+  b += ((uint64_t)1 << 44) - 1 + lsb;
+  b &= ~(((uint64_t)1 << 45) - 1);
+  memcpy(&v, &b, sizeof v);
+  return v;
+}
 
 int oracle_num_threads(void) {
 #ifdef _OPENMP
@@ -175,9 +197,9 @@ int oracle_dispatch(int T, int H, int E, int R, int K, int dtype, const void *x,
  * [H,F] matrices (an expert without rows may have NULL pointers: its weights are never read).
  * out: [rows,H] fp64.
  */
-int oracle_expert_ffn(int H, int F, int E, int dtype, const void *recv, const int32_t *offset,
-                      const void *const *wg, const void *const *wu, const void *const *wd,
-                      double *out) {
+static int expert_ffn_impl(int H, int F, int E, int dtype, const void *recv, const int32_t *offset,
+                           const void *const *wg, const void *const *wu, const void *const *wd,
+                           double *out, int stored) {
   if (H <= 0 || F <= 0 || E <= 0) return -1;
   for (int e = 0; e < E; ++e) {
     const int r0 = offset[e], r1 = offset[e + 1];
@@ -195,11 +217,12 @@ int oracle_expert_ffn(int H, int F, int E, int dtype, const void *recv, const in
           for (int h = 0; h < H; ++h) g += a[h] * (double)widen(wg[e], dtype, (int64_t)f * H + h);
           for (int h = 0; h < H; ++h) u += a[h] * (double)widen(wu[e], dtype, (int64_t)f * H + h);
           s[f] = g / (1.0 + exp(-g)) * u;
+          if (stored) s[f] = oracle_round_bf16(s[f]); /* the intermediate is kept in bf16 */
         }
         for (int j = 0; j < H; ++j) {
           double o = 0.0;
           for (int f = 0; f < F; ++f) o += s[f] * (double)widen(wd[e], dtype, (int64_t)j * F + f);
-          out[(int64_t)r * H + j] = o;
+          out[(int64_t)r * H + j] = stored ? oracle_round_bf16(o) : o; /* expert output rows in bf16 */
         }
       }
       free(a);
@@ -207,6 +230,19 @@ int oracle_expert_ffn(int H, int F, int E, int dtype, const void *recv, const in
     }
   }
   return 0;
+}
+
+int oracle_expert_ffn(int H, int F, int E, int dtype, const void *recv, const int32_t *offset,
+                      const void *const *wg, const void *const *wu, const void *const *wd,
+                      double *out) {
+  return expert_ffn_impl(H, F, E, dtype, recv, offset, wg, wu, wd, out, 0);
+}
+
+/* Diagnostic mode: step 3 with the intermediate and the output rows rounded to bf16 (see the header). */
+int oracle_expert_ffn_stored(int H, int F, int E, int dtype, const void *recv, const int32_t *offset,
+                             const void *const *wg, const void *const *wu, const void *const *wd,
+                             double *out) {
+  return expert_ffn_impl(H, F, E, dtype, recv, offset, wg, wu, wd, out, 1);
 }
 
 /* Identity experts: o = a (used by the dispatch/combine-only sweep). out: [rows,H] fp64. */
@@ -221,8 +257,8 @@ int oracle_identity_ffn(int64_t rows, int H, int dtype, const void *recv, double
  * Steps 4+5, combine and scaling: y[t,j] = sum_{k ascending} w[t,k] * rows[slot_of[t,k], j].
  * rows: [*,H] fp64, y: [T,H] fp64.
  */
-int oracle_combine(int T, int H, int K, const double *rows, const int32_t *slot_of,
-                   const float *topk_w, double *y) {
+static int combine_impl(int T, int H, int K, const double *rows, const int32_t *slot_of,
+                        const float *topk_w, double *y, int stored) {
   if (T < 0 || H <= 0 || K <= 0) return -1;
 #pragma omp parallel for schedule(static)
   for (int t = 0; t < T; ++t) {
@@ -230,8 +266,19 @@ int oracle_combine(int T, int H, int K, const double *rows, const int32_t *slot_
       double acc = 0.0;
       for (int k = 0; k < K; ++k)
         acc += (double)topk_w[(int64_t)t * K + k] * rows[(int64_t)slot_of[(int64_t)t * K + k] * H + j];
-      y[(int64_t)t * H + j] = acc;
+      y[(int64_t)t * H + j] = stored ? oracle_round_bf16(acc) : acc;
     }
   }
   return 0;
+}
+
+int oracle_combine(int T, int H, int K, const double *rows, const int32_t *slot_of,
+                   const float *topk_w, double *y) {
+  return combine_impl(T, H, K, rows, slot_of, topk_w, y, 0);
+}
+
+/* Diagnostic mode: steps 4+5 with y rounded to bf16 (see the header). */
+int oracle_combine_stored(int T, int H, int K, const double *rows, const int32_t *slot_of,
+                          const float *topk_w, double *y) {
+  return combine_impl(T, H, K, rows, slot_of, topk_w, y, 1);
 }

@@ -32,6 +32,8 @@ class MoeConfig(ctypes.Structure):
                 ("K", ctypes.c_int32), ("F", ctypes.c_int32), ("dtype", ctypes.c_int32),
                 ("renormalize", ctypes.c_int32), ("dispatch_mode", ctypes.c_int32),
                 ("identity_experts", ctypes.c_int32), ("ffn_kernel", ctypes.c_int32), ("ffn_split", ctypes.c_int32),
+                ("ffn_hot_min_tiles", ctypes.c_int32), ("ffn_thin_tiles", ctypes.c_int32),
+                ("reserved_", ctypes.c_int32 * 2),
                 ("capacity_rows", ctypes.c_int64), ("spin_limit", ctypes.c_uint64), ("wait_limit_ns", ctypes.c_uint64)]
 
 
@@ -103,9 +105,10 @@ def _stream(stream) -> int:
 
 
 def make_config(T, H, E, R, K, F, dtype, renormalize=0, dispatch_mode=DISPATCH_ATOMIC_PAGED, identity_experts=0,
-                ffn_kernel=0, capacity_rows=0, spin_limit=0, ffn_split=0, wait_limit_ns=0) -> MoeConfig:
+                ffn_kernel=0, capacity_rows=0, spin_limit=0, ffn_split=0, wait_limit_ns=0,
+                ffn_hot_min_tiles=0, ffn_thin_tiles=0) -> MoeConfig:
     return MoeConfig(T, H, E, R, K, F, dtype, int(renormalize), dispatch_mode, int(identity_experts), ffn_kernel, int(ffn_split),
-                     capacity_rows, spin_limit, wait_limit_ns)
+                     int(ffn_hot_min_tiles), int(ffn_thin_tiles), (ctypes.c_int32 * 2)(0, 0), capacity_rows, spin_limit, wait_limit_ns)
 
 
 def moe_pool_tiles(cfg: MoeConfig) -> int:
@@ -234,7 +237,8 @@ class Plan:
         el = torch.bfloat16 if c.dtype == DTYPE_BF16 else torch.float32
         shapes = {0: ((c.T, c.K), torch.int32), 1: ((c.T, c.K), torch.float32), 2: ((rows, c.H), el),
                   3: ((c.E,), torch.int32), 4: ((self.P,), torch.int32), 5: ((rows,), torch.int32),
-                  6: ((c.T, c.K), torch.int32), 7: ((rows, c.H), el), 8: ((self.P + 2,), torch.int64)}
+                  6: ((c.T, c.K), torch.int32), 7: ((rows, c.H), el), 8: ((self.P + 2,), torch.int64),
+                  9: ((self.P * ((c.F + 127) // 128 + (c.H + 255) // 256), 4), torch.int64)}
         shape, dt = shapes[which]
         ptr = self.moe_layer_buffer(which)
         off = ptr - self.workspace.data_ptr()

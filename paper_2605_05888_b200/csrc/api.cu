@@ -76,6 +76,10 @@ size_t carve(const moe_config_t& c, const Geometry& g, char* base, Scratch* s, s
   t.tile_base = (int*)take(sizeof(int) * (size_t)(c.E + 1));
   t.clock_probe = (unsigned long long*)take(sizeof(unsigned long long) * 2);
   t.avail_ns = (unsigned long long*)take(sizeof(unsigned long long) * (size_t)((g.P > 0 ? g.P : 1) + 2));
+  if (!c.identity_experts && c.dtype == MOE_DTYPE_BF16) {
+    const size_t items = (size_t)(g.P > 0 ? g.P : 1) * ((c.F + 127) / 128 + (c.H + 255) / 256);
+    t.item_ns = (unsigned long long*)take(sizeof(unsigned long long) * 4 * items);
+  }
   t.gemm1_done = (int*)take(sizeof(int) * (size_t)((g.P > 0 ? g.P : 1) + 4));  // + the expert kernel's item and exit counters
   const size_t pool_rows = (size_t)g.P * kTileRows;
   if (!c.identity_experts) t.inter = take(pool_rows * c.F * g.eb);
@@ -335,9 +339,9 @@ int moe_layer_host_wait(moe_plan_t* p, int64_t ticket) {
 int moe_layer_buffer(moe_plan_t* p, int which, void** out_ptr) {
   if (!p || !out_ptr) return MOE_ERR_ARG;
   Scratch& s = p->s;
-  void* tab[9] = {s.topk_idx, s.topk_w, s.recv, s.expert_count, s.tile_expert, s.src_info, s.slot_of, s.out_rows,
-                  s.avail_ns};
-  if (which < 0 || which >= 9) return MOE_ERR_ARG;
+  void* tab[10] = {s.topk_idx, s.topk_w, s.recv, s.expert_count, s.tile_expert, s.src_info, s.slot_of, s.out_rows,
+                   s.avail_ns, s.item_ns};
+  if (which < 0 || which >= 10) return MOE_ERR_ARG;
   *out_ptr = tab[which];
   return MOE_OK;
 }

@@ -32,6 +32,7 @@ struct Scratch {          // device pointers carved out of the caller's workspac
   int* tile_base;         // [E + 1]    mode 0: first pool tile of each expert
   unsigned long long* clock_probe;  // [2] cycles, nanoseconds of CTA 0 inside the tensor-core kernels
   unsigned long long* avail_ns;  // [P+2] availability trace (measurement): dispatch start, all-ready time, per-tile ready time
+  unsigned long long* item_ns;   // [4 * P * (NB1 + NB2)] work-item timeline of the tensor-core expert kernel (measurement)
   int* gemm1_done;        // [P+4]  per-tile status counter: GEMM1 blocks finished (x4 epilogue warps); [P..P+1] item counters, [P+2..P+3] exit counters of the expert kernel's launches
   void* inter;            // [P*128, F] SwiGLU intermediate
   // moe_layer's internal buffers
@@ -98,6 +99,20 @@ template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
                               Args&&... args) {
   return launch_maybe_pdl(true, kern, grid, block, smem, st, static_cast<Args&&>(args)...);
+}
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) applies to the CURRENT device only, so the "already
+// set" flag of a kernel is kept per device (a process may hold plans on several GPUs).  Setting it twice
+// is harmless, so concurrent first calls need no lock.
+struct SmemAttrOnce {
+  bool done[64] = {};
+};
+template <typename Kern>
+inline cudaError_t ensure_dynamic_smem(Kern kern, size_t bytes, int device, SmemAttrOnce& once) {
+  if (device >= 0 && device < 64 && once.done[device]) return cudaSuccess;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess && device >= 0 && device < 64) once.done[device] = true;
+  return e;
 }
 
 // ---- launchers (defined in the other .cu files); each returns a cudaError_t as int ------------

@@ -106,7 +106,7 @@ __device__ __forceinline__ void signal_rows(const int* s_slot, int na, int* __re
 // Mode 0, kernel 1: histogram of one token block.  cta_count[blk][e].
 __global__ void __launch_bounds__(kDispThreads)
 hist_kernel(const int* __restrict__ topk_idx, int T, int E, int K, int tok_per_blk,
-            int* __restrict__ cta_count, unsigned long long* __restrict__ avail_ns) {
+            int* __restrict__ cta_count, int* __restrict__ status, unsigned long long* __restrict__ avail_ns) {
   extern __shared__ int s_cnt[];  // [E]
   for (int e = threadIdx.x; e < E; e += kDispThreads) s_cnt[e] = 0;
   __syncthreads();
@@ -115,7 +115,11 @@ hist_kernel(const int* __restrict__ topk_idx, int T, int E, int K, int tok_per_b
   if (avail_ns != nullptr && threadIdx.x == 0) atomicMin(avail_ns, now_ns());
   const int t0 = blockIdx.x * tok_per_blk;
   const int na = min(tok_per_blk, T - t0) * K;
-  for (int a = threadIdx.x; a < na; a += kDispThreads) atomicAdd(&s_cnt[topk_idx[(size_t)t0 * K + a]], 1);
+  for (int a = threadIdx.x; a < na; a += kDispThreads) {
+    const int e = topk_idx[(size_t)t0 * K + a];
+    if (e >= 0 && e < E) atomicAdd(&s_cnt[e], 1);
+    else set_status(status, MOE_ERR_ARG, t0 + a / K);  // an expert id outside [0, E): the assignment is dropped
+  }
   __syncthreads();
   for (int e = threadIdx.x; e < E; e += kDispThreads) cta_count[(size_t)blockIdx.x * E + e] = s_cnt[e];
 }
@@ -208,6 +212,7 @@ scatter_kernel(const uint4* __restrict__ x, const int* __restrict__ topk_idx, in
   const int a = threadIdx.x;  // one assignment per thread, na <= 256
   int e = -1, wrank = 0;
   if (a < na) e = topk_idx[(size_t)t0 * K + a];
+  if (e >= E) e = -1;  // reported by the histogram kernel; dropped here
   {
     const unsigned peers = __match_any_sync(0xffffffffu, e);
     wrank = __popc(peers & ((1u << lane) - 1u));
@@ -215,12 +220,15 @@ scatter_kernel(const uint4* __restrict__ x, const int* __restrict__ topk_idx, in
   }
   __syncthreads();
   if (a < na) {
-    int before = 0;
-    for (int w = 0; w < warp; ++w) before += s_wcnt[w * E + e];
-    const int slot = tile_base[e] * kTileRows + cta_base[(size_t)blockIdx.x * E + e] + before + wrank;
+    int slot = -1;
+    if (e >= 0) {
+      int before = 0;
+      for (int w = 0; w < warp; ++w) before += s_wcnt[w * E + e];
+      slot = tile_base[e] * kTileRows + cta_base[(size_t)blockIdx.x * E + e] + before + wrank;
+      src_info[slot] = t0 * K + a;
+    }
     s_slot[a] = slot;
     slot_of[(size_t)t0 * K + a] = slot;
-    src_info[slot] = t0 * K + a;
   }
   __syncthreads();
   copy_rows<4>(x, recv, s_slot, t0, ntok, K, vec_per_row);
@@ -255,7 +263,13 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
   // (a) rank inside the block: warp-aggregated shared-memory atomics
   const int a = threadIdx.x;
   int e = -1, lrank = 0;
-  if (a < na) e = topk_idx[(size_t)t0 * K + a];
+  if (a < na) {
+    e = topk_idx[(size_t)t0 * K + a];
+    if (e < 0 || e >= E) {  // not an expert: report it, drop the assignment, touch no table with it
+      set_status(status, MOE_ERR_ARG, t0 + a / K);
+      e = -1;
+    }
+  }
   {
     const unsigned peers = __match_any_sync(0xffffffffu, e);
     const int leader = __ffs(peers) - 1;
@@ -291,16 +305,19 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
 
   // (c) LocalRowID -> physical row (address = Base + LocalRowID*RowSize), staged in shared memory
   if (a < na) {
-    const int local_row = s_base[e] + lrank;
+    const int local_row = e >= 0 ? s_base[e] + lrank : 0;
     int slot = -1;
-    if (PAGED) {
+    if (e < 0) {
+      // dropped above
+    } else if (PAGED) {
       const int lt = local_row / kTileRows;
       if (lt < tiles_per_expert) {
         const int* entry = &tile_table[(size_t)e * tiles_per_expert + lt];
         int tile = ld_acquire(entry);
         unsigned long long spins = 0;
         while (tile < 0) {  // bounded wait for the block that opened this tile
-          if (ld_acquire(status) != 0 || ++spins > spin_limit) {
+          const int seen = ld_acquire(status);  // an overflow means the opener may never publish; a bad id elsewhere does not
+          if ((seen != 0 && seen != MOE_ERR_ARG) || ++spins > spin_limit) {
             set_status(status, MOE_ERR_TIMEOUT, kWaitTileTable);
             break;
           }
@@ -370,7 +387,7 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
   const int nblk = p->nblk, tpb = p->dispatch_tokens;
   if (c.dispatch_mode == MOE_DISPATCH_SCAN) {
     launch_maybe_pdl(false, hist_kernel, dim3(nblk), dim3(kDispThreads), sizeof(int) * c.E, st, topk_idx, c.T, c.E, c.K, tpb,
-               p->s.cta_count, p->trace ? p->s.avail_ns : nullptr);
+               p->s.cta_count, p->s.status, p->trace ? p->s.avail_ns : nullptr);
     launch_maybe_pdl(false, scan_kernel, dim3(c.E), dim3(kDispThreads), 0, st, p->s.cta_count, nblk, c.E, (int)p->P, p->s.cta_base,
                expert_count, p->s.tile_base, tile_expert, p->s.scan_ticket);
     const size_t smem = sizeof(int) * ((kDispThreads / 32) * c.E + kMaxAssign);

@@ -1,12 +1,12 @@
 // Step 3 of the MoE layer (paper Section II-A, expert computation: two GEMMs with an activation
-// between) for bf16 on the 5th-generation tensor cores: a persistent, warp-specialised grouped
+// between them) for bf16 on the 5th-generation tensor cores: a persistent, warp-specialised grouped
 // GEMM.  Operands are staged in shared memory by TMA (128-byte swizzle), tcgen05.mma accumulates
 // 128 x 256 fp32 tiles in tensor memory, and the epilogue warps read them back with tcgen05.ld.
 //
 // The unit of work is what the paper's dependency table calls a thread-block group: one 128-row
 // tile of one expert's receive region times one block of output columns (Section IV-D, static
 // tiling).  Tiles nobody wrote to are not in the work list, so their experts' weights are never
-// touched (the "counters that stay zero are never scheduled" rule of Section IV-D).
+// touched (Section IV-D: thread blocks whose counters stay at zero are never scheduled).
 //
 //   GEMM1 (SWIGLU): D[128, 256] = A[128, H] * [Wg[e, f0:f0+128, :] ; Wu[e, f0:f0+128, :]]^T
 //                   inter[:, f0:f0+128] = bf16( silu(D[:, 0:128]) * D[:, 128:256] )
@@ -36,9 +36,10 @@
 namespace moehub {
 
 // ---- the grouped GEMM -----------------------------------------------------------------------
-// Items are handed out dynamically: every CTA starts with item blockIdx.x and then takes the next
-// unclaimed item of the list (one global atomicAdd per item, issued by the producer thread while the
-// previous item's loads run), so CTAs whose items were short take more of them.  The producer
+// Items are handed out dynamically: a CTA takes the next unclaimed item of the list, its first one
+// included (one global atomicAdd per item, issued by the producer thread while the previous item's
+// loads run), so CTAs whose items were short take more of them, and an item that another one waits
+// for is never held by a CTA that has not started yet.  The producer
 // publishes each item index (-1: no more) to the other roles through a ring in shared memory with one
 // mbarrier per slot.  The producer is at most 4 items (one per pipeline stage) ahead of the MMA
 // thread and that at most 2 (the accumulators) ahead of the epilogue, so 16 slots never wrap onto an
@@ -53,6 +54,7 @@ struct TcShared {
   int item_ring[kItemRing];
   uint32_t tmem_base;
   int abort_flag;
+  int last_cta;
 };
 
 __global__ void __launch_bounds__(kTcThreads, 1)
@@ -94,7 +96,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   pdl_wait();  // everything above needs no global data and overlaps the predecessor's tail
-  build_worklist(wl, prm.tile_expert, prm.P, E, (F + 127) / 128, (H + 255) / 256, prm.lag, prm.fused, 1);
+  int* work_counter = prm.work_counter + (phase == 2 ? 1 : 0);
+  int first_claim = 0;
+  if (threadIdx.x == 0) first_claim = atomicAdd(work_counter, 1);  // in flight while the work list is built
+  build_worklist(wl, prm.tile_expert, prm.P, E, (F + 127) / 128, (H + 255) / 256, prm.lag, prm.fused, 1, prm.hot_min);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -109,13 +114,27 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   if (phase == 1) item_end = wl.n1;
   if (phase == 2) item_begin = wl.n1;
 
+  // Interleaving (two launches, skewed load): the launch's items are two runs, hot then cold (see
+  // WorkList).  Claim number i is spread evenly over both: floor(i * n_cold / n) of the first i claims
+  // are cold ones, so both runs are used up at the same pace and end together.
+  const int n_hot = phase == 0 ? -1 : wl.n_hot[phase - 1];
+  const long long n_cold = (long long)(item_end - item_begin) - n_hot;
+  const long long n_all = item_end - item_begin;
+
   // item -> (type, expert, column block, tile); inside a segment column-block-major, tile-minor
   // Shared-memory reads are slow while the tensor pipe streams its operands from the same memory
   // (a microsecond for the nine dependent reads of a binary search, measured), so only the first
-  // lookup is a search: a thread's items only move forward through the segment list.
-  int seg_cursor = -1;
+  // lookup is a search: a thread's items only move forward through each run of the segment list.
+  int seg_cursor = -1, seg_cursor_cold = -1;
   auto decode = [&](int item) {
-    int lo = seg_cursor;
+    bool cold = false;
+    if (n_hot >= 0 && n_cold > 0) {
+      const long long i = item - item_begin;
+      const long long before = i * n_cold / n_all;
+      cold = (i + 1) * n_cold / n_all > before;
+      item = item_begin + (cold ? n_hot + (int)before : (int)(i - before));
+    }
+    int lo = cold ? seg_cursor_cold : seg_cursor;
     if (lo < 0) {  // largest segment whose first item is <= item
       int hi = nseg;
       lo = 0;
@@ -126,19 +145,18 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     } else {
       while (wl.seg_start[lo + 1] <= item) ++lo;  // seg_start[nseg] is the item count, above every item
     }
-    seg_cursor = lo;
+    if (cold) seg_cursor_cold = lo; else seg_cursor = lo;
     Item it;
     it.type = wl.seg_info[lo] >> 16;
     it.e = wl.seg_info[lo] & 0xffff;
     const int m = wl.estart[it.e + 1] - wl.estart[it.e];
     it.m = m;
+    it.cold = m < prm.cold_below;
     const int local = item - wl.seg_start[lo];
     it.nb = local / m;
     it.tile = wl.tiles[wl.estart[it.e] + local % m];
     return it;
   };
-  const int first_item = item_begin + blockIdx.x;
-  int* work_counter = prm.work_counter + (phase == 2 ? 1 : 0);
   volatile int* item_ring = sh->item_ring;
 
   int fail_site = 0;
@@ -150,7 +168,8 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       int armed[kStages];
 #pragma unroll
       for (int s = 0; s < kStages; ++s) armed[s] = 0;
-      int item = first_item;
+      int item = item_begin + first_claim;
+      const uint64_t pol_stream = l2_policy_evict_first();
       for (int local_item = 0; !fail_site; ++local_item) {
         const int slot = local_item & (kItemRing - 1);
         if (item >= item_end) {
@@ -158,7 +177,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
           mbar_arrive(smem_u32(&sh->item_bar[slot]));
           break;
         }
-        const int next_item = item_begin + (int)gridDim.x + atomicAdd(work_counter, 1);  // used after this item's loads
+        const int next_item = item_begin + atomicAdd(work_counter, 1);  // used after this item's loads
         const Item it = decode(item);
         if (it.type == 0 && tile_count != nullptr) {
           // Availability of this tile's rows (dispatch side): 128 rows stored, or every assignment of
@@ -197,14 +216,23 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
         // its first 64 rows only (M = 64 MMAs, the same count of instructions at half the work each: under the
         // power cap the Phi-like layer and C3 gain 1.5 %).  The row count is final here: the tile was
         // declared ready above (GEMM1) or long ago (GEMM2).
+        unsigned long long* trace = prm.item_ns ? prm.item_ns + 4 * (size_t)item : nullptr;
         int n16 = 0;
         if (tile_count != nullptr) {
           const int r = tile_count[it.tile];
-          if (r <= kThinRows && it.m == 1) n16 = max(1, (r + 15) / 16);
+          if (r <= kThinRows && it.m == 1 && prm.thin) n16 = max(1, (r + 15) / 16);
           else if (r <= kThinRows) n16 = kHalfForm;  // the short last tile of a larger expert: M = 64 MMAs
         }
         item_ring[slot] = item | (n16 << kThinShift);
         mbar_arrive(smem_u32(&sh->item_bar[slot]));  // release: the slot is written before the phase completes
+        if (trace) {
+          unsigned smid;
+          asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+          trace[0] = globaltimer();
+          trace[2] = (unsigned long long)it.type | ((unsigned long long)it.cold << 1) | ((unsigned long long)n16 << 2) |
+                     ((unsigned long long)it.e << 8) | ((unsigned long long)it.nb << 24) |
+                     ((unsigned long long)it.tile << 32) | ((unsigned long long)smid << 52);
+        }
         const CUtensorMap* ma = it.type == 0 ? (n16 ? &map_a1t : &map_a1) : (n16 ? &map_a2t : &map_a2);
         const uint32_t stage_tx = n16 ? (uint32_t)(kThinRows * kBK * 2 + kBBytes) : (uint32_t)kStageBytes;
         const int KB = it.type == 0 ? KB1 : KB2;
@@ -215,7 +243,14 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
           const uint32_t b_dst = a_dst + kABytes;
           mbar_expect_tx(full, stage_tx);
           tma_load_2d(a_dst, ma, full, kb * kBK, it.tile * kTileRows);
-          if (it.type == 0) {
+          if (it.cold) {  // weights that are read this once: first in line for eviction from L2
+            if (it.type == 0) {
+              tma_load_3d_hint(b_dst, &map_bg, full, kb * kBK, it.nb * 128, it.e, pol_stream);
+              tma_load_3d_hint(b_dst + kBBytes / 2, &map_bu, full, kb * kBK, it.nb * 128, it.e, pol_stream);
+            } else {
+              tma_load_3d_hint(b_dst, &map_bd, full, kb * kBK, it.nb * 256, it.e, pol_stream);
+            }
+          } else if (it.type == 0) {
             tma_load_3d(b_dst, &map_bg, full, kb * kBK, it.nb * 128, it.e);
             tma_load_3d(b_dst + kBBytes / 2, &map_bu, full, kb * kBK, it.nb * 128, it.e);
           } else {
@@ -226,6 +261,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
             if (s == stage) armed[s] += 1;
           if (++stage == kStages) { stage = 0; phase_bit ^= 1u; }
         }
+        if (trace) trace[3] = globaltimer();  // every load of the item issued
         item = next_item;
       }
       if (fail_site || *abort_flag) {
@@ -307,6 +343,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       const uint32_t acc_phase = (uint32_t)(local_item >> 1) & 1u;
       if (!mbar_wait(smem_u32(&sh->tmem_full[acc]), acc_phase, abort_flag, wait_ns, 500)) { fail_site = kWaitMbarEpi; break; }
       tc_fence_after();
+      if (prm.item_ns && warp == 2 && lane == 0) prm.item_ns[4 * (size_t)item + 1] = globaltimer();  // MMAs complete
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * kUmmaN);
       size_t row = (size_t)it.tile * kTileRows + row_in_tile;
       bool row_live = true;
@@ -422,10 +459,19 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     // Every CTA has taken its last item index by now; the last one to leave puts the counters back to
     // zero, so a launch never depends on the host having cleared them.
     int* exit_counter = work_counter + 2;
-    if (atomicAdd(exit_counter, 1) == (int)gridDim.x - 1) {
+    const bool last = atomicAdd(exit_counter, 1) == (int)gridDim.x - 1;
+    if (last) {
       *work_counter = 0;
       *exit_counter = 0;
     }
+    sh->last_cta = last ? 1 : 0;
+  }
+  __syncthreads();
+  if (sh->last_cta && phase != 1) {
+    // The last CTA of the launch that ran the GEMM2 items: every wait on the per-tile GEMM1 counters is
+    // over, so they go back to zero too.  A later call on the same tiles (another set of weights on one
+    // dispatch result) then waits for ITS OWN GEMM1 blocks instead of finding the old counts.
+    for (int pt = threadIdx.x; pt < prm.P; pt += kTcThreads) gemm1_done[pt] = 0;
   }
   if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
@@ -492,12 +538,8 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   if ((rc = make_map_2d(enc, &a1t, recv, pool_rows, c.H, kThinRows)) != MOE_OK) return rc;
   if ((rc = make_map_2d(enc, &a2t, p->s.inter, pool_rows, c.F, kThinRows)) != MOE_OK) return rc;
 
-  static bool attr_done = false;  // per-process, idempotent
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem) != cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  static SmemAttrOnce once;
+  if (ensure_dynamic_smem(ffn_tc_kernel, kTcSmem, p->device, once) != cudaSuccess) return MOE_ERR_CUDA;
   const int grid = p->sm_count;
   const int NB1 = (c.F + 127) / 128, NB2 = (c.H + 255) / 256;
   // One launch for both GEMMs, or one per GEMM.  With many small experts (E = 256 under Zipf routing)
@@ -508,7 +550,10 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   const int workers = pairs ? grid / 2 : grid;
   if (p->P > kMaxListTiles) return MOE_ERR_UNSUPPORTED;  // the work list lives in the kernel's shared memory
   if ((long long)p->P * (NB1 + NB2) >= (1ll << kThinShift)) return MOE_ERR_UNSUPPORTED;  // item index field of the ring
-  if (tile_count == nullptr &&  // a call outside moe_layer: the GEMM1 and item counters are not reset by a dispatch
+  // The one-CTA kernel puts its counters back to zero itself; the pair kernel has static item assignment
+  // and no last-one-out step, so its GEMM1 counters are cleared here (also for a call without counters,
+  // which no dispatch preceded).
+  if ((tile_count == nullptr || pairs) &&
       cudaMemsetAsync(p->s.gemm1_done, 0, sizeof(int) * (size_t)(p->P + 4), st) != cudaSuccess)
     return MOE_ERR_CUDA;
   mark(p, 3, st);
@@ -517,6 +562,12 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   prm.P = (int)p->P;
   prm.lag = 2 * workers;
   prm.fused = fused;
+  // Interleaving (opt-in, two-launch form only).  Measured on the DeepSeek-like layer it changes nothing:
+  // every kind of item there takes 57-75 us whether the kinds are mixed or not, because none of them is
+  // bound by HBM bandwidth alone.
+  prm.hot_min = (fused || pairs || c.ffn_hot_min_tiles <= 0) ? 0 : c.ffn_hot_min_tiles;
+  prm.cold_below = prm.hot_min > 0 ? prm.hot_min : 3;
+  prm.thin = c.ffn_thin_tiles >= 0;
   prm.E = c.E;
   prm.F = c.F;
   prm.H = c.H;
@@ -530,6 +581,7 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   prm.total_rows = c.T * c.K;
   prm.status = p->s.status;
   prm.clock_probe = reinterpret_cast<unsigned long long*>(p->s.clock_probe);
+  prm.item_ns = (p->trace && !pairs) ? p->s.item_ns : nullptr;
   auto launch = [&](int phase) -> int {
     prm.phase = phase;
     if (pairs) return launch_ffn_tc2_kernel(a1, bg, bu, a2, bd, prm, grid, st);

@@ -325,12 +325,10 @@ ffn_tc2_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant
 
 int launch_ffn_tc2_kernel(const CUtensorMap& a1, const CUtensorMap& bg, const CUtensorMap& bu, const CUtensorMap& a2,
                           const CUtensorMap& bd, const FfnParams& prm, int grid, cudaStream_t st) {
-  static bool attr_done = false;  // per-process, idempotent
-  if (!attr_done) {
-    if (cudaFuncSetAttribute(ffn_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem2) != cudaSuccess)
-      return MOE_ERR_CUDA;
-    attr_done = true;
-  }
+  static SmemAttrOnce once;
+  int device = -1;
+  cudaGetDevice(&device);
+  if (ensure_dynamic_smem(ffn_tc2_kernel, kTcSmem2, device, once) != cudaSuccess) return MOE_ERR_CUDA;
   return launch_pdl(ffn_tc2_kernel, dim3(grid & ~1), dim3(kTcThreads), kTcSmem2, st, a1, bg, bu, a2, bd, prm) ==
                  cudaSuccess ? 0 : MOE_ERR_CUDA;
 }

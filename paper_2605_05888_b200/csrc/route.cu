@@ -243,12 +243,8 @@ static int launch_wide_tmt(moe_plan* p, const void* x, const void* wr, const flo
   constexpr size_t stage = sizeof(float) * 2 * kWideBuf, logits = sizeof(float) * 8 * TMT * kWideEP;
   constexpr size_t smem = stage > logits ? stage : logits;
   auto kern = route_wide_kernel<XT, TMT>;
-  static bool attr_done = false;  // per instantiation and process, idempotent
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return (int)e;
-    attr_done = true;
-  }
+  static SmemAttrOnce once;  // per instantiation
+  if (cudaError_t e = ensure_dynamic_smem(kern, smem, p->device, once)) return (int)e;
   const moe_config_t& c = p->cfg;
   p->launches += 1;
   return (int)launch_maybe_pdl(false, kern, dim3((c.T + 8 * TMT - 1) / (8 * TMT)), dim3(kWideThreads), smem, st,
@@ -466,12 +462,9 @@ static int launch_narrow(moe_plan* p, const void* x, const void* wr, const float
   constexpr int G = SWAP ? 16 : 2, EP = EW * G * 2, TB = (32 / G) * TWP;
   constexpr size_t smem = sizeof(float) * (2 * (TB + EP) * (HC + 4) > TB * EP ? 2 * (TB + EP) * (HC + 4) : TB * EP);
   auto kern = route_narrow_kernel<XT, SWAP, EW, TWP, HC>;
-  static bool attr_done = false;  // per instantiation and process, idempotent
-  if (smem > 48 * 1024 && !attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e != cudaSuccess) return (int)e;
-    attr_done = true;
-  }
+  static SmemAttrOnce once;  // per instantiation
+  if (smem > 48 * 1024)
+    if (cudaError_t e = ensure_dynamic_smem(kern, smem, p->device, once)) return (int)e;
   const moe_config_t& c = p->cfg;
   p->launches += 1;
   return (int)launch_maybe_pdl(false, kern, dim3((c.T + TB - 1) / TB), dim3(32 * (EW * TWP + kNarrowFillWarps)), smem, st,

@@ -68,6 +68,18 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+// The same load with an L2 eviction-priority hint (a policy made by l2_policy_evict_first/_last).
+__device__ __forceinline__ void tma_load_3d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                                 int c2, uint64_t policy) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "l"(policy) : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -136,6 +148,7 @@ struct Item {
   int type;   // 0: GEMM1 (+SwiGLU), 1: GEMM2
   int e, nb, tile;
   int m;      // tiles of expert e
+  bool cold;  // item of the weight-streaming-bound run (interleaved work list)
 };
 
 // The work list, built by every CTA for itself in shared memory from tile_expert[P] (the same
@@ -145,6 +158,11 @@ struct Item {
 //   expert: seg_start[i] first item of segment i (seg_start[2E] = number of items), seg_info[i] =
 //   expert | type << 16 (type 0: GEMM1, 1: GEMM2); n1 = items before the first GEMM2 item when the
 //   two GEMMs are separate launches.
+//   With hot_min > 0 (separate launches only) each GEMM's segments are ordered "hot" experts first
+//   (at least hot_min tiles: their items are bound by the tensor pipe, the weights come out of L2),
+//   then "cold" ones (fewer tiles: bound by streaming the expert's weights from HBM once), both in
+//   ascending expert order, and n_hot[g] counts the hot items of GEMM g: the kernel walks the two
+//   runs interleaved, so that at any moment some SMs pull weights from HBM while the others run MMAs.
 constexpr int kMaxListTiles = 4608;
 struct WorkList {
   int estart[kMaxExperts + 1];
@@ -152,6 +170,7 @@ struct WorkList {
   int seg_info[2 * kMaxExperts];
   int cursor[kMaxExperts];
   int n1;
+  int n_hot[2];
   int tiles[kMaxListTiles];
 };
 
@@ -160,7 +179,7 @@ struct WorkList {
 // GEMM1 segment, as long as `lag` GEMM2 items stay in reserve for the end of the list; otherwise all
 // GEMM1 segments come first.
 __device__ __forceinline__ void build_worklist(WorkList& wl, const int* __restrict__ tile_expert, int P, int E,
-                                               int NB1, int NB2, int lag, int fused, int pair) {
+                                               int NB1, int NB2, int lag, int fused, int pair, int hot_min = 0) {
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid % 32;
   for (int e = tid; e < kMaxExperts; e += nthr) wl.cursor[e] = 0;
   __syncthreads();
@@ -206,7 +225,27 @@ __device__ __forceinline__ void build_worklist(WorkList& wl, const int* __restri
       if (e >= 0 && lane == __ffs(peers) - 1) wl.cursor[e] += __popc(peers);
       __syncwarp();
     }
-    if (lane == 0) {
+    if (lane == 0 && !fused && hot_min > 0) {
+      // two passes per GEMM: hot experts, then cold ones
+      int pos = 0, nseg = 0;
+      for (int g = 0; g < 2; ++g) {
+        const int nb = g == 0 ? NB1 : NB2;
+        const int begin = pos;
+        for (int cold = 0; cold < 2; ++cold) {
+          for (int e = 0; e < E; ++e) {
+            const int m = wl.estart[e + 1] - wl.estart[e];
+            if ((m >= hot_min ? 0 : 1) != cold) continue;
+            wl.seg_start[nseg] = pos;
+            wl.seg_info[nseg++] = e | (g << 16);
+            pos += (m + pair - 1) / pair * nb;
+          }
+          if (cold == 0) wl.n_hot[g] = pos - begin;
+        }
+        if (g == 0) wl.n1 = pos;
+      }
+      wl.seg_start[nseg] = pos;  // nseg == 2E
+    } else if (lane == 0) {
+      wl.n_hot[0] = wl.n_hot[1] = -1;  // no interleaving
       int pos = 0, nseg = 0, q = 0;
       // GEMM2 items of experts q+1 .. E-2: what would still stand between the last expert's GEMM1 and
       // its GEMM2 if expert q's GEMM2 segment were placed now.  Keeping `lag` items in that reserve
@@ -244,6 +283,9 @@ __device__ __forceinline__ void build_worklist(WorkList& wl, const int* __restri
 struct FfnParams {
   const int* tile_expert;  // [P]
   int P, lag, fused;
+  int hot_min;  // > 0: interleave tensor-bound and weight-streaming-bound items (see WorkList)
+  int thin;         // the narrow (transposed) form for single tiles of at most 64 rows is in use
+  int cold_below;   // experts with fewer tiles than this stream their weights once: their loads are evict-first
   int phase, E, F, H;
   __nv_bfloat16* inter;
   __nv_bfloat16* out;
@@ -256,6 +298,7 @@ struct FfnParams {
   unsigned long long wait_ns;  // bound on every wait inside the kernel
   int* status;
   unsigned long long* clock_probe;  // [2]: SM cycles and nanoseconds CTA 0 spent in the kernel (accumulated)
+  unsigned long long* item_ns;      // work-item timeline (measurement; nullptr: off): 4 words per position of the item list
 };
 
 // Effective SM clock while a kernel runs: CTA 0 adds its elapsed %clock64 and %globaltimer.

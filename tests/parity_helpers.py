@@ -92,6 +92,55 @@ def max_rel_err(got: np.ndarray, ref: np.ndarray) -> float:
     return elementwise_rel_err(got, ref)
 
 
+# Distance between a bf16 result of the CUDA path and the oracle's bf16-storage restatement (same three
+# roundings, sums in fp64).  The two round nearly equal reals at the same three places, so a stored value
+# can differ only by landing on the other side of a rounding boundary: by one bf16 step.  (It happens to
+# several percent of the elements: one step in a few of the F intermediates moves an expert output by
+# ~1e-4 of its size, a twentieth of the distance between boundaries.)  Hence, element by element,
+#   |y_gpu - y_stored| <= step(y) + sum_k w_k * (step(o_k) + noise_k),
+# step(v) = the spacing of bf16 numbers at |v| (2^(floor(log2|v|) - 7)), o_k the token's expert rows of the
+# restatement, noise_k = 2^-10 of the row's rms for what the flipped intermediates move before rounding.
+# A few bf16 steps of each element itself: a kernel that lost a further bit anywhere would fail it.
+def bf16_step(v: np.ndarray) -> np.ndarray:
+    v = np.maximum(np.abs(v), 2.0 ** -120)
+    return 2.0 ** (np.floor(np.log2(v)) - 7)
+
+
+def assert_close_to_bf16_storage(got: np.ndarray, stored: dict, what: str = "output") -> None:
+    """got: y of the CUDA path [T,H] as fp64; stored: the oracle layer dict computed with bf16_storage=True
+    on the same tokens."""
+    y, rows, slot, w = stored["y"], stored["out_rows"], stored["slot_of"], stored["topk_w"].astype(np.float64)
+    T, K = slot.shape
+    bound = bf16_step(np.maximum(np.abs(y), np.abs(got)))
+    for k in range(K):
+        o = rows[slot[:, k]]
+        rms = np.sqrt(np.mean(o * o, axis=1, keepdims=True))
+        bound = bound + w[:, k:k + 1] * (bf16_step(o) * 2.0 + rms * 2.0 ** -10)   # 2 steps: |o| may sit just under a binade edge
+    excess = np.abs(got - y) / bound
+    worst = float(excess.max()) if excess.size else 0.0
+    assert worst <= 1.0, f"{what}: {worst:.2f} x the few-bf16-steps bound from the bf16-storage restatement"
+
+
+def tokens_covering_every_tile(slot_of: np.ndarray, extra: np.ndarray | None = None) -> np.ndarray:
+    """A set of tokens whose rows touch every used 128-row tile of the receive pool (greedy: walk the tiles
+    in order, take the token of the lowest row of every tile not yet touched), plus `extra` tokens."""
+    T, K = slot_of.shape
+    tile_of = slot_of // 128
+    order = np.argsort(slot_of.ravel(), kind="stable")       # assignments by physical row
+    covered, chosen = set(), []
+    for a in order:
+        tile = int(tile_of.ravel()[a])
+        if tile in covered:
+            continue
+        t = int(a // K)
+        chosen.append(t)
+        covered.update(int(v) for v in tile_of[t])
+    tokens = np.array(chosen, np.int64)
+    if extra is not None:
+        tokens = np.union1d(tokens, extra)
+    return np.unique(tokens)
+
+
 def check_route(idx_gpu, w_gpu, idx_ref, w_ref):
     idx_gpu, w_gpu = idx_gpu.cpu().numpy(), w_gpu.cpu().numpy()
     bad = np.nonzero((idx_gpu != idx_ref).any(axis=1))[0]
@@ -144,7 +193,8 @@ def oracle_inputs(w: inputs.Workload, with_experts=True):
     return x, wr, bias, wg, wu, wd
 
 
-def oracle_layer_for(w: inputs.Workload, x, wr, bias, wg, wu, wd):
+def oracle_layer_for(w: inputs.Workload, x, wr, bias, wg, wu, wd, bf16_storage=False):
     ws = (None, None, None) if wg is None else ([wg[e] for e in range(w.E)], [wu[e] for e in range(w.E)],
                                                  [wd[e] for e in range(w.E)])
-    return oracle.layer(x, wr, bias, *ws, w.E, w.R, w.K, w.dtype, identity_experts=w.identity_experts)
+    return oracle.layer(x, wr, bias, *ws, w.E, w.R, w.K, w.dtype, identity_experts=w.identity_experts,
+                        bf16_storage=bf16_storage)

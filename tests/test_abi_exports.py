@@ -32,8 +32,38 @@ def test_every_declared_symbol_is_exported(lib):
     assert sorted(B.EXPORTS) == names, "binding.EXPORTS and the header disagree"
 
 
+def header_config_fields():
+    """(name, ctypes type) of every field of moe_config_t, parsed from the header."""
+    text = open(os.path.join(ROOT, "include", "moehub.h")).read()
+    body = re.search(r"typedef struct \{(.*?)\} moe_config_t;", text, flags=re.S).group(1)
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    ctype = {"int32_t": ctypes.c_int32, "int64_t": ctypes.c_int64, "uint64_t": ctypes.c_uint64}
+    fields = []
+    for decl in body.split(";"):
+        decl = decl.strip()
+        if not decl:
+            continue
+        ty, names = decl.split(None, 1)
+        for name in names.split(","):
+            name = name.strip()
+            m = re.fullmatch(r"(\w+)\[(\d+)\]", name)
+            fields.append((m.group(1), ctype[ty] * int(m.group(2))) if m else (name, ctype[ty]))
+    return fields
+
+
 def test_config_struct_matches_header():
-    assert ctypes.sizeof(B.MoeConfig) == 12 * 4 + 8 + 8 + 8
+    """Same fields, same order, same types: the binding's ctypes structure mirrors the C struct."""
+    want = header_config_fields()
+    got = [(n, t) for n, t in B.MoeConfig._fields_]
+    assert [n for n, _ in got] == [n for n, _ in want]
+    for (n, t_got), (_, t_want) in zip(got, want):
+        assert ctypes.sizeof(t_got) == ctypes.sizeof(t_want), n
+
+    class Mirror(ctypes.Structure):
+        _fields_ = want
+    assert ctypes.sizeof(B.MoeConfig) == ctypes.sizeof(Mirror)
+    for n, _ in want:
+        assert getattr(B.MoeConfig, n).offset == getattr(Mirror, n).offset, n
 
 
 def test_host_side_checks_without_gpu(lib):

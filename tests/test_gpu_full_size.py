@@ -2,9 +2,11 @@
 paged atomic dispatch, tensor-core experts).
 
 Routing and dispatch are compared with the oracle in full (bit-exact).  The expert FFN at these
-sizes is 3-6 TFLOP, too much for the CPU oracle, so the combined output is compared on a seeded
-sample of tokens: tokens are independent, so the oracle layer run on x[sample] gives exactly the
-rows y[sample] of the full batch.  Properties that hold at any size (identity experts give
+sizes is 3-6 TFLOP, too much for the CPU oracle, so the combined output is compared on a sample of
+tokens: tokens are independent, so the oracle layer run on x[sample] gives exactly the rows
+y[sample] of the full batch.  The sample is drawn from the run's own slot_of so that EVERY used
+128-row tile of the receive pool holds at least one compared row (every work item of the expert
+kernel, whatever its form, contributes to a compared output), plus a seeded random sample.  Properties that hold at any size (identity experts give
 x * sum_k w) cover the largest dispatch/combine sweep point.
 """
 import numpy as np
@@ -37,12 +39,19 @@ def check_full_routing_and_dispatch(w, plan, x, wr, bias):
     return idx, d
 
 
-def check_sampled_output(w, y, x, wr, bias, wg, wu, wd, n_sample, seed=0):
+def check_sampled_output(w, plan, y, x, wr, bias, wg, wu, wd, n_sample, seed=0):
     rng = np.random.default_rng(seed)
-    sample = np.sort(rng.choice(w.T, size=n_sample, replace=False))
-    ref = oracle.layer(np.ascontiguousarray(x[sample]), wr, bias, list(wg), list(wu), list(wd), w.E, w.R, w.K, w.dtype)
+    slot = plan.layer_tensor(6).cpu().numpy()
+    sample = Hh.tokens_covering_every_tile(slot, np.sort(rng.choice(w.T, size=n_sample, replace=False)))
+    used = np.unique(slot // 128)
+    assert np.array_equal(np.unique(slot[sample] // 128), used), "a used tile has no compared row"
+    xs = np.ascontiguousarray(x[sample])
+    ref = oracle.layer(xs, wr, bias, list(wg), list(wu), list(wd), w.E, w.R, w.K, w.dtype)
     got = Hh.to_host_f64(y[torch.from_numpy(sample).cuda()])
     Hh.assert_output_close(got, ref["y"], w.dtype, "sampled tokens")
+    stored = oracle.layer(xs, wr, bias, list(wg), list(wu), list(wd), w.E, w.R, w.K, w.dtype, bf16_storage=True)
+    Hh.assert_close_to_bf16_storage(got, stored, "sampled tokens")
+    return sample.size, used.size
 
 
 @pytest.mark.parametrize("mode", [B.DISPATCH_ATOMIC_PAGED, B.DISPATCH_SCAN])
@@ -53,7 +62,7 @@ def test_c2_mixtral_like_full_size(mode):
     _, d = check_full_routing_and_dispatch(w, plan, x, wr, bias)
     # near-uniform load (the recipe's forecast: every expert within a few percent of T*K/E)
     assert d["count"].min() > 0.9 * w.T * w.K / w.E and d["count"].max() < 1.1 * w.T * w.K / w.E
-    check_sampled_output(w, y, x, wr, bias, wg, wu, wd, 32)
+    check_sampled_output(w, plan, y, x, wr, bias, wg, wu, wd, 32)
 
 
 def test_c3_deepseek_like_full_size_skewed():
@@ -63,7 +72,7 @@ def test_c3_deepseek_like_full_size_skewed():
     _, d = check_full_routing_and_dispatch(w, plan, x, wr, bias)
     # the Zipf bias really skews the load: hottest expert far above the mean, some experts below one tile
     assert d["count"].max() > 8 * w.T * w.K / w.E and (d["count"] < 128).sum() > 32
-    check_sampled_output(w, y, x, wr, bias, wg, wu, wd, 24)
+    check_sampled_output(w, plan, y, x, wr, bias, wg, wu, wd, 24)
 
 
 @pytest.mark.parametrize("mode", [B.DISPATCH_SCAN, B.DISPATCH_ATOMIC_STATIC, B.DISPATCH_ATOMIC_PAGED])
@@ -74,6 +83,8 @@ def test_c4_qwen_like_full_size(mode):
     check_full_routing_and_dispatch(w, plan, x, wr, bias)
     ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)      # small enough for the whole oracle layer
     Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+    stored = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd, bf16_storage=True)
+    Hh.assert_close_to_bf16_storage(Hh.to_host_f64(y), stored)
 
 
 @pytest.mark.parametrize("w", [inputs.PHI35, inputs.QWEN64], ids=lambda w: w.name)
@@ -83,7 +94,7 @@ def test_other_table2_shapes(w):
     x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
     plan, y = run_layer(w, B.DISPATCH_ATOMIC_PAGED, x, wr, bias, Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd))
     check_full_routing_and_dispatch(w, plan, x, wr, bias)
-    check_sampled_output(w, y, x, wr, bias, wg, wu, wd, 32)
+    check_sampled_output(w, plan, y, x, wr, bias, wg, wu, wd, 32)
 
 
 @pytest.mark.parametrize("zipf", [0.0, 1.2])

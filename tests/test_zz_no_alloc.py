@@ -1,13 +1,16 @@
 """moe_dispatch_noalloc, the dispatch entry point for callers that cannot allocate device memory
-(it keeps its scratch in a fixed array inside the library), against the ordinary moe_dispatch.
+(it keeps its scratch in a fixed array inside the library).
 
 This file is collected last on purpose: a run that stops at the first failure has then already
 run every other test.  It passes alone in a fresh process and after the other tests.
 
-Both entry points are called through the C ABI on the same inputs, twice in a row with different
-routing, so the second call meets the scratch array exactly as the first one left it.  Dispatch is
-byte and index work, so the comparison is exact; only the order of rows inside an expert is free
-(arrival order), which is removed by reading every row through slot_of.
+The entry point is called through the C ABI twice in a row with different routing, so the second
+call meets the scratch array exactly as the first one left it.  Dispatch is byte and index work,
+so every check is exact: each assignment's row is the bytes of its token (read through slot_of,
+which removes the one freedom, the arrival order of rows inside an expert), it sits in a tile of
+its expert, counts are a bincount of the routing, tiles are densely packed.  The ordinary
+moe_dispatch is run on the same inputs and must agree on everything that is unique; and the warm
+second call must leave the amount of free device memory exactly where it was.
 """
 import numpy as np
 import pytest
@@ -44,7 +47,7 @@ def canonical(b, w):
     return b["cnt"].cpu().numpy(), rows, owner, tiles
 
 
-def test_noalloc_dispatch_matches_plan_dispatch_twice_in_a_row():
+def test_noalloc_dispatch_moves_the_right_bytes_twice_in_a_row():
     w = inputs.Workload("noalloc", T=1500, H=512, E=32, R=4, K=4, F=64, dtype=inputs.BF16, zipf_s=1.0)
     x = inputs.make_x(w)
     dx = dev_bf16(x)
@@ -60,15 +63,23 @@ def test_noalloc_dispatch_matches_plan_dispatch_twice_in_a_row():
         old, new = buffers(plan.P, w), buffers(plan.P, w)
         plan.moe_dispatch(dx, didx, old["recv"], old["cnt"], old["te"], old["src"], old["slot"])
         assert plan.moe_last_status() == (0, 0)
+        torch.cuda.synchronize()
+        free_before, torch_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         B.moe_dispatch_noalloc(cfg, dx, didx, new["recv"], new["cnt"], new["te"], new["src"], new["slot"], status)
         torch.cuda.synchronize()
+        if call == 1:   # the warm call: the library took no device memory, through torch or past it
+            assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == torch_before
         assert status.cpu().tolist() == [0, 0]
-        c_old, r_old, o_old, t_old = canonical(old, w)
         c_new, r_new, o_new, t_new = canonical(new, w)
-        assert np.array_equal(c_new, c_old) and np.array_equal(c_new, np.bincount(idx.ravel(), minlength=w.E))
-        assert r_new.tobytes() == r_old.tobytes()
-        assert np.array_equal(o_new, o_old) and np.array_equal(o_new, idx.ravel())
-        assert np.array_equal(t_new, t_old) and np.array_equal(t_new, (c_new + 127) // 128)
+        # against the definition: row of assignment (t, k) == x[t] bytewise, in a tile of expert idx[t, k]
+        assert r_new.tobytes() == np.repeat(x.view(np.int16), w.K, axis=0).tobytes()
+        assert np.array_equal(o_new, idx.ravel())
+        assert np.array_equal(c_new, np.bincount(idx.ravel(), minlength=w.E))
+        assert np.array_equal(t_new, (c_new + 127) // 128)
+        # and against the existing entry point
+        c_old, r_old, o_old, t_old = canonical(old, w)
+        assert np.array_equal(c_new, c_old) and r_new.tobytes() == r_old.tobytes()
+        assert np.array_equal(o_new, o_old) and np.array_equal(t_new, t_old)
 
 
 def test_noalloc_dispatch_rejects_sizes_beyond_its_scratch():
