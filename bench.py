@@ -203,10 +203,12 @@ def run_cuda(args, w: inputs.Workload) -> None:
         wg, wu, wd = inputs.make_all_expert_weights(w.with_(seed=0))  # same parameters on every rank
     dx, dwr, dbias, dwg, dwu, dwd = dev(x), dev(wr), dev(bias), dev(wg), dev(wu), dev(wd)
     el = torch.bfloat16 if w.dtype == inputs.BF16 else torch.float32
-    mode = {"scan": B.DISPATCH_SCAN, "static": B.DISPATCH_ATOMIC_STATIC, "paged": B.DISPATCH_ATOMIC_PAGED}[args.dispatch]
+    mode = {"scan": B.DISPATCH_SCAN, "static": B.DISPATCH_ATOMIC_STATIC, "paged": B.DISPATCH_ATOMIC_PAGED,
+            "ordered": B.DISPATCH_ATOMIC_ORDERED}[args.dispatch]
     plan = B.Plan(B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype, dispatch_mode=mode,
                                 identity_experts=int(w.identity_experts), ffn_split=int(args.ffn_split),
-                                ffn_kernel=args.ffn_kernel, ffn_hot_min_tiles=args.ffn_hot_min_tiles, ffn_thin_tiles=args.ffn_thin_tiles))
+                                ffn_kernel=args.ffn_kernel, ffn_hot_min_tiles=args.ffn_hot_min_tiles, ffn_thin_tiles=args.ffn_thin_tiles,
+                                overlap=args.overlap))
     y = torch.empty((w.T, w.H), dtype=el, device="cuda")
     stream = torch.cuda.current_stream()
 
@@ -401,7 +403,7 @@ def main() -> None:
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
-    ap.add_argument("--dispatch", default="paged", choices=["scan", "static", "paged"])
+    ap.add_argument("--dispatch", default="paged", choices=["scan", "static", "paged", "ordered"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ffn-kernel", type=int, default=0, choices=[0, 1, 2],
                     help="0: tcgen05 one CTA per tile (default), 2: tcgen05 CTA pairs, 1: SIMT check path")
@@ -411,6 +413,8 @@ def main() -> None:
                     help="two-launch expert GEMMs: experts with at least this many tiles are walked as tensor-bound "
                          "work, interleaved with the weight-streaming-bound rest (0: library default, -1: off)")
     ap.add_argument("--ffn-thin-tiles", type=int, default=0, help="-1: no transposed narrow form for small single tiles")
+    ap.add_argument("--overlap", type=int, default=0,
+                    help="with --dispatch ordered: dispatch inside the expert kernel's launch (1: half of the SMs dispatch, n: n CTAs)")
     args = ap.parse_args()
     w = WORKLOADS[args.workload]
     if args.impl == "reference":

@@ -34,7 +34,7 @@
  *    expert's rows are dense inside its tiles (only its last tile may be partly filled).
  *    Physical row = tile*128 + row-in-tile.  Within one expert the order of rows is
  *    unspecified in the atomic modes (arrival order, Section IV-B) and is (token, k) order in
- *    mode 0.
+ *    mode 0.  In mode 3 an expert's tiles are consecutive pool tiles, experts in ascending order.
  */
 #ifndef MOEHUB_H_
 #define MOEHUB_H_
@@ -55,6 +55,8 @@ extern "C" {
 #define MOE_ERR_TIMEOUT (-6)     /* device status: a bounded device-side wait ran out */
 #define MOE_ERR_WORKSPACE (-7)   /* workspace too small or misaligned */
 #define MOE_ERR_TOO_LARGE (-8)   /* moe_dispatch_noalloc: T or E beyond its fixed built-in scratch */
+#define MOE_ERR_INTERNAL (-9)    /* device status: a kernel's own index check failed (the access was
+                                    skipped); detail names the check */
 
 #define MOE_DTYPE_FP32 0
 #define MOE_DTYPE_BF16 1
@@ -62,6 +64,10 @@ extern "C" {
 #define MOE_DISPATCH_SCAN 0          /* baseline: histogram -> exclusive scan -> stable scatter */
 #define MOE_DISPATCH_ATOMIC_STATIC 1 /* row-pointer atomics, one static region per expert   */
 #define MOE_DISPATCH_ATOMIC_PAGED 2  /* row-pointer atomics, 128-row tiles paged on demand  */
+#define MOE_DISPATCH_ATOMIC_ORDERED 3 /* row-pointer atomics; persistent CTAs emit the tokens in one
+                                        ascending order (Section IV-C: smallest RowID first), regions
+                                        sized by the rows per expert that the router counted, rows
+                                        moved by bulk asynchronous copies                           */
 
 #define MOE_TILE_ROWS 128
 
@@ -89,7 +95,14 @@ typedef struct {
   int32_t ffn_thin_tiles;       /* tensor-core kernel: 0 = an expert's only tile, if it holds at
                                    most 64 rows, is computed in the transposed narrow form;
                                    negative = never (such a tile runs M = 64 MMAs instead)      */
-  int32_t reserved_[2];         /* must be 0                                                  */
+  int32_t overlap;              /* moe_layer, dispatch mode 3, bf16, tensor-core kernel: != 0 =
+                                   dispatch and expert computation in ONE launch: n producer CTAs
+                                   (1: half as many as SMs, n > 1: n) only dispatch, and as many
+                                   consumer CTAs as there are SMs compute every tile as soon as
+                                   its status counter has reached its threshold (Section IV-D);
+                                   negative: the same launch, but the consumers wait for the whole
+                                   dispatch (for comparison); 0 = stream-ordered launches        */
+  int32_t reserved_[1];         /* must be 0                                                  */
   int64_t capacity_rows;        /* mode 1: rows per expert region, multiple of 128, 0 = T
                                    rounded up (overflow-free); modes 0/2: ignored            */
   uint64_t spin_limit;          /* bound (iterations) on the dispatch kernels' waits, 0 = 1<<22 */
@@ -98,7 +111,7 @@ typedef struct {
 } moe_config_t;
 
 /* Number P of 128-row tiles in the receive pool for this configuration:
- * modes 0/2: floor(T*K/128) + E;  mode 1: E * capacity_rows/128. */
+ * modes 0/2/3: floor(T*K/128) + E;  mode 1: E * capacity_rows/128. */
 int moe_pool_tiles(const moe_config_t* cfg, int64_t* out_tiles);
 
 /* Bytes of device workspace moe_plan_create needs (scratch counters, tile tables, the SwiGLU
@@ -272,6 +285,12 @@ int moe_last_launch_count(moe_plan_t* plan, int32_t* out);
  * MOE_ERR_TIMEOUT or MOE_ERR_ARG; *detail says where (expert id for an overflow, wait site for
  * a timeout, token index for an expert id outside [0, E)).  The first error of a call wins. */
 int moe_last_status(moe_plan_t* plan, void* stream, int32_t* code, int32_t* detail);
+
+/* After moe_layer returned MOE_ERR_CUDA: which of its steps met the CUDA error (1 router, 2 dispatch,
+ * 3 experts, 4 combine; 0: none so far) and the error's name as the CUDA runtime spells it (a static
+ * string).  Kernel launches are asynchronous, so an error raised while a kernel RUNS is reported by a
+ * later step (or by the next synchronising call) unless launches are made blocking. */
+int moe_last_cuda_error(moe_plan_t* plan, int32_t* step, const char** name);
 
 const char* moe_strerror(int code);
 

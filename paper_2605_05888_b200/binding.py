@@ -17,14 +17,14 @@ _lib = None
 
 MOE_OK = 0
 DTYPE_FP32, DTYPE_BF16 = 0, 1
-DISPATCH_SCAN, DISPATCH_ATOMIC_STATIC, DISPATCH_ATOMIC_PAGED = 0, 1, 2
+DISPATCH_SCAN, DISPATCH_ATOMIC_STATIC, DISPATCH_ATOMIC_PAGED, DISPATCH_ATOMIC_ORDERED = 0, 1, 2, 3
 TILE_ROWS = 128
 STAGES = ["route", "dispatch", "worklist", "gemm1", "gemm2", "combine"]
 
 EXPORTS = ["moe_dispatch_noalloc", "moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
            "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host", "moe_layer_host_submit", "moe_layer_host_wait", "moe_layer_timed",
            "moe_layer_buffer", "moe_availability_trace",
-           "moe_ffn_clock_mhz", "moe_last_launch_count", "moe_last_status", "moe_strerror"]
+           "moe_ffn_clock_mhz", "moe_last_launch_count", "moe_last_status", "moe_last_cuda_error", "moe_strerror"]
 
 
 class MoeConfig(ctypes.Structure):
@@ -33,7 +33,7 @@ class MoeConfig(ctypes.Structure):
                 ("renormalize", ctypes.c_int32), ("dispatch_mode", ctypes.c_int32),
                 ("identity_experts", ctypes.c_int32), ("ffn_kernel", ctypes.c_int32), ("ffn_split", ctypes.c_int32),
                 ("ffn_hot_min_tiles", ctypes.c_int32), ("ffn_thin_tiles", ctypes.c_int32),
-                ("reserved_", ctypes.c_int32 * 2),
+                ("overlap", ctypes.c_int32), ("reserved_", ctypes.c_int32 * 1),
                 ("capacity_rows", ctypes.c_int64), ("spin_limit", ctypes.c_uint64), ("wait_limit_ns", ctypes.c_uint64)]
 
 
@@ -71,6 +71,7 @@ def lib() -> ctypes.CDLL:
         L.moe_ffn_clock_mhz.argtypes = [vp, vp, ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
         L.moe_last_launch_count.argtypes = [vp, ctypes.POINTER(ctypes.c_int32)]
         L.moe_last_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
+        L.moe_last_cuda_error.argtypes = [vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_char_p)]
         L.moe_strerror.argtypes = [ctypes.c_int]
         L.moe_strerror.restype = ctypes.c_char_p
         for name in EXPORTS:
@@ -106,9 +107,9 @@ def _stream(stream) -> int:
 
 def make_config(T, H, E, R, K, F, dtype, renormalize=0, dispatch_mode=DISPATCH_ATOMIC_PAGED, identity_experts=0,
                 ffn_kernel=0, capacity_rows=0, spin_limit=0, ffn_split=0, wait_limit_ns=0,
-                ffn_hot_min_tiles=0, ffn_thin_tiles=0) -> MoeConfig:
+                ffn_hot_min_tiles=0, ffn_thin_tiles=0, overlap=0) -> MoeConfig:
     return MoeConfig(T, H, E, R, K, F, dtype, int(renormalize), dispatch_mode, int(identity_experts), ffn_kernel, int(ffn_split),
-                     int(ffn_hot_min_tiles), int(ffn_thin_tiles), (ctypes.c_int32 * 2)(0, 0), capacity_rows, spin_limit, wait_limit_ns)
+                     int(ffn_hot_min_tiles), int(ffn_thin_tiles), int(overlap), (ctypes.c_int32 * 1)(0), capacity_rows, spin_limit, wait_limit_ns)
 
 
 def moe_pool_tiles(cfg: MoeConfig) -> int:
@@ -223,6 +224,12 @@ class Plan:
         out = ctypes.c_int32()
         _check(lib().moe_last_launch_count(self.handle, ctypes.byref(out)), "moe_last_launch_count")
         return out.value
+
+    def moe_last_cuda_error(self) -> tuple[int, str]:
+        """(step of moe_layer that met a CUDA error, the error's name); step 0: none."""
+        step, name = ctypes.c_int32(), ctypes.c_char_p()
+        _check(lib().moe_last_cuda_error(self.handle, ctypes.byref(step), ctypes.byref(name)), "moe_last_cuda_error")
+        return step.value, (name.value or b"").decode()
 
     def moe_last_status(self, stream=None) -> tuple[int, int]:
         code, detail = ctypes.c_int32(), ctypes.c_int32()

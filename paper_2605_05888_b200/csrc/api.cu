@@ -15,6 +15,7 @@ inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 struct Geometry {
   int64_t P, cap_rows;
   int tiles_per_expert, dispatch_tokens, nblk, eb;
+  int ord_tokens, ord_nblk;
 };
 
 int check_config(const moe_config_t* c, Geometry* g) {
@@ -22,9 +23,10 @@ int check_config(const moe_config_t* c, Geometry* g) {
   if (c->T < 0 || c->H <= 0 || c->E <= 0 || c->R <= 0 || c->K <= 0) return MOE_ERR_ARG;
   if (c->K > c->E || c->E % c->R != 0) return MOE_ERR_ARG;
   if (c->dtype != MOE_DTYPE_FP32 && c->dtype != MOE_DTYPE_BF16) return MOE_ERR_ARG;
-  if (c->dispatch_mode < 0 || c->dispatch_mode > 2) return MOE_ERR_ARG;
+  if (c->dispatch_mode < 0 || c->dispatch_mode > 3) return MOE_ERR_ARG;
   if (!c->identity_experts && c->F <= 0) return MOE_ERR_ARG;
   if (c->E > 256 || c->K > 32) return MOE_ERR_UNSUPPORTED;
+  if (c->reserved_[0] != 0) return MOE_ERR_ARG;
   const int eb = c->dtype == MOE_DTYPE_BF16 ? 2 : 4;
   if (((int64_t)c->H * eb) % 16 != 0) return MOE_ERR_ALIGN;
   if (!c->identity_experts && ((int64_t)c->F * eb) % 16 != 0) return MOE_ERR_ALIGN;
@@ -50,6 +52,13 @@ int check_config(const moe_config_t* c, Geometry* g) {
   while (tpb > 1 && (c->T + tpb - 1) / tpb < 2 * 148) tpb /= 2;  // small batches: enough CTAs to fill the GPU
   g->dispatch_tokens = tpb;
   g->nblk = (c->T + tpb - 1) / tpb;
+  // ordered dispatch: at most 128 assignments per token block, smaller blocks while there are fewer blocks than SMs
+  int otb = 128 / c->K;
+  if (otb > 16) otb = 16;
+  if (otb < 1) otb = 1;
+  while (otb > 1 && (c->T + otb - 1) / otb < 148) otb /= 2;
+  g->ord_tokens = otb;
+  g->ord_nblk = (c->T + otb - 1) / otb;
   return MOE_OK;
 }
 
@@ -74,6 +83,9 @@ size_t carve(const moe_config_t& c, const Geometry& g, char* base, Scratch* s, s
   t.cta_count = (int*)take(sizeof(int) * (size_t)(g.nblk > 0 ? g.nblk : 1) * c.E);
   t.cta_base = (int*)take(sizeof(int) * (size_t)(g.nblk > 0 ? g.nblk : 1) * c.E);
   t.tile_base = (int*)take(sizeof(int) * (size_t)(c.E + 1));
+  t.hist = (int*)take(sizeof(int) * (size_t)c.E);
+  t.row_pointer = (int*)take(sizeof(int) * (size_t)c.E);
+  t.ord_exit = (int*)take(sizeof(int) * 2);
   t.clock_probe = (unsigned long long*)take(sizeof(unsigned long long) * 2);
   t.avail_ns = (unsigned long long*)take(sizeof(unsigned long long) * (size_t)((g.P > 0 ? g.P : 1) + 2));
   if (!c.identity_experts && c.dtype == MOE_DTYPE_BF16) {
@@ -140,7 +152,11 @@ int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, mo
   p->tiles_per_expert = g.tiles_per_expert;
   p->dispatch_tokens = g.dispatch_tokens;
   p->nblk = g.nblk;
+  p->ord_tokens = g.ord_tokens;
+  p->ord_nblk = g.ord_nblk;
   p->launches = 0;
+  p->cuda_error = 0;
+  p->cuda_error_step = 0;
   p->encode_tiled = nullptr;
   p->timing = 0;
   for (int i = 0; i <= MOE_STAGE_COUNT; ++i) p->tev[i] = nullptr;
@@ -155,6 +171,9 @@ int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, mo
   }
   // The status word must start clean even if a stage other than dispatch is called first.
   if (cudaMemset(p->s.status, 0, p->counters_bytes) != cudaSuccess ||
+      cudaMemset(p->s.hist, 0, sizeof(int) * (size_t)cfg->E) != cudaSuccess ||
+      cudaMemset(p->s.ord_exit, 0, sizeof(int) * 2) != cudaSuccess ||
+      cudaMemset(p->s.gemm1_done, 0, sizeof(int) * (size_t)(g.P + 4)) != cudaSuccess ||
       cudaMemset(p->s.clock_probe, 0, 2 * sizeof(unsigned long long)) != cudaSuccess) {
     delete p;
     return MOE_ERR_CUDA;
@@ -184,7 +203,7 @@ int moe_route(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_b
   if (!p || !d_wr || !d_topk_idx || !d_topk_w || (!d_x && p->cfg.T > 0)) return MOE_ERR_ARG;
   if (misaligned(d_x) || misaligned(d_wr)) return MOE_ERR_ALIGN;
   p->launches = 0;
-  return launch_route(p, d_x, d_wr, d_bias, d_topk_idx, d_topk_w, (cudaStream_t)stream) ? MOE_ERR_CUDA : MOE_OK;
+  return launch_route(p, d_x, d_wr, d_bias, d_topk_idx, d_topk_w, nullptr, (cudaStream_t)stream) ? MOE_ERR_CUDA : MOE_OK;
 }
 
 int moe_dispatch(moe_plan_t* p, const void* d_x, const int32_t* d_topk_idx, void* d_recv,
@@ -197,7 +216,7 @@ int moe_dispatch(moe_plan_t* p, const void* d_x, const int32_t* d_topk_idx, void
   if ((d_tile_count == nullptr) != (d_rows_done == nullptr)) return MOE_ERR_ARG;
   return launch_dispatch(p, d_x, d_topk_idx, d_recv, d_expert_count, d_tile_expert, d_src_info, d_slot_of,
                          d_tile_count ? d_tile_count : p->s.tile_count, d_rows_done ? d_rows_done : p->s.rows_done,
-                         (cudaStream_t)stream) ? MOE_ERR_CUDA : MOE_OK;
+                         false, (cudaStream_t)stream) ? MOE_ERR_CUDA : MOE_OK;
 }
 
 static int ffn_dispatch(moe_plan* p, const void* recv, const int* tile_expert, const void* wg, const void* wu,
@@ -243,22 +262,46 @@ int moe_layer(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_b
   Scratch& s = p->s;
   p->launches = 0;
   mark(p, 0, st);
-  if (launch_route(p, d_x, d_wr, d_bias, s.topk_idx, s.topk_w, st)) return MOE_ERR_CUDA;
-  mark(p, 1, st);
-  if (launch_dispatch(p, d_x, s.topk_idx, s.recv, s.expert_count, s.tile_expert, s.src_info, s.slot_of, s.tile_count,
-                      s.rows_done, st))
+  // The router puts the dispatch's counters and tables into their start state on the side (and counts the
+  // rows per expert for the ordered scheme), so no reset launch stands between it and the dispatch.
+  const bool prepared = p->cfg.T > 0;
+  const PrepArgs prep = make_prep(p, s.expert_count, s.tile_expert, s.src_info, s.tile_count, s.rows_done);
+  auto cuda_failed = [&](int step) {
+    p->cuda_error = (int)cudaGetLastError();
+    p->cuda_error_step = step;
     return MOE_ERR_CUDA;
+  };
+  if (launch_route(p, d_x, d_wr, d_bias, s.topk_idx, s.topk_w, prepared ? &prep : nullptr, st)) return cuda_failed(1);
+  mark(p, 1, st);
+  // Overlapped form: the dispatch runs inside the expert kernel's launch (ordered scheme, tensor-core kernel).
+  const moe_config_t& c = p->cfg;
+  const bool overlap = c.overlap != 0 && prepared && c.dispatch_mode == MOE_DISPATCH_ATOMIC_ORDERED &&
+                       !c.identity_experts && c.dtype == MOE_DTYPE_BF16 && c.ffn_kernel == 0;
+  if (!overlap && launch_dispatch(p, d_x, s.topk_idx, s.recv, s.expert_count, s.tile_expert, s.src_info, s.slot_of,
+                                  s.tile_count, s.rows_done, prepared, st))
+    return cuda_failed(2);
   mark(p, 2, st);
-  if (!p->cfg.identity_experts) {
+  if (overlap) {
+    int rc = launch_ffn_tc(p, s.recv, s.tile_expert, d_wg, d_wu, d_wd, s.out_rows, s.tile_count, s.rows_done, st, d_x,
+                           s.topk_idx);
+    if (rc != 0) return rc < 0 && rc != MOE_ERR_CUDA ? rc : cuda_failed(3);
+  } else if (!p->cfg.identity_experts) {
     int rc = ffn_dispatch(p, s.recv, s.tile_expert, d_wg, d_wu, d_wd, s.out_rows, s.tile_count, s.rows_done, st);
-    if (rc != 0) return rc < 0 ? rc : MOE_ERR_CUDA;
+    if (rc != 0) return rc < 0 && rc != MOE_ERR_CUDA ? rc : cuda_failed(3);
   } else {
     mark(p, 3, st);
     mark(p, 4, st);
   }
   mark(p, 5, st);
-  if (launch_combine(p, s.out_rows, s.slot_of, s.topk_w, d_y, st)) return MOE_ERR_CUDA;
+  if (launch_combine(p, s.out_rows, s.slot_of, s.topk_w, d_y, st)) return cuda_failed(4);
   mark(p, 6, st);
+  return MOE_OK;
+}
+
+int moe_last_cuda_error(moe_plan_t* p, int32_t* step, const char** name) {
+  if (!p) return MOE_ERR_ARG;
+  if (step) *step = p->cuda_error_step;
+  if (name) *name = cudaGetErrorName((cudaError_t)p->cuda_error);
   return MOE_OK;
 }
 
@@ -394,6 +437,7 @@ const char* moe_strerror(int code) {
     case MOE_ERR_TIMEOUT: return "bounded device-side wait ran out";
     case MOE_ERR_WORKSPACE: return "workspace too small or misaligned";
     case MOE_ERR_TOO_LARGE: return "T or E beyond the fixed scratch of moe_dispatch_noalloc";
+    case MOE_ERR_INTERNAL: return "a kernel's own index check failed";
     default: return "unknown error";
   }
 }

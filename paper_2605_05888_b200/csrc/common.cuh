@@ -30,6 +30,10 @@ struct Scratch {          // device pointers carved out of the caller's workspac
   int* cta_count;         // [nblk * E] mode 0: per token-block histogram
   int* cta_base;          // [nblk * E] mode 0: exclusive prefix inside the expert
   int* tile_base;         // [E + 1]    mode 0: first pool tile of each expert
+  int* hist;              // [E]   mode 3: rows per expert, counted by the router (or a counting pass) before the dispatch;
+                          //       zero between calls (the dispatch puts it back)
+  int* row_pointer;       // [E]   mode 3: next free LocalRowID per expert
+  int* ord_exit;          // [2]   mode 3: CTAs that left the dispatch kernel / the fused kernel
   unsigned long long* clock_probe;  // [2] cycles, nanoseconds of CTA 0 inside the tensor-core kernels
   unsigned long long* avail_ns;  // [P+2] availability trace (measurement): dispatch start, all-ready time, per-tile ready time
   unsigned long long* item_ns;   // [4 * P * (NB1 + NB2)] work-item timeline of the tensor-core expert kernel (measurement)
@@ -50,6 +54,27 @@ struct Scratch {          // device pointers carved out of the caller's workspac
 
 }  // namespace moehub
 
+namespace moehub {
+// What the kernel that runs right before a dispatch does on the side (inside moe_layer that kernel is the
+// router, so no reset launch stands between the two): it puts the per-call counters and tables into their
+// start state and, for the ordered scheme, adds its part of the experts' row counts to hist.
+struct PrepArgs {
+  struct Fill { int* ptr; int n; int value; };
+  Fill fill[9];
+  int nfill;                     // 0: nothing to do
+  unsigned long long* avail_ns;  // [avail_n] availability trace to re-arm, or nullptr
+  int avail_n;
+  int* hist;                     // [E] rows per expert (ordered dispatch), or nullptr
+  int E;
+};
+__device__ __forceinline__ void prep_reset(const PrepArgs& a, int gtid, int gthreads) {
+  for (int j = 0; j < a.nfill; ++j)
+    for (int i = gtid; i < a.fill[j].n; i += gthreads) a.fill[j].ptr[i] = a.fill[j].value;
+  if (a.avail_ns != nullptr)
+    for (int i = gtid; i < a.avail_n; i += gthreads) a.avail_ns[i] = i == 0 ? ~0ull : 0ull;
+}
+}  // namespace moehub
+
 struct moe_plan {
   moe_config_t cfg;
   int64_t P;                 // pool tiles
@@ -57,6 +82,7 @@ struct moe_plan {
   int tiles_per_expert;      // paged tile-table width
   int dispatch_tokens;       // tokens per dispatch CTA
   int nblk;                  // dispatch CTAs
+  int ord_tokens, ord_nblk;  // mode 3: tokens per token block, token blocks
   int device;
   int sm_count;
   int launches;
@@ -67,6 +93,8 @@ struct moe_plan {
   cudaStream_t copy_in, copy_out;
   cudaEvent_t ev_in[2], ev_done[2], ev_out[2];
   long long submitted;       // steps submitted so far
+  int cuda_error;            // last CUDA error a call of this plan met (cudaError_t), 0 if none
+  int cuda_error_step;       // which step of moe_layer met it: 1 router, 2 dispatch, 3 experts, 4 combine
   int timing;                // moe_layer_timed: record an event after every kernel of the layer
   int trace;                 // moe_availability_trace: the dispatch kernels write avail_ns
   cudaEvent_t tev[MOE_STAGE_COUNT + 1];
@@ -105,22 +133,25 @@ inline cudaError_t launch_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, siz
 // set" flag of a kernel is kept per device (a process may hold plans on several GPUs).  Setting it twice
 // is harmless, so concurrent first calls need no lock.
 struct SmemAttrOnce {
-  bool done[64] = {};
+  size_t set[64] = {};  // bytes the attribute was last set to, per device
 };
 template <typename Kern>
 inline cudaError_t ensure_dynamic_smem(Kern kern, size_t bytes, int device, SmemAttrOnce& once) {
-  if (device >= 0 && device < 64 && once.done[device]) return cudaSuccess;
+  if (device >= 0 && device < 64 && once.set[device] >= bytes) return cudaSuccess;
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
-  if (e == cudaSuccess && device >= 0 && device < 64) once.done[device] = true;
+  if (e == cudaSuccess && device >= 0 && device < 64) once.set[device] = bytes;
   return e;
 }
 
 // ---- launchers (defined in the other .cu files); each returns a cudaError_t as int ------------
+// prep: the per-call resets and the row counts of an ordered dispatch that follows (nullptr: none).
 int launch_route(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
-                 float* topk_w, cudaStream_t st);
+                 float* topk_w, const PrepArgs* prep, cudaStream_t st);
+// prepared: the kernel before this call has already done what make_prep() describes.
 int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv, int* expert_count,
                     int* tile_expert, int* src_info, int* slot_of, int* tile_count, int* rows_done,
-                    cudaStream_t st);
+                    bool prepared, cudaStream_t st);
+PrepArgs make_prep(moe_plan* p, int* expert_count, int* tile_expert, int* src_info, int* tile_count, int* rows_done);
 int launch_combine(moe_plan* p, const void* rows, const int* slot_of, const float* topk_w, void* y,
                    cudaStream_t st);
 int launch_ffn_simt(moe_plan* p, const void* recv, const int* tile_expert, const void* wg,
@@ -129,7 +160,8 @@ int launch_ffn_simt(moe_plan* p, const void* recv, const int* tile_expert, const
 // (nullptr: the rows are complete when the kernel starts).
 int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const void* wg,
                   const void* wu, const void* wd, void* out_rows, const int* tile_count,
-                  const int* rows_done, cudaStream_t st);
+                  const int* rows_done, cudaStream_t st, const void* overlap_x = nullptr,
+                  const int* overlap_idx = nullptr);
 
 // ---- element helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ float to_float(float v) { return v; }

@@ -17,7 +17,7 @@
 // Row movement is the same in every mode: one warp per token reads the row once with 16-byte
 // vectors (several in flight per lane) and stores it to its K slots; the slot indices are staged
 // in shared memory first so the copy loop has no dependent index loads.
-#include "common.cuh"
+#include "dispatch_ordered.cuh"
 
 namespace moehub {
 
@@ -340,50 +340,138 @@ dispatch_atomic_kernel(const uint4* __restrict__ x, const int* __restrict__ topk
 }
 
 // ------------------------------------------------------------------------------------------------
-// One launch that puts every per-call counter and table into its start state.
+// The per-call start state of every dispatch scheme (counters, tile owners, source info, tile table: see
+// make_prep) and, for the ordered scheme, the rows per expert.  When a dispatch is called on its own this
+// small pass does it; inside moe_layer the router does it on the side and this launch does not exist.
 __global__ void __launch_bounds__(kDispThreads)
-reset_kernel(int* __restrict__ counters, int n_counters, int* __restrict__ expert_count, int E,
-             int* __restrict__ tile_expert, int P, int* __restrict__ src_info, int n_src,
-             int* __restrict__ tile_table, int n_table, int* __restrict__ tile_count,
-             int* __restrict__ rows_done, int* __restrict__ gemm1_done, unsigned long long* __restrict__ avail_ns) {
-  const int stride = gridDim.x * kDispThreads;
-  const int i0 = blockIdx.x * kDispThreads + threadIdx.x;
+prep_count_kernel(const PrepArgs prep, const int* __restrict__ topk_idx, int n_assign, int K) {
+  __shared__ int s_hist[kMaxExperts];
+  for (int e = threadIdx.x; e < kMaxExperts; e += kDispThreads) s_hist[e] = 0;
+  __syncthreads();
   pdl_wait();
   pdl_trigger();
-  for (int i = i0; i < n_counters; i += stride) counters[i] = 0;
-  if (i0 == 0) *rows_done = 0;
-  if (i0 < 4) gemm1_done[P + i0] = 0;  // the expert kernel's item and exit counters
-  if (avail_ns != nullptr)
-    for (int i = i0; i < P + 2; i += stride) avail_ns[i] = i == 0 ? ~0ull : 0ull;
-  for (int i = i0; i < E; i += stride) expert_count[i] = 0;
-  for (int i = i0; i < P; i += stride) {
-    tile_expert[i] = -1;
-    tile_count[i] = 0;
-    gemm1_done[i] = 0;
+  const int gtid = blockIdx.x * kDispThreads + threadIdx.x, gthreads = gridDim.x * kDispThreads;
+  prep_reset(prep, gtid, gthreads);
+  if (prep.hist == nullptr) return;
+  for (int a = gtid; a < n_assign; a += gthreads) {
+    const int e = topk_idx[a];
+    if (e >= 0 && e < prep.E) atomicAdd(&s_hist[e], 1);  // ids that are no expert are reported by the dispatch itself
   }
-  for (int i = i0; i < n_table; i += stride) tile_table[i] = -1;
-  for (int i = i0; i < n_src; i += stride) src_info[i] = -1;
+  __syncthreads();
+  for (int e = threadIdx.x; e < prep.E; e += kDispThreads)
+    if (s_hist[e] != 0) atomicAdd(&prep.hist[e], s_hist[e]);
+}
+
+__global__ void __launch_bounds__(kDispThreads, 2)
+dispatch_ordered_kernel(const OrderedParams prm, int* __restrict__ hist_rw, int* __restrict__ exit_counter) {
+  extern __shared__ uint8_t ord_smem_raw[];
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(ord_smem_raw) + 127) & ~(uintptr_t)127);
+  __shared__ OrdShared sh;
+  pdl_wait();
+  pdl_trigger();
+  dispatch_ordered_cta<kDispThreads>(prm, sh, ring, blockIdx.x, gridDim.x);
+  // Every CTA has read hist by now; the last one to leave clears it for the next call's counting.
+  if (threadIdx.x == 0) sh.index_abort = atomicAdd(exit_counter, 1) == (int)gridDim.x - 1;
+  __syncthreads();
+  if (sh.index_abort) {
+    for (int e = threadIdx.x; e < prm.E; e += kDispThreads) hist_rw[e] = 0;
+    if (threadIdx.x == 0) *exit_counter = 0;
+  }
+}
+
+PrepArgs make_prep(moe_plan* p, int* expert_count, int* tile_expert, int* src_info, int* tile_count, int* rows_done) {
+  const moe_config_t& c = p->cfg;
+  const int P = (int)p->P;
+  PrepArgs a = {};
+  auto add = [&](int* ptr, long long n, int value) {
+    if (ptr != nullptr && n > 0) a.fill[a.nfill++] = PrepArgs::Fill{ptr, (int)n, value};
+  };
+  add(p->s.status, (long long)(p->counters_bytes / sizeof(int)), 0);  // status, pool cursor, scan ticket, global counter
+  add(rows_done, 1, 0);
+  add(tile_count, P, 0);
+  add(p->s.gemm1_done, P + 4, 0);
+  if (c.dispatch_mode == MOE_DISPATCH_ATOMIC_ORDERED) {
+    add(p->s.row_pointer, c.E, 0);  // expert_count, tile_expert and the empty slots' source info are written by the dispatch
+    a.hist = p->s.hist;
+  } else {
+    add(expert_count, c.E, 0);
+    add(tile_expert, P, -1);
+    add(src_info, (long long)P * kTileRows, -1);
+    if (c.dispatch_mode == MOE_DISPATCH_ATOMIC_PAGED) add(p->s.tile_table, (long long)c.E * p->tiles_per_expert, -1);
+  }
+  a.E = c.E;
+  a.avail_ns = p->trace ? p->s.avail_ns : nullptr;
+  a.avail_n = P + 2;
+  return a;
+}
+
+OrderedParams make_ordered_params(moe_plan* p, const void* x, const int* topk_idx, void* recv, int* expert_count,
+                                  int* tile_expert, int* src_info, int* slot_of, int* tile_count, int* rows_done) {
+  const moe_config_t& c = p->cfg;
+  OrderedParams q;
+  q.x = (const uint8_t*)x;
+  q.topk_idx = topk_idx;
+  q.T = c.T;
+  q.E = c.E;
+  q.K = c.K;
+  q.P = (int)p->P;
+  q.row_bytes = c.H * (c.dtype == MOE_DTYPE_BF16 ? 2 : 4);
+  q.tok_per_blk = p->ord_tokens;
+  q.nblk = p->ord_nblk;
+  q.ring_bytes = kOrdRingBytes;
+  q.hist = p->s.hist;
+  q.row_pointer = p->s.row_pointer;
+  q.recv = (uint8_t*)recv;
+  q.src_info = src_info;
+  q.slot_of = slot_of;
+  q.expert_count = expert_count;
+  q.tile_expert = tile_expert;
+  q.tile_count = tile_count;
+  q.rows_done = rows_done;
+  q.status = p->s.status;
+  q.avail_ns = p->trace ? p->s.avail_ns : nullptr;
+  q.wait_ns = c.wait_limit_ns ? c.wait_limit_ns : kDefaultWaitNs;
+  return q;
+}
+
+static int launch_dispatch_ordered(moe_plan* p, const void* x, const int* topk_idx, void* recv, int* expert_count,
+                                   int* tile_expert, int* src_info, int* slot_of, int* tile_count, int* rows_done,
+                                   cudaStream_t st) {
+  const moe_config_t& c = p->cfg;
+  OrderedParams q = make_ordered_params(p, x, topk_idx, recv, expert_count, tile_expert, src_info, slot_of, tile_count,
+                                        rows_done);
+  // Two CTAs per SM, each with half of the shared memory for its ring: one thread per CTA issues the bulk
+  // copies, and two issuing threads per SM move small rows faster than one.
+  q.ring_bytes = 96 * 1024;
+  const size_t smem = (size_t)ord_ring(q.row_bytes, q.ring_bytes) * ord_buf_bytes(q.row_bytes) + 128;
+  static SmemAttrOnce once;
+  if (ensure_dynamic_smem(dispatch_ordered_kernel, smem, p->device, once) != cudaSuccess) return (int)cudaErrorInvalidValue;
+  const int grid = max(1, min(2 * p->sm_count, q.nblk));
+  launch_pdl(dispatch_ordered_kernel, dim3(grid), dim3(kDispThreads), smem, st, q, p->s.hist, p->s.ord_exit);
+  p->launches += 1;
+  return (int)cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------------
 int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv, int* expert_count,
                     int* tile_expert, int* src_info, int* slot_of, int* tile_count, int* rows_done,
-                    cudaStream_t st) {
+                    bool prepared, cudaStream_t st) {
   const moe_config_t& c = p->cfg;
   const int eb = c.dtype == MOE_DTYPE_BF16 ? 2 : 4;
   const int vec_per_row = c.H * eb / 16;
-  // Per-call reset in one launch: scratch counters and tile table, the caller's counters, owner and
-  // source arrays.
-  {
-    const int table = c.dispatch_mode == MOE_DISPATCH_ATOMIC_PAGED ? c.E * p->tiles_per_expert : 0;
-    const long long most = max((long long)p->P * kTileRows, (long long)table);
-    const int grid = (int)max(1ll, (most + 4 * kDispThreads - 1) / (4 * kDispThreads));
-    launch_pdl(reset_kernel, dim3(grid), dim3(kDispThreads), 0, st, p->s.status,
-               (int)(p->counters_bytes / sizeof(int)), expert_count, c.E, tile_expert, (int)p->P, src_info,
-               (int)(p->P * kTileRows), p->s.tile_table, table, tile_count, rows_done, p->s.gemm1_done, p->trace ? p->s.avail_ns : nullptr);
+  // Per-call start state (and, for the ordered scheme, the rows per expert): done by the kernel before this
+  // call when `prepared`, else by one small launch here.
+  if (!prepared) {
+    const PrepArgs prep = make_prep(p, expert_count, tile_expert, src_info, tile_count, rows_done);
+    const long long work = max((long long)p->P * kTileRows, (long long)c.T * c.K);
+    const int grid = (int)max(1ll, min((long long)4 * p->sm_count, (work + 4 * kDispThreads - 1) / (4 * kDispThreads)));
+    launch_pdl(prep_count_kernel, dim3(grid), dim3(kDispThreads), 0, st, prep, topk_idx, c.T * c.K, c.K);
     p->launches += 1;
   }
   if (c.T == 0) return 0;
+  if (c.dispatch_mode == MOE_DISPATCH_ATOMIC_ORDERED)
+    return launch_dispatch_ordered(p, x, topk_idx, recv, expert_count, tile_expert, src_info, slot_of, tile_count,
+                                   rows_done, st);
   const int nblk = p->nblk, tpb = p->dispatch_tokens;
   if (c.dispatch_mode == MOE_DISPATCH_SCAN) {
     launch_maybe_pdl(false, hist_kernel, dim3(nblk), dim3(kDispThreads), sizeof(int) * c.E, st, topk_idx, c.T, c.E, c.K, tpb,

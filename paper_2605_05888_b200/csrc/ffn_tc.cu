@@ -31,9 +31,20 @@
 // warps 2-5 = epilogue (TMEM lane quarter = warp % 4).  Every wait is bounded in time; on expiry
 // the CTA records MOE_ERR_TIMEOUT, drains its outstanding TMA copies (bounded), frees its TMEM and
 // returns.
-#include "tc_common.cuh"
+#include "dispatch_ordered.cuh"
 
 namespace moehub {
+
+// The producer side of the overlapped form: with ord.x != nullptr the launch has n_dispatch more CTAs than
+// SMs; its first n_dispatch CTAs only run the ordered dispatch (dispatch_ordered.cuh) and leave, the others
+// are consumers that start on a tile when its status counter reaches the number of rows the tile will hold
+// (the last n_dispatch of them become resident as the producers leave).
+struct OverlapParams {
+  OrderedParams ord;
+  int n_dispatch;
+  int gate_all;  // consumers wait for the WHOLE dispatch (global counter) instead of their tile's counter
+  int* hist_rw;  // [E] the row counts, cleared by the last CTA to leave
+};
 
 // ---- the grouped GEMM -----------------------------------------------------------------------
 // Items are handed out dynamically: a CTA takes the next unclaimed item of the list, its first one
@@ -61,7 +72,7 @@ __global__ void __launch_bounds__(kTcThreads, 1)
 ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant__ CUtensorMap map_bg,
               const __grid_constant__ CUtensorMap map_bu, const __grid_constant__ CUtensorMap map_a2,
               const __grid_constant__ CUtensorMap map_bd, const __grid_constant__ CUtensorMap map_a1t,
-              const __grid_constant__ CUtensorMap map_a2t, const FfnParams prm) {
+              const __grid_constant__ CUtensorMap map_a2t, const FfnParams prm, const OverlapParams ov) {
   const int phase = prm.phase, E = prm.E, F = prm.F, H = prm.H;
   __nv_bfloat16* __restrict__ inter = prm.inter;
   __nv_bfloat16* __restrict__ out = prm.out;
@@ -73,7 +84,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   extern __shared__ uint8_t smem_raw[];
   uint8_t* stage_base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   TcShared* sh = reinterpret_cast<TcShared*>(stage_base + kStages * kStageBytes);
-  __shared__ WorkList wl;
+  __shared__ __align__(16) WorkList wl;  // a producer CTA keeps the dispatch's bookkeeping (with its mbarriers) here first
 
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const int nseg = 2 * E;
@@ -96,10 +107,20 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   pdl_wait();  // everything above needs no global data and overlaps the predecessor's tail
+  const bool producer_cta = ov.ord.x != nullptr && (int)blockIdx.x < ov.n_dispatch;
+  if (producer_cta) {
+    // A producer CTA: dispatch this CTA's share of the token blocks.  The buffer ring is the stage area and the
+    // dispatch's bookkeeping sits in the work list's place; every bulk copy has completed when the call
+    // returns.  Afterwards the CTA takes no work item: it only goes through the common tear-down.
+    __syncthreads();
+    dispatch_ordered_cta<kTcThreads>(ov.ord, *reinterpret_cast<OrdShared*>(&wl), stage_base, (int)blockIdx.x, ov.n_dispatch);
+    __syncthreads();
+  }
   int* work_counter = prm.work_counter + (phase == 2 ? 1 : 0);
   int first_claim = 0;
-  if (threadIdx.x == 0) first_claim = atomicAdd(work_counter, 1);  // in flight while the work list is built
-  build_worklist(wl, prm.tile_expert, prm.P, E, (F + 127) / 128, (H + 255) / 256, prm.lag, prm.fused, 1, prm.hot_min);
+  if (threadIdx.x == 0 && !producer_cta) first_claim = atomicAdd(work_counter, 1);  // in flight while the work list is built
+  build_worklist(wl, prm.tile_expert, prm.P, E, (F + 127) / 128, (H + 255) / 256, prm.lag, prm.fused, 1, prm.hot_min,
+                 prm.hist, prm.hot_first);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -172,14 +193,43 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       const uint64_t pol_stream = l2_policy_evict_first();
       for (int local_item = 0; !fail_site; ++local_item) {
         const int slot = local_item & (kItemRing - 1);
-        if (item >= item_end) {
+        if (item >= item_end || producer_cta) {
           item_ring[slot] = -1;
           mbar_arrive(smem_u32(&sh->item_bar[slot]));
           break;
         }
         const int next_item = item_begin + atomicAdd(work_counter, 1);  // used after this item's loads
         const Item it = decode(item);
-        if (it.type == 0 && tile_count != nullptr) {
+        if (it.tile < 0 || it.tile >= prm.P || it.e < 0 || it.e >= E) {  // own index check on what the work list gave
+          set_status(status, MOE_ERR_INTERNAL, 201);
+          fail_site = kWaitItem;
+          break;
+        }
+        // Rows the tile will hold, when the work list was built from the experts' row counts: the threshold of
+        // its status counter (a partly filled last tile is ready as soon as ITS rows have arrived).
+        int tile_rows = -1;
+        if (wl.count[it.e] >= 0) tile_rows = min(kTileRows, wl.count[it.e] - (it.tile - wl.estart[it.e]) * kTileRows);
+        if (it.type == 0 && tile_count != nullptr && tile_rows >= 0 && ov.gate_all) {
+          if (ld_acquire(rows_done) < total_rows) {
+            const unsigned long long t0 = globaltimer();
+            while (ld_acquire(rows_done) < total_rows) {
+              if (*abort_flag || globaltimer() - t0 > wait_ns) { fail_site = kWaitTileReady; break; }
+              __nanosleep(64);
+            }
+            if (fail_site) break;
+          }
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+        } else if (it.type == 0 && tile_count != nullptr && tile_rows >= 0) {
+          if (ld_acquire(&tile_count[it.tile]) < tile_rows) {
+            const unsigned long long t0 = globaltimer();
+            while (ld_acquire(&tile_count[it.tile]) < tile_rows) {
+              if (*abort_flag || globaltimer() - t0 > wait_ns) { fail_site = kWaitTileReady; break; }
+              __nanosleep(64);
+            }
+            if (fail_site) break;
+          }
+          asm volatile("fence.proxy.async.global;" ::: "memory");
+        } else if (it.type == 0 && tile_count != nullptr) {
           // Availability of this tile's rows (dispatch side): 128 rows stored, or every assignment of
           // the batch stored (then a partly filled tile is final).
           if (ld_acquire(&tile_count[it.tile]) < kTileRows && ld_acquire(rows_done) < total_rows) {
@@ -219,7 +269,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
         unsigned long long* trace = prm.item_ns ? prm.item_ns + 4 * (size_t)item : nullptr;
         int n16 = 0;
         if (tile_count != nullptr) {
-          const int r = tile_count[it.tile];
+          const int r = tile_rows >= 0 ? tile_rows : tile_count[it.tile];
           if (r <= kThinRows && it.m == 1 && prm.thin) n16 = max(1, (r + 15) / 16);
           else if (r <= kThinRows) n16 = kHalfForm;  // the short last tile of a larger expert: M = 64 MMAs
         }
@@ -473,6 +523,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     // dispatch result) then waits for ITS OWN GEMM1 blocks instead of finding the old counts.
     for (int pt = threadIdx.x; pt < prm.P; pt += kTcThreads) gemm1_done[pt] = 0;
   }
+  if (sh->last_cta && ov.ord.x != nullptr) {
+    // the launch that carried the dispatch: every CTA has read the row counts; clear them for the next call
+    for (int e = threadIdx.x; e < E; e += kTcThreads) ov.hist_rw[e] = 0;
+  }
   if (warp == 1)
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
 }
@@ -520,8 +574,14 @@ static int make_map_3d(EncodeTiledFn enc, CUtensorMap* m, const void* base, uint
   return r == CUDA_SUCCESS ? MOE_OK : MOE_ERR_CUDA;
 }
 
+OrderedParams make_ordered_params(moe_plan* p, const void* x, const int* topk_idx, void* recv, int* expert_count,
+                                  int* tile_expert, int* src_info, int* slot_of, int* tile_count, int* rows_done);
+
+// overlap_x / overlap_idx != nullptr: the overlapped form - the launch that runs the GEMM1 items also
+// dispatches x (ordered scheme, into recv and the plan's own dispatch outputs) on its first CTAs.
 int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const void* wg, const void* wu,
-                  const void* wd, void* out_rows, const int* tile_count, const int* rows_done, cudaStream_t st) {
+                  const void* wd, void* out_rows, const int* tile_count, const int* rows_done, cudaStream_t st,
+                  const void* overlap_x, const int* overlap_idx) {
   const moe_config_t& c = p->cfg;
   if (p->P == 0 || c.T == 0) return 0;
   EncodeTiledFn enc;
@@ -582,10 +642,40 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   prm.status = p->s.status;
   prm.clock_probe = reinterpret_cast<unsigned long long*>(p->s.clock_probe);
   prm.item_ns = (p->trace && !pairs) ? p->s.item_ns : nullptr;
+  prm.hist = nullptr;
+  prm.hot_first = 0;
+  OverlapParams ov = {};
+  const bool overlap = overlap_x != nullptr && !pairs;
+  if (overlap) {
+    Scratch& s = p->s;
+    ov.ord = make_ordered_params(p, overlap_x, overlap_idx, s.recv, s.expert_count, s.tile_expert, s.src_info, s.slot_of,
+                                 s.tile_count, s.rows_done);
+    ov.ord.ring_bytes = kStages * kStageBytes;
+    // Producer CTAs: enough of them to keep HBM busy with the row copies (half of the SMs move about 85 % of
+    // what all of them do), the rest start on expert tiles at once.
+    ov.gate_all = c.overlap < 0 ? 1 : 0;
+    ov.n_dispatch = c.overlap > 1 ? min(c.overlap, grid - 1) : grid / 2;
+    ov.n_dispatch = max(1, min(ov.n_dispatch, ov.ord.nblk));
+    ov.hist_rw = s.hist;
+  }
   auto launch = [&](int phase) -> int {
     prm.phase = phase;
     if (pairs) return launch_ffn_tc2_kernel(a1, bg, bu, a2, bd, prm, grid, st);
-    return launch_pdl(ffn_tc_kernel, dim3(grid), dim3(kTcThreads), kTcSmem, st, a1, bg, bu, a2, bd, a1t, a2t, prm) == cudaSuccess
+    OverlapParams ovp = {};
+    if (overlap && phase != 2) {
+      // The launch that carries the dispatch: its work list comes from the row counts (no tile owner is
+      // written yet), hottest experts first.  One CTA per SM and CTAs start in index order, so the producer
+      // CTAs (the lowest indices) are resident before any consumer waits for their rows; a consumer's wait is
+      // bounded in any case.
+      ovp = ov;
+      prm.hist = p->s.hist;
+      prm.hot_first = 1;
+      return launch_pdl(ffn_tc_kernel, dim3(grid + ov.n_dispatch), dim3(kTcThreads), kTcSmem, st, a1, bg, bu, a2, bd, a1t, a2t, prm,
+                        ovp) == cudaSuccess ? 0 : MOE_ERR_CUDA;
+    }
+    prm.hist = nullptr;
+    prm.hot_first = 0;
+    return launch_pdl(ffn_tc_kernel, dim3(grid), dim3(kTcThreads), kTcSmem, st, a1, bg, bu, a2, bd, a1t, a2t, prm, ovp) == cudaSuccess
                ? 0 : MOE_ERR_CUDA;
   };
   if (fused) {

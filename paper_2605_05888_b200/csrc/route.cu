@@ -20,9 +20,10 @@ namespace moehub {
 // One warp per token: the token's logits sit in registers (EP/32 per lane); K rounds of a shuffle
 // arg-max on (value, lowest index); then the softmax weights of the picks.  ls: [tokens][EP] logits
 // in shared memory.
+// s_hist (shared memory, [E], or nullptr): every pick is also counted per expert.
 template <int EP>
 __device__ __forceinline__ void select_topk(const float* ls, int tvalid, int t0, int E, int K, int renorm,
-                                            int* __restrict__ topk_idx, float* __restrict__ topk_w) {
+                                            int* __restrict__ topk_idx, float* __restrict__ topk_w, int* s_hist) {
   constexpr int NJ = (EP + 31) / 32;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   for (int tl = warp; tl < tvalid; tl += blockDim.x / 32) {
@@ -71,8 +72,24 @@ __device__ __forceinline__ void select_topk(const float* ls, int tvalid, int t0,
     if (lane < K) {
       topk_idx[(size_t)(t0 + tl) * K + lane] = my_e;
       topk_w[(size_t)(t0 + tl) * K + lane] = p;
+      if (s_hist != nullptr) atomicAdd(&s_hist[my_e], 1);
     }
   }
+}
+
+// The side job of a router that is followed by an ordered dispatch (see PrepArgs): before the chains, clear
+// the per-call counters; after the picks, add this CTA's rows per expert to the global counts.
+constexpr int kRouteMaxExperts = 256;
+__device__ __forceinline__ void route_prep_begin(const PrepArgs& prep, int* s_hist) {
+  if (prep.nfill == 0) return;
+  for (int e = threadIdx.x; e < kRouteMaxExperts; e += blockDim.x) s_hist[e] = 0;
+  prep_reset(prep, blockIdx.x * blockDim.x + threadIdx.x, gridDim.x * blockDim.x);
+}
+__device__ __forceinline__ void route_prep_end(const PrepArgs& prep, const int* s_hist) {
+  if (prep.hist == nullptr) return;
+  __syncthreads();
+  for (int e = threadIdx.x; e < prep.E; e += blockDim.x)
+    if (s_hist[e] != 0) atomicAdd(&prep.hist[e], s_hist[e]);
 }
 
 // The compute-bound shape (64 < E <= 256): up to 64 tokens x 256 experts per CTA.  Four compute warps
@@ -124,9 +141,11 @@ struct WideChunk {
 template <typename XT, int TMT>
 __global__ void __launch_bounds__(kWideThreads)
 route_wide_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias, int T,
-                  int H, int E, int K, int renorm, int* __restrict__ topk_idx, float* __restrict__ topk_w) {
+                  int H, int E, int K, int renorm, int* __restrict__ topk_idx, float* __restrict__ topk_w,
+                  const PrepArgs prep) {
   constexpr int TB = 8 * TMT;  // tokens per CTA: 4 warps x 2 lane groups x TMT
   extern __shared__ __align__(16) float smem[];
+  __shared__ int s_hist[kRouteMaxExperts];
   float* ls = smem;  // [TB][256] after the h loop
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   const bool computes = warp < kWideComputeWarps;
@@ -154,6 +173,7 @@ route_wide_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const flo
   WideChunk<XT, kWideEP> wrg[P];
   pdl_wait();
   pdl_trigger();
+  route_prep_begin(prep, s_hist);
   if (!computes) {  // chunk 0 into buffer 0, chunks 1..P into the registers (slot = chunk % P)
     xr[0].load(ft, x, x_row, H, 0);
     wrg[0].load(ft, wr, w_row, H, 0);
@@ -234,12 +254,13 @@ route_wide_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const flo
     }
   }
   __syncthreads();
-  select_topk<kWideEP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w);
+  select_topk<kWideEP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w, prep.hist ? s_hist : nullptr);
+  route_prep_end(prep, s_hist);
 }
 
 template <typename XT, int TMT>
 static int launch_wide_tmt(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
-                           float* topk_w, cudaStream_t st) {
+                           float* topk_w, const PrepArgs& prep, cudaStream_t st) {
   constexpr size_t stage = sizeof(float) * 2 * kWideBuf, logits = sizeof(float) * 8 * TMT * kWideEP;
   constexpr size_t smem = stage > logits ? stage : logits;
   auto kern = route_wide_kernel<XT, TMT>;
@@ -248,12 +269,12 @@ static int launch_wide_tmt(moe_plan* p, const void* x, const void* wr, const flo
   const moe_config_t& c = p->cfg;
   p->launches += 1;
   return (int)launch_maybe_pdl(false, kern, dim3((c.T + 8 * TMT - 1) / (8 * TMT)), dim3(kWideThreads), smem, st,
-                               (const XT*)x, (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w);
+                               (const XT*)x, (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w, prep);
 }
 
 template <typename XT>
 static int launch_wide(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
-                       float* topk_w, cudaStream_t st) {
+                       float* topk_w, const PrepArgs& prep, cudaStream_t st) {
   // Tokens per thread: the time is (waves of CTAs over the SMs) x TMT; ties go to the larger tile.
   const int T = p->cfg.T, sms = p->sm_count > 0 ? p->sm_count : 148;
   int best = 8, best_cost = 1 << 30;
@@ -263,11 +284,11 @@ static int launch_wide(moe_plan* p, const void* x, const void* wr, const float* 
     if (cost < best_cost) { best_cost = cost; best = tmt; }
   }
   switch (best) {
-    case 4: return launch_wide_tmt<XT, 4>(p, x, wr, bias, topk_idx, topk_w, st);
-    case 5: return launch_wide_tmt<XT, 5>(p, x, wr, bias, topk_idx, topk_w, st);
-    case 6: return launch_wide_tmt<XT, 6>(p, x, wr, bias, topk_idx, topk_w, st);
-    case 7: return launch_wide_tmt<XT, 7>(p, x, wr, bias, topk_idx, topk_w, st);
-    default: return launch_wide_tmt<XT, 8>(p, x, wr, bias, topk_idx, topk_w, st);
+    case 4: return launch_wide_tmt<XT, 4>(p, x, wr, bias, topk_idx, topk_w, prep, st);
+    case 5: return launch_wide_tmt<XT, 5>(p, x, wr, bias, topk_idx, topk_w, prep, st);
+    case 6: return launch_wide_tmt<XT, 6>(p, x, wr, bias, topk_idx, topk_w, prep, st);
+    case 7: return launch_wide_tmt<XT, 7>(p, x, wr, bias, topk_idx, topk_w, prep, st);
+    default: return launch_wide_tmt<XT, 8>(p, x, wr, bias, topk_idx, topk_w, prep, st);
   }
 }
 
@@ -345,7 +366,9 @@ struct NaturalChunk {
 template <typename XT, bool SWAP, int EW, int TWP, int HC>
 __global__ void __launch_bounds__(32 * (EW * TWP + kNarrowFillWarps))
 route_narrow_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias, int T,
-                    int H, int E, int K, int renorm, int* __restrict__ topk_idx, float* __restrict__ topk_w) {
+                    int H, int E, int K, int renorm, int* __restrict__ topk_idx, float* __restrict__ topk_w,
+                    const PrepArgs prep) {
+  __shared__ int s_hist[kRouteMaxExperts];
   constexpr int TN = 2;                    // experts per lane
   constexpr int G = SWAP ? 16 : 2;         // expert groups per warp
   constexpr int TW = 32 / G;               // tokens per warp
@@ -375,6 +398,7 @@ route_narrow_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const f
   NaturalChunk<XT, EP, HC> wrg[P];
   pdl_wait();
   pdl_trigger();
+  route_prep_begin(prep, s_hist);
   if (!computes) {  // chunk 0 into buffer 0, chunks 1..P into the registers (slot = chunk % P)
     xr[0].load(ft, x, t0, tvalid, H, 0);
     wrg[0].load(ft, wr, 0, E, H, 0);
@@ -453,12 +477,13 @@ route_narrow_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const f
     }
   }
   __syncthreads();
-  select_topk<EP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w);
+  select_topk<EP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w, prep.hist ? s_hist : nullptr);
+  route_prep_end(prep, s_hist);
 }
 
 template <typename XT, bool SWAP, int EW, int TWP, int HC>
 static int launch_narrow(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
-                         float* topk_w, cudaStream_t st) {
+                         float* topk_w, const PrepArgs& prep, cudaStream_t st) {
   constexpr int G = SWAP ? 16 : 2, EP = EW * G * 2, TB = (32 / G) * TWP;
   constexpr size_t smem = sizeof(float) * (2 * (TB + EP) * (HC + 4) > TB * EP ? 2 * (TB + EP) * (HC + 4) : TB * EP);
   auto kern = route_narrow_kernel<XT, SWAP, EW, TWP, HC>;
@@ -468,29 +493,31 @@ static int launch_narrow(moe_plan* p, const void* x, const void* wr, const float
   const moe_config_t& c = p->cfg;
   p->launches += 1;
   return (int)launch_maybe_pdl(false, kern, dim3((c.T + TB - 1) / TB), dim3(32 * (EW * TWP + kNarrowFillWarps)), smem, st,
-                               (const XT*)x, (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w);
+                               (const XT*)x, (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w, prep);
 }
 
 template <typename XT>
 static int launch_typed(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
-                        float* topk_w, cudaStream_t st) {
+                        float* topk_w, const PrepArgs& prep, cudaStream_t st) {
   const moe_config_t& c = p->cfg;
   // 16 tokens x 2 expert groups per warp, two compute warps per CTA (32 tokens: T = 4096 gives 128
   // CTAs); with many experts 2 tokens x 16 groups, so that the chains still spread over the SMs.
   constexpr int HL = sizeof(XT) == 2 ? 256 : 128;  // h per chunk
-  if (c.E <= 8) return launch_narrow<XT, false, 2, 2, HL>(p, x, wr, bias, topk_idx, topk_w, st);   // 32 tokens per CTA
-  if (c.E <= 16) return launch_narrow<XT, false, 4, 2, HL>(p, x, wr, bias, topk_idx, topk_w, st);  // 32 tokens per CTA
-  if (c.E <= 32) return launch_narrow<XT, true, 1, 4, HL / 2>(p, x, wr, bias, topk_idx, topk_w, st);  // 8 tokens per CTA
-  if (c.E <= 64) return launch_narrow<XT, true, 2, 2, HL / 2>(p, x, wr, bias, topk_idx, topk_w, st);  // 4 tokens per CTA
-  return launch_wide<XT>(p, x, wr, bias, topk_idx, topk_w, st);
+  if (c.E <= 8) return launch_narrow<XT, false, 2, 2, HL>(p, x, wr, bias, topk_idx, topk_w, prep, st);   // 32 tokens per CTA
+  if (c.E <= 16) return launch_narrow<XT, false, 4, 2, HL>(p, x, wr, bias, topk_idx, topk_w, prep, st);  // 32 tokens per CTA
+  if (c.E <= 32) return launch_narrow<XT, true, 1, 4, HL / 2>(p, x, wr, bias, topk_idx, topk_w, prep, st);  // 8 tokens per CTA
+  if (c.E <= 64) return launch_narrow<XT, true, 2, 2, HL / 2>(p, x, wr, bias, topk_idx, topk_w, prep, st);  // 4 tokens per CTA
+  return launch_wide<XT>(p, x, wr, bias, topk_idx, topk_w, prep, st);
 }
 
 int launch_route(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
-                 float* topk_w, cudaStream_t st) {
+                 float* topk_w, const PrepArgs* prep_or_null, cudaStream_t st) {
   if (p->cfg.T == 0) return 0;
+  PrepArgs prep = {};
+  if (prep_or_null != nullptr) prep = *prep_or_null;
   if (p->cfg.dtype == MOE_DTYPE_BF16)
-    return launch_typed<__nv_bfloat16>(p, x, wr, bias, topk_idx, topk_w, st);
-  return launch_typed<float>(p, x, wr, bias, topk_idx, topk_w, st);
+    return launch_typed<__nv_bfloat16>(p, x, wr, bias, topk_idx, topk_w, prep, st);
+  return launch_typed<float>(p, x, wr, bias, topk_idx, topk_w, prep, st);
 }
 
 }  // namespace moehub

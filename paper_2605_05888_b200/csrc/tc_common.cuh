@@ -169,6 +169,8 @@ struct WorkList {
   int seg_start[2 * kMaxExperts + 1];
   int seg_info[2 * kMaxExperts];
   int cursor[kMaxExperts];
+  int order[kMaxExperts];  // the experts in the order their segments are placed
+  int count[kMaxExperts];  // rows per expert when the list was built from row counts, else -1
   int n1;
   int n_hot[2];
   int tiles[kMaxListTiles];
@@ -178,14 +180,36 @@ struct WorkList {
 // tiles.  fused: the GEMM2 segment of an expert follows once at least `lag` items were placed after its
 // GEMM1 segment, as long as `lag` GEMM2 items stay in reserve for the end of the list; otherwise all
 // GEMM1 segments come first.
+// hist != nullptr: the list is built from the experts' row counts instead of tile_expert - expert e then
+// owns the consecutive tiles [estart[e], estart[e + 1]) (the layout of the ordered dispatch), which is known
+// before a single row has been dispatched.  hot_first: experts are placed by descending row count (the
+// experts whose first tiles fill earliest come first) instead of by index.
 __device__ __forceinline__ void build_worklist(WorkList& wl, const int* __restrict__ tile_expert, int P, int E,
-                                               int NB1, int NB2, int lag, int fused, int pair, int hot_min = 0) {
+                                               int NB1, int NB2, int lag, int fused, int pair, int hot_min = 0,
+                                               const int* __restrict__ hist = nullptr, int hot_first = 0) {
   const int tid = threadIdx.x, nthr = blockDim.x, lane = tid % 32;
-  for (int e = tid; e < kMaxExperts; e += nthr) wl.cursor[e] = 0;
+  for (int e = tid; e < kMaxExperts; e += nthr) {
+    wl.cursor[e] = (hist != nullptr && e < E) ? (hist[e] + kTileRows - 1) / kTileRows : 0;
+    wl.count[e] = (hist != nullptr && e < E) ? hist[e] : -1;
+    wl.order[e] = e;
+  }
   __syncthreads();
-  for (int p = tid; p < P; p += nthr) {
-    const int e = tile_expert[p];
-    if (e >= 0 && e < E) atomicAdd(&wl.cursor[e], 1);
+  if (hist == nullptr) {
+    for (int p = tid; p < P; p += nthr) {
+      const int e = tile_expert[p];
+      if (e >= 0 && e < E) atomicAdd(&wl.cursor[e], 1);
+    }
+  } else if (hot_first) {
+    // position of expert e = experts with more rows, or as many and a lower index
+    for (int e = tid; e < E; e += nthr) {
+      const int c = wl.count[e];
+      int rank = 0;
+      for (int o = 0; o < E; ++o) {
+        const int co = wl.count[o];
+        rank += (co > c || (co == c && o < e)) ? 1 : 0;
+      }
+      wl.order[rank] = e;
+    }
   }
   __syncthreads();
   if (tid < 32) {  // exclusive scan of the per-expert tile counts: 8 experts per lane
@@ -214,17 +238,24 @@ __device__ __forceinline__ void build_worklist(WorkList& wl, const int* __restri
     }
     if (lane == 31) wl.estart[E] = incl;
     __syncwarp();
-    // stable scatter, 32 tiles at a time: the same list in every CTA
-    for (int p0 = 0; p0 < P; p0 += 32) {
-      const int p = p0 + lane;
-      int e = p < P ? tile_expert[p] : -1;
-      if (e >= E) e = -1;
-      const unsigned peers = __match_any_sync(0xffffffffu, e);
-      if (e >= 0) wl.tiles[wl.cursor[e] + __popc(peers & ((1u << lane) - 1u))] = p;
-      __syncwarp();
-      if (e >= 0 && lane == __ffs(peers) - 1) wl.cursor[e] += __popc(peers);
-      __syncwarp();
+    if (hist != nullptr) {
+      const int total = min(__shfl_sync(0xffffffffu, incl, 31), kMaxListTiles);
+      for (int t = lane; t < total; t += 32) wl.tiles[t] = t;  // regions are consecutive tiles
+    } else {
+      // stable scatter, 32 tiles at a time: the same list in every CTA
+      for (int p0 = 0; p0 < P; p0 += 32) {
+        const int p = p0 + lane;
+        int e = p < P ? tile_expert[p] : -1;
+        if (e >= E) e = -1;
+        const unsigned peers = __match_any_sync(0xffffffffu, e);
+        if (e >= 0) wl.tiles[wl.cursor[e] + __popc(peers & ((1u << lane) - 1u))] = p;
+        __syncwarp();
+        if (e >= 0 && lane == __ffs(peers) - 1) wl.cursor[e] += __popc(peers);
+        __syncwarp();
+      }
     }
+    __syncwarp();
+    auto tiles_of = [&](int e) { return wl.estart[e + 1] - wl.estart[e]; };
     if (lane == 0 && !fused && hot_min > 0) {
       // two passes per GEMM: hot experts, then cold ones
       int pos = 0, nseg = 0;
@@ -233,7 +264,7 @@ __device__ __forceinline__ void build_worklist(WorkList& wl, const int* __restri
         const int begin = pos;
         for (int cold = 0; cold < 2; ++cold) {
           for (int e = 0; e < E; ++e) {
-            const int m = wl.estart[e + 1] - wl.estart[e];
+            const int m = tiles_of(e);
             if ((m >= hot_min ? 0 : 1) != cold) continue;
             wl.seg_start[nseg] = pos;
             wl.seg_info[nseg++] = e | (g << 16);
@@ -246,32 +277,32 @@ __device__ __forceinline__ void build_worklist(WorkList& wl, const int* __restri
       wl.seg_start[nseg] = pos;  // nseg == 2E
     } else if (lane == 0) {
       wl.n_hot[0] = wl.n_hot[1] = -1;  // no interleaving
-      int pos = 0, nseg = 0, q = 0;
-      // GEMM2 items of experts q+1 .. E-2: what would still stand between the last expert's GEMM1 and
-      // its GEMM2 if expert q's GEMM2 segment were placed now.  Keeping `lag` items in that reserve
-      // gives the last experts the same distance as the first ones (without it their GEMM2 items
+      int pos = 0, nseg = 0, q = 0;  // i, q: positions in wl.order
+      // GEMM2 items of the experts at positions q+1 .. E-2: what would still stand between the last expert's
+      // GEMM1 and its GEMM2 if the GEMM2 segment of position q were placed now.  Keeping `lag` items in that
+      // reserve gives the last experts the same distance as the first ones (without it their GEMM2 items
       // waited up to half an item for the intermediate).
       int reserve = 0;
-      for (int j = 1; j + 1 < E; ++j) reserve += (wl.estart[j + 1] - wl.estart[j] + pair - 1) / pair * NB2;
-      for (int e = 0; e < E; ++e) {
-        const int m = wl.estart[e + 1] - wl.estart[e];
+      for (int j = 1; j + 1 < E; ++j) reserve += (tiles_of(wl.order[j]) + pair - 1) / pair * NB2;
+      for (int i = 0; i < E; ++i) {
+        const int e = wl.order[i];
         wl.seg_start[nseg] = pos;
         wl.seg_info[nseg++] = e;
-        pos += (m + pair - 1) / pair * NB1;
-        wl.cursor[e] = pos;  // end of this expert's GEMM1 items
-        while (fused && q < e && pos - wl.cursor[q] >= lag && reserve >= lag) {
+        pos += (tiles_of(e) + pair - 1) / pair * NB1;
+        wl.cursor[i] = pos;  // end of the GEMM1 items of position i
+        while (fused && q < i && pos - wl.cursor[q] >= lag && reserve >= lag) {
           wl.seg_start[nseg] = pos;
-          wl.seg_info[nseg++] = q | (1 << 16);
-          pos += (wl.estart[q + 1] - wl.estart[q] + pair - 1) / pair * NB2;
+          wl.seg_info[nseg++] = wl.order[q] | (1 << 16);
+          pos += (tiles_of(wl.order[q]) + pair - 1) / pair * NB2;
           ++q;
-          if (q + 1 < E) reserve -= (wl.estart[q + 1] - wl.estart[q] + pair - 1) / pair * NB2;
+          if (q + 1 < E) reserve -= (tiles_of(wl.order[q]) + pair - 1) / pair * NB2;
         }
       }
       wl.n1 = fused ? 0 : pos;
       for (; q < E; ++q) {
         wl.seg_start[nseg] = pos;
-        wl.seg_info[nseg++] = q | (1 << 16);
-        pos += (wl.estart[q + 1] - wl.estart[q] + pair - 1) / pair * NB2;
+        wl.seg_info[nseg++] = wl.order[q] | (1 << 16);
+        pos += (tiles_of(wl.order[q]) + pair - 1) / pair * NB2;
       }
       wl.seg_start[nseg] = pos;  // nseg == 2E
     }
@@ -284,6 +315,8 @@ struct FfnParams {
   const int* tile_expert;  // [P]
   int P, lag, fused;
   int hot_min;  // > 0: interleave tensor-bound and weight-streaming-bound items (see WorkList)
+  const int* hist;  // rows per expert (the ordered dispatch's counts): the work list is built from them, or nullptr
+  int hot_first;    // with hist: experts are walked by descending row count
   int thin;         // the narrow (transposed) form for single tiles of at most 64 rows is in use
   int cold_below;   // experts with fewer tiles than this stream their weights once: their loads are evict-first
   int phase, E, F, H;

@@ -1,6 +1,7 @@
 """Dispatch/combine-only sweep (identity experts): H = 7168, E = 256 on R = 32 logical ranks, top-8, bf16,
 T from 128 to 65536 in powers of two, unbiased and Zipf(1.2) routing.  For every point it times the
-dispatch stage (baseline scan scheme and the destination-agnostic paged scheme) and the combine stage
+dispatch stage (baseline scan scheme, the destination-agnostic paged scheme and the token-ordered
+bulk-copy scheme) and the combine stage
 with CUDA events and prints algorithmic GB/s and the fraction of the measured HBM copy bandwidth.
 
     python -m paper_2605_05888_b200.sweep [--max-t 65536] [--iters 20] [--markdown]
@@ -127,22 +128,26 @@ def main() -> None:
             comb_bytes = w.T * w.H * eb * (w.K + 1) + 8 * n
             scan = time_point(w, B.DISPATCH_SCAN, args.iters)
             paged = time_point(w, B.DISPATCH_ATOMIC_PAGED, args.iters)
+            ordered = time_point(w, B.DISPATCH_ATOMIC_ORDERED, args.iters)
             rows.append({"T": T, "routing": "zipf1.2" if zipf else "uniform", "hottest_share": paged["hottest_share"],
                          "dispatch_scan_us": 1e3 * scan["dispatch_ms"], "dispatch_paged_us": 1e3 * paged["dispatch_ms"],
+                         "dispatch_ordered_us": 1e3 * ordered["dispatch_ms"],
                          "dispatch_scan_GBps": disp_bytes / scan["dispatch_ms"] / 1e6,
                          "dispatch_paged_GBps": disp_bytes / paged["dispatch_ms"] / 1e6,
+                         "dispatch_ordered_GBps": disp_bytes / ordered["dispatch_ms"] / 1e6,
                          "combine_us": 1e3 * paged["combine_ms"], "combine_GBps": comb_bytes / paged["combine_ms"] / 1e6})
             torch.cuda.empty_cache()
         T *= 2
     if args.markdown:
         print(f"HBM copy peak: {peak:.1f} GB/s ({kind}). Times are medians of {args.iters} runs, CUDA events around the stage.")
         print()
-        print("| T | routing | hottest expert (rows/T) | dispatch scan us | GB/s | % | dispatch paged us | GB/s | % | combine us | GB/s | % |")
-        print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+        print("| T | routing | hottest expert (rows/T) | dispatch scan us | GB/s | % | dispatch paged us | GB/s | % | dispatch ordered us | GB/s | % | combine us | GB/s | % |")
+        print("|---|---|---|---|---|---|---|---|---|---|---|---|---|---|---|")
         for r in rows:
             print(f"| {r['T']} | {r['routing']} | {r['hottest_share']:.2f} | {r['dispatch_scan_us']:.1f} | "
                   f"{r['dispatch_scan_GBps']:.0f} | {100 * r['dispatch_scan_GBps'] / peak:.0f} | {r['dispatch_paged_us']:.1f} | "
-                  f"{r['dispatch_paged_GBps']:.0f} | {100 * r['dispatch_paged_GBps'] / peak:.0f} | {r['combine_us']:.1f} | "
+                  f"{r['dispatch_paged_GBps']:.0f} | {100 * r['dispatch_paged_GBps'] / peak:.0f} | {r['dispatch_ordered_us']:.1f} | "
+                  f"{r['dispatch_ordered_GBps']:.0f} | {100 * r['dispatch_ordered_GBps'] / peak:.0f} | {r['combine_us']:.1f} | "
                   f"{r['combine_GBps']:.0f} | {100 * r['combine_GBps'] / peak:.0f} |")
     else:
         for r in rows:

@@ -54,7 +54,7 @@ def check_sampled_output(w, plan, y, x, wr, bias, wg, wu, wd, n_sample, seed=0):
     return sample.size, used.size
 
 
-@pytest.mark.parametrize("mode", [B.DISPATCH_ATOMIC_PAGED, B.DISPATCH_SCAN])
+@pytest.mark.parametrize("mode", [B.DISPATCH_ATOMIC_PAGED, B.DISPATCH_SCAN, B.DISPATCH_ATOMIC_ORDERED])
 def test_c2_mixtral_like_full_size(mode):
     w = inputs.C2
     x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
@@ -65,17 +65,44 @@ def test_c2_mixtral_like_full_size(mode):
     check_sampled_output(w, plan, y, x, wr, bias, wg, wu, wd, 32)
 
 
-def test_c3_deepseek_like_full_size_skewed():
+@pytest.mark.parametrize("mode", [B.DISPATCH_ATOMIC_PAGED, B.DISPATCH_ATOMIC_ORDERED])
+def test_c3_deepseek_like_full_size_skewed(mode):
     w = inputs.C3
     x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
-    plan, y = run_layer(w, B.DISPATCH_ATOMIC_PAGED, x, wr, bias, Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd))
+    plan, y = run_layer(w, mode, x, wr, bias, Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd))
     _, d = check_full_routing_and_dispatch(w, plan, x, wr, bias)
     # the Zipf bias really skews the load: hottest expert far above the mean, some experts below one tile
     assert d["count"].max() > 8 * w.T * w.K / w.E and (d["count"] < 128).sum() > 32
     check_sampled_output(w, plan, y, x, wr, bias, wg, wu, wd, 24)
 
 
-@pytest.mark.parametrize("mode", [B.DISPATCH_SCAN, B.DISPATCH_ATOMIC_STATIC, B.DISPATCH_ATOMIC_PAGED])
+@pytest.mark.parametrize("w", [inputs.C2, inputs.C3, inputs.C4], ids=lambda w: w.name)
+def test_overlapped_launch_full_size(w):
+    """Dispatch inside the expert kernel's launch (producer CTAs emit the tokens in ascending order, consumer
+    CTAs start on a tile when its status counter reaches the rows it will hold) at the benchmark's sizes:
+    routing and dispatch in full, output on a row of every used tile; and in one traced layer the first expert
+    item begins before the last row is stored."""
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, overlap=1)
+    y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
+    args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    plan.moe_layer(*args, y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    check_full_routing_and_dispatch(w, plan, x, wr, bias)
+    check_sampled_output(w, plan, y, x, wr, bias, wg, wu, wd, 16)
+    plan.moe_availability_trace(True)
+    plan.layer_tensor(9).zero_()
+    plan.moe_layer(*args, y)
+    torch.cuda.synchronize()
+    tr = plan.layer_tensor(8).cpu().numpy()
+    items = plan.layer_tensor(9).cpu().numpy()
+    started = items[items[:, 0] > 0]
+    gemm1 = started[(started[:, 2] & 1) == 0]
+    assert gemm1[:, 0].min() < tr[1], "no expert item began before the dispatch was over"
+
+
+@pytest.mark.parametrize("mode", [B.DISPATCH_SCAN, B.DISPATCH_ATOMIC_STATIC, B.DISPATCH_ATOMIC_PAGED, B.DISPATCH_ATOMIC_ORDERED])
 def test_c4_qwen_like_full_size(mode):
     w = inputs.C4
     x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
@@ -97,18 +124,19 @@ def test_other_table2_shapes(w):
     check_sampled_output(w, plan, y, x, wr, bias, wg, wu, wd, 32)
 
 
+@pytest.mark.parametrize("mode", [B.DISPATCH_ATOMIC_PAGED, B.DISPATCH_ATOMIC_ORDERED])
 @pytest.mark.parametrize("zipf", [0.0, 1.2])
-def test_c5_sweep_point_8192_against_oracle(zipf):
+def test_c5_sweep_point_8192_against_oracle(zipf, mode):
     w = inputs.C5(8192, zipf)
     x, wr, bias, *_ = Hh.oracle_inputs(w, with_experts=False)
-    plan, y = run_layer(w, B.DISPATCH_ATOMIC_PAGED, x, wr, bias, None, None, None)
+    plan, y = run_layer(w, mode, x, wr, bias, None, None, None)
     idx, d = check_full_routing_and_dispatch(w, plan, x, wr, bias)
     _, tw, _ = oracle.route(x, wr, bias, w.K, w.dtype)
     ref = oracle.combine(oracle.identity_ffn(d["recv"], w.dtype), d["slot_of"], tw)
     Hh.assert_output_close(Hh.to_host_f64(y), ref, w.dtype)
 
 
-@pytest.mark.parametrize("mode", [B.DISPATCH_SCAN, B.DISPATCH_ATOMIC_PAGED])
+@pytest.mark.parametrize("mode", [B.DISPATCH_SCAN, B.DISPATCH_ATOMIC_PAGED, B.DISPATCH_ATOMIC_ORDERED])
 def test_c5_largest_sweep_point_properties(mode):
     """T = 65536 (8.5 GB moved per direction): checked by properties that hold at any size."""
     w = inputs.C5(65536, 1.2)

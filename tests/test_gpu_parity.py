@@ -16,7 +16,7 @@ import parity_helpers as Hh
 
 pytestmark = pytest.mark.gpu
 FP32, BF16 = inputs.FP32, inputs.BF16
-MODES = [B.DISPATCH_SCAN, B.DISPATCH_ATOMIC_STATIC, B.DISPATCH_ATOMIC_PAGED]
+MODES = [B.DISPATCH_SCAN, B.DISPATCH_ATOMIC_STATIC, B.DISPATCH_ATOMIC_PAGED, B.DISPATCH_ATOMIC_ORDERED]
 
 SMALL = [
     inputs.C1,
@@ -418,6 +418,93 @@ def test_consumer_wait_runs_out_and_reports_it(kernel):
     torch.cuda.synchronize()
     assert plan.moe_last_status() == (0, 0)
     Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+
+
+# ------------------------------------------------------------------ dispatch and experts in one launch
+OVERLAP_CASES = [SMALL[3], SMALL[4], SMALL[5], SMALL[7],
+                 inputs.Workload("three_tiles", T=700, H=320, E=4, R=2, K=2, F=392, dtype=BF16),
+                 inputs.Workload("many_items", T=2100, H=520, E=12, R=3, K=3, F=1032, dtype=BF16, seed=5, zipf_s=1.0),
+                 inputs.Workload("long_rows", T=260, H=9216, E=8, R=2, K=2, F=128, dtype=BF16)]   # rows of 18 KB: two chunks per row
+
+
+@pytest.mark.parametrize("split", [1, 2])
+@pytest.mark.parametrize("w", OVERLAP_CASES, ids=lambda w: w.name)
+def test_overlapped_dispatch_and_experts_match_oracle(w, split):
+    """Section IV-D end to end: the launch that computes the experts also dispatches (its first CTAs walk the
+    tokens in ascending order and raise the tiles' status counters, the others start on a tile when its counter
+    reaches the rows the tile will hold).  Routing, dispatch contents and output against the oracle; both as one
+    launch for the two GEMMs and as two."""
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, overlap=1, ffn_split=split)
+    y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
+    args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    for _ in range(2):      # twice: the second call meets the counters as the first one left them
+        plan.moe_layer(*args, y)
+        torch.cuda.synchronize()
+        assert plan.moe_last_status() == (0, 0)
+        assert plan.moe_last_launch_count() == 2 + (2 if split == 1 else 1)   # router, expert launch(es) carrying the dispatch, combine
+        Hh.check_route(plan.layer_tensor(0), plan.layer_tensor(1), ref["topk_idx"], ref["topk_w"])
+        Hh.check_dispatch(w, plan.P, x, ref["topk_idx"], ref, plan.layer_tensor(2), plan.layer_tensor(3),
+                          plan.layer_tensor(4), plan.layer_tensor(5), plan.layer_tensor(6))
+        Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+    # the same bytes as the stream-ordered launches give
+    plan2 = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, ffn_split=split)
+    y2 = torch.empty_like(y)
+    plan2.moe_layer(*args, y2)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y2)
+
+
+def test_overlapped_consumer_wait_runs_out_and_reports_it():
+    """The consumer's wait for a tile's status counter, in the overlapped launch, with a limit far below the time
+    the producers need (1 microsecond): waits run out, the kernel returns by itself with MOE_ERR_TIMEOUT and a
+    wait site, nothing hangs, and a plan with the normal limit then computes the right layer."""
+    w = inputs.Workload("overlap_timeout", T=4096, H=2048, E=8, R=2, K=2, F=256, dtype=BF16)
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, overlap=1, wait_limit_ns=1000)
+    y = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    plan.moe_layer(*args, y)
+    t1.record()
+    code, detail = plan.moe_last_status()
+    assert code == -6 and detail in (3, 4, 5, 7, 8), (code, detail)
+    assert t0.elapsed_time(t1) < 2000.0
+    good = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, overlap=1)
+    good.moe_layer(*args, y)
+    torch.cuda.synchronize()
+    assert good.moe_last_status() == (0, 0)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+
+
+def test_overlapped_launch_starts_expert_work_before_the_dispatch_ends():
+    """The timeline of one traced overlapped layer: full tiles appear throughout the dispatch (ascending token
+    order: the first one early), and the first GEMM1 item begins to load before the last row has been stored."""
+    w = inputs.Workload("overlap_trace", T=8192, H=2048, E=8, R=2, K=2, F=512, dtype=BF16)
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, overlap=1)
+    y = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+    plan.moe_layer(*args, y)
+    plan.moe_availability_trace(True)
+    plan.layer_tensor(9).zero_()
+    plan.moe_layer(*args, y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    tr = plan.layer_tensor(8).cpu().numpy()
+    items = plan.layer_tensor(9).cpu().numpy()
+    t0, t_all, ready = tr[0], tr[1], tr[2:]
+    full = ready[ready > 0]
+    assert full.size > 0 and t_all > t0
+    first_tile = (full.min() - t0) / (t_all - t0)
+    started = items[items[:, 0] > 0]
+    gemm1 = started[(started[:, 2] & 1) == 0]
+    assert gemm1[:, 0].min() < t_all, "no expert item began before the dispatch was over"
+    assert first_tile < 0.5, f"first full tile only after {first_tile:.2f} of the dispatch"
+    plan.moe_availability_trace(False)
 
 
 # ------------------------------------------------------------------ random small shapes
