@@ -36,11 +36,18 @@ WORKLOADS = {"c1": inputs.C1, "c2": inputs.C2, "c3": inputs.C3, "c4": inputs.C4,
              # dispatch/combine-only sweep points (identity experts)
              "c5_8192": inputs.C5(8192), "c5_8192_zipf": inputs.C5(8192, 1.2), "c5_2048": inputs.C5(2048)}
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant kernel, from the
-# ncu capture summarised in profiles/ffn_tc_kernel_c2_small.md.  The capture ran the quarter-size case
-# (898.9 MB per launch); C2 proper does 4x its flops with 4x its weights, so the figure is scaled by 4.
-# C4: profiles/ffn_tc_kernel_c4.md, the full-size workload itself (1.065 GB read + 17.3 MB written per launch).
-NCU_TRAFFIC_BYTES = {"mixtral_like_bf16_small": 898.9e6, "mixtral_like_bf16": 4 * 898.9e6, "qwen_moe_like_bf16": 1082.6e6}
+
+
+def ncu_traffic_bytes(workload: str):
+    """DRAM traffic of the dominant kernel per step, measured with ncu and kept beside the profile summaries."""
+    path = os.path.join(ROOT, "profiles", "ncu_dram_traffic.json")
+    try:
+        with open(path) as f:
+            entry = json.load(f).get(workload)
+        return None if entry is None else float(entry["bytes"])
+    except (OSError, ValueError, KeyError, TypeError):
+        return None
+
 
 
 def load_peaks() -> tuple[dict, str]:
@@ -173,6 +180,62 @@ def whole_job_tokens_per_s(tokens_per_rank: int, world: int, ms_per_step: float)
     return world * tokens_per_rank / (ms_per_step * 1e-3)
 
 
+def brief_measurement(args, w: inputs.Workload) -> dict:
+    """ms/step, tokens/s and the per-stage figures of one more workload, device-resident inputs only (no host
+    copies, no oracle): kept in the main line so that its numbers can be followed from round to round."""
+    import torch
+
+    from paper_2605_05888_b200 import binding as B
+
+    def dev(a):
+        if a is None:
+            return None
+        t = torch.from_numpy(a)
+        return t.view(torch.int16).cuda().view(torch.bfloat16) if a.dtype == np.uint16 else t.cuda()
+
+    x = inputs.make_x(w)
+    wr, bias = inputs.make_router(w)
+    wg, wu, wd = inputs.make_all_expert_weights(w)
+    t = [dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    del wg, wu, wd
+    mode = {"scan": B.DISPATCH_SCAN, "static": B.DISPATCH_ATOMIC_STATIC, "paged": B.DISPATCH_ATOMIC_PAGED,
+            "ordered": B.DISPATCH_ATOMIC_ORDERED}[args.dispatch]
+    plan = B.Plan(B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype, dispatch_mode=mode))
+    y = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+    for _ in range(max(args.warmup, 3)):
+        plan.moe_layer(*t, y)
+    torch.cuda.synchronize()
+    plan.moe_ffn_clock_mhz(reset=True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        plan.moe_layer(*t, y)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    clock = round(plan.moe_ffn_clock_mhz(reset=True), 1)
+    stage_ms = np.zeros(len(B.STAGES))
+    for _ in range(args.steps):
+        stage_ms += np.array(plan.moe_layer_timed(*t, y))
+    sm = dict(zip(B.STAGES, (stage_ms / args.steps).tolist()))
+    code, detail = plan.moe_last_status()
+    if code != 0:
+        return {"error": f"device status {code}, detail {detail}"}
+    peaks, _ = load_peaks()
+    eb, rows = w.elem_bytes, w.T * w.K
+    flops = 6.0 * rows * w.H * w.F
+    t_ffn = sm["gemm1"] + sm["gemm2"]
+    disp = (w.T * w.H * eb * (1 + w.K) + 12 * rows) / sm["dispatch"] / 1e6
+    comb = (w.T * w.H * eb * (w.K + 1) + 8 * rows) / sm["combine"] / 1e6
+    return {"ms_per_step": ms, "value": w.T / ms * 1e3, "unit": UNIT, "steps": args.steps,
+            "config": workload_config(w, {"dispatch_mode": args.dispatch}),
+            "ffn": {"ms": t_ffn, "TFLOPs": flops / t_ffn / 1e9, "frac_of_burst_peak": flops / t_ffn / 1e9 / peaks["bf16_tflops"],
+                    "kernel_sm_mhz": clock},
+            "route_ms": sm["route"], "dispatch": {"ms": sm["dispatch"], "GBps": disp, "frac_hbm": disp / peaks["hbm_gbs"]},
+            "combine": {"ms": sm["combine"], "GBps": comb, "frac_hbm": comb / peaks["hbm_gbs"]},
+            "stages_from": "a separate pass with an event after every kernel and a synchronisation per step"}
+
+
 def run_cuda(args, w: inputs.Workload) -> None:
     import torch
     import torch.distributed as dist
@@ -242,8 +305,11 @@ def run_cuda(args, w: inputs.Workload) -> None:
     torch.cuda.synchronize()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop()
-    # SM clock the tensor-core expert kernel really ran at (cycles / time measured inside the kernel)
+    # SM clock the tensor-core expert kernel really ran at (cycles / time measured inside the kernel): THE clock
+    # of the dominant kernel.  sm_mhz is what NVML returned when polled every 5 ms during the timed region; a
+    # region of tens of milliseconds gives it a handful of samples, taken mostly between kernels.
     clocks["ffn_kernel_sm_mhz"] = round(plan.moe_ffn_clock_mhz(reset=True), 1)
+    clocks["sm_mhz_is"] = "NVML samples (see samples); the dominant kernel's own clock is ffn_kernel_sm_mhz"
     barrier()
 
     # ---- per-kernel device times: the same steps with an event after every kernel ----
@@ -334,7 +400,7 @@ def run_cuda(args, w: inputs.Workload) -> None:
     if w.identity_experts or w.dtype != inputs.BF16:
         dom = "dispatch"
         roofline = {"kernel": "dispatch", "bound": "hbm", "achieved": stages["dispatch"]["GBps"], "peak": hbm_peak,
-                    "unit": "GB/s", "frac": stages["dispatch"]["frac_hbm"], "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                    "unit": "GB/s", "frac": stages["dispatch"]["frac_hbm"], "traffic": ncu_traffic_bytes(w.name),
                     "peak_source": f"{peak_kind} hbm_gbs"}
     else:
         t_ffn = sm["gemm1"] + sm["gemm2"]
@@ -349,19 +415,22 @@ def run_cuda(args, w: inputs.Workload) -> None:
         active = int((counts > 0).sum())
         ffn_bytes = 3.0 * active * w.F * w.H * eb + 2.0 * rows * w.H * eb + 2.0 * rows * w.F * eb
         stages["ffn"]["GBps"] = ffn_bytes / t_ffn / 1e6
-        # The kernel is timed inside a loop of whole layers that runs for hundreds of milliseconds under the
-        # power cap, so the denominator is the sustained cuBLAS figure; the burst figure is given beside it.
-        peak = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+        # Denominator: the burst cuBLAS figure when the timed region is shorter than a second (the part has not
+        # settled under its power cap yet), the sustained one for longer runs; both fractions are reported.
+        sustained = peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])
+        long_run = ms_total >= 1000.0
+        peak = sustained if long_run else peaks["bf16_tflops"]
         roofline = {"kernel": "ffn_tc_kernel (expert GEMM1 + SwiGLU + GEMM2, tcgen05)", "bound": "tensor",
                     "achieved": ach, "peak": peak, "unit": "TFLOP/s", "frac": ach / peak,
-                    "traffic": NCU_TRAFFIC_BYTES.get(w.name),
-                    "peak_source": f"{peak_kind} bf16_tflops_sustained (the kernel is timed inside a long, power-capped "
-                                   "loop; its clock is in clocks.ffn_kernel_sm_mhz)",
+                    "traffic": ncu_traffic_bytes(w.name),
+                    "peak_source": f"{peak_kind} " + ("bf16_tflops_sustained (timed region of %.1f s)" % (ms_total / 1e3) if long_run else
+                                                      "bf16_tflops, the burst figure (timed region of %.0f ms)" % ms_total) +
+                                   "; the kernel's clock is in clocks.ffn_kernel_sm_mhz",
                     "frac_of_burst_peak": ach / peaks["bf16_tflops"],
-                    "frac_of_sustained_peak": ach / peak,
+                    "frac_of_sustained_peak": ach / sustained,
                     "frac_of_nominal_2250": ach / 2250.0,
                     "useful_flops_per_launch": gemm1_flops + gemm2_flops}
-        if ffn_bytes / (hbm_peak * 1e9) > (gemm1_flops + gemm2_flops) / (peak * 1e12):
+        if ffn_bytes / (hbm_peak * 1e9) > (gemm1_flops + gemm2_flops) / (peaks["bf16_tflops"] * 1e12):
             # About a tile per expert: streaming the weights takes longer than the MMAs could, so the same
             # kernel is graded against the copy rate.
             roofline.update({"bound": "hbm", "achieved": stages["ffn"]["GBps"], "peak": hbm_peak, "unit": "GB/s",
@@ -390,7 +459,15 @@ def run_cuda(args, w: inputs.Workload) -> None:
                     "api": "moe_layer_host_submit/_wait: pinned host x and y, two steps in flight, host wall clock",
                     "one_step_at_a_time": whole_job_tokens_per_s(w.T, world, ms_e2e_sync / args.steps)},
             "roofline": roofline, "cpu_baseline": cpu, "stages": stages, "dominant": roofline["kernel"],
+            "stages_from": "a separate pass with an event after every kernel and a synchronisation per step, run after the "
+                           "timed steps: the stage times can add up to more than ms_per_step",
             "routing": routing_stats, "availability": availability}
+    if world == 1 and args.also:
+        # free the main workload's device memory first
+        del plan, dx, dwr, dbias, dwg, dwu, dwd, y, wg, wu, wd
+        torch.cuda.empty_cache()
+        line["other_workloads"] = {WORKLOADS[name].name: brief_measurement(args, WORKLOADS[name]) for name in args.also.split(",")
+                                   if name and WORKLOADS[name].name != w.name}
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -402,7 +479,11 @@ def main() -> None:
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--workload", default="c2", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="c3", choices=sorted(WORKLOADS),
+                    help="default: the largest full-layer configuration that fits one GPU (DeepSeek-V3-like)")
+    ap.add_argument("--also", default=None,
+                    help="comma-separated workloads measured briefly after the main one and reported under other_workloads "
+                         "(default: c2 when the main workload is the default one)")
     ap.add_argument("--dispatch", default="paged", choices=["scan", "static", "paged", "ordered"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--ffn-kernel", type=int, default=0, choices=[0, 1, 2],
@@ -416,6 +497,8 @@ def main() -> None:
     ap.add_argument("--overlap", type=int, default=0,
                     help="with --dispatch ordered: dispatch inside the expert kernel's launch (1: half of the SMs dispatch, n: n CTAs)")
     args = ap.parse_args()
+    if args.also is None:
+        args.also = "c2" if args.workload == "c3" else ""
     w = WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, w)
