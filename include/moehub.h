@@ -102,7 +102,13 @@ typedef struct {
                                    its status counter has reached its threshold (Section IV-D);
                                    negative: the same launch, but the consumers wait for the whole
                                    dispatch (for comparison); 0 = stream-ordered launches        */
-  int32_t reserved_[1];         /* must be 0                                                  */
+  int32_t combine_mode;         /* moe_layer: 0 = gather (the combine kernel fetches every token's K
+                                   expert rows from the pool through slot_of); 1 = push (Section
+                                   IV-B, all-to-all combine: the expert kernel's final epilogue
+                                   reads each row's source information and stores the result at
+                                   the token's own position [t*K+k], the combine kernel then reads
+                                   K consecutive rows per token).  Push needs bf16 and the
+                                   one-CTA-per-tile tensor-core kernel (ffn_kernel 0)            */
   int64_t capacity_rows;        /* mode 1: rows per expert region, multiple of 128, 0 = T
                                    rounded up (overflow-free); modes 0/2: ignored            */
   uint64_t spin_limit;          /* bound (iterations) on the dispatch kernels' waits, 0 = 1<<22 */
@@ -201,6 +207,23 @@ int moe_expert_ffn(moe_plan_t* plan, const void* d_recv, const int32_t* d_tile_e
 int moe_dispatch_noalloc(const moe_config_t* cfg, const void* d_x, const int32_t* d_topk_idx,
                          void* d_recv, int32_t* d_expert_count, int32_t* d_tile_expert,
                          int32_t* d_src_info, int32_t* d_slot_of, int32_t* d_status, void* stream);
+
+/* Step 3 with the push-style return of Section IV-B (all-to-all combine: the expert reads the source
+ * information that travelled with each row and stores its output at the row's origin): as
+ * moe_expert_ffn, but the result of the row in pool slot r goes to d_staged[d_src_info[r], :] - the
+ * position t*K+k of its assignment - and slots whose source is -1 produce nothing.
+ * in: as moe_expert_ffn, plus d_src_info [P*128] from moe_dispatch.  out: d_staged [T*K,H] (dtype);
+ * rows of dropped assignments keep their old contents.  bf16 with ffn_kernel 0 only
+ * (MOE_ERR_UNSUPPORTED otherwise). */
+int moe_expert_ffn_push(moe_plan_t* plan, const void* d_recv, const int32_t* d_tile_expert,
+                        const int32_t* d_src_info, const void* d_wg, const void* d_wu, const void* d_wd,
+                        void* d_staged, const int32_t* d_tile_count, const int32_t* d_rows_done, void* stream);
+
+/* Steps 4+5 after moe_expert_ffn_push: y[t,:] = sum_k w[t,k]*staged[t*K+k,:], k ascending, fp32
+ * accumulation, one rounding: the same arithmetic as moe_combine, hence the same bytes in y.
+ * d_slot_of is only looked at to skip dropped assignments (slot -1). */
+int moe_combine_staged(moe_plan_t* plan, const void* d_staged, const int32_t* d_slot_of,
+                       const float* d_topk_w, void* d_y, void* stream);
 
 /* Steps 4+5 (Section II-A, combine and scaling): y[t,:] = sum_k w[t,k]*rows[slot_of[t,k],:],
  * k ascending, fp32 accumulation, rounded once to dtype.  Assignments with slot -1 add 0.

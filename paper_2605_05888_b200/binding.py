@@ -22,7 +22,7 @@ TILE_ROWS = 128
 STAGES = ["route", "dispatch", "worklist", "gemm1", "gemm2", "combine"]
 
 EXPORTS = ["moe_dispatch_noalloc", "moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
-           "moe_dispatch", "moe_expert_ffn", "moe_combine", "moe_layer", "moe_layer_host", "moe_layer_host_submit", "moe_layer_host_wait", "moe_layer_timed",
+           "moe_dispatch", "moe_expert_ffn", "moe_expert_ffn_push", "moe_combine", "moe_combine_staged", "moe_layer", "moe_layer_host", "moe_layer_host_submit", "moe_layer_host_wait", "moe_layer_timed",
            "moe_layer_buffer", "moe_availability_trace",
            "moe_ffn_clock_mhz", "moe_last_launch_count", "moe_last_status", "moe_last_cuda_error", "moe_strerror"]
 
@@ -33,7 +33,7 @@ class MoeConfig(ctypes.Structure):
                 ("renormalize", ctypes.c_int32), ("dispatch_mode", ctypes.c_int32),
                 ("identity_experts", ctypes.c_int32), ("ffn_kernel", ctypes.c_int32), ("ffn_split", ctypes.c_int32),
                 ("ffn_hot_min_tiles", ctypes.c_int32), ("ffn_thin_tiles", ctypes.c_int32),
-                ("overlap", ctypes.c_int32), ("reserved_", ctypes.c_int32 * 1),
+                ("overlap", ctypes.c_int32), ("combine_mode", ctypes.c_int32),
                 ("capacity_rows", ctypes.c_int64), ("spin_limit", ctypes.c_uint64), ("wait_limit_ns", ctypes.c_uint64)]
 
 
@@ -61,6 +61,8 @@ def lib() -> ctypes.CDLL:
         L.moe_dispatch_noalloc.argtypes = [cfgp, vp, i32p, vp, i32p, i32p, i32p, i32p, i32p, vp]
         L.moe_expert_ffn.argtypes = [vp, vp, i32p, vp, vp, vp, vp, i32p, i32p, vp]
         L.moe_combine.argtypes = [vp, vp, i32p, fp, vp, vp]
+        L.moe_expert_ffn_push.argtypes = [vp, vp, i32p, i32p, vp, vp, vp, vp, i32p, i32p, vp]
+        L.moe_combine_staged.argtypes = [vp, vp, i32p, fp, vp, vp]
         L.moe_layer.argtypes = [vp] * 9
         L.moe_layer_host.argtypes = [vp] * 9
         L.moe_layer_host_submit.argtypes = [vp] * 9 + [ctypes.POINTER(ctypes.c_int64)]
@@ -107,9 +109,9 @@ def _stream(stream) -> int:
 
 def make_config(T, H, E, R, K, F, dtype, renormalize=0, dispatch_mode=DISPATCH_ATOMIC_PAGED, identity_experts=0,
                 ffn_kernel=0, capacity_rows=0, spin_limit=0, ffn_split=0, wait_limit_ns=0,
-                ffn_hot_min_tiles=0, ffn_thin_tiles=0, overlap=0) -> MoeConfig:
+                ffn_hot_min_tiles=0, ffn_thin_tiles=0, overlap=0, combine_mode=0) -> MoeConfig:
     return MoeConfig(T, H, E, R, K, F, dtype, int(renormalize), dispatch_mode, int(identity_experts), ffn_kernel, int(ffn_split),
-                     int(ffn_hot_min_tiles), int(ffn_thin_tiles), int(overlap), (ctypes.c_int32 * 1)(0), capacity_rows, spin_limit, wait_limit_ns)
+                     int(ffn_hot_min_tiles), int(ffn_thin_tiles), int(overlap), int(combine_mode), capacity_rows, spin_limit, wait_limit_ns)
 
 
 def moe_pool_tiles(cfg: MoeConfig) -> int:
@@ -173,6 +175,16 @@ class Plan:
         _check(lib().moe_expert_ffn(self.handle, _ptr(recv), _ptr(tile_expert), _ptr(wg), _ptr(wu), _ptr(wd),
                                     _ptr(out_rows), _ptr(tile_count), _ptr(rows_done), _stream(stream)),
                "moe_expert_ffn")
+
+    def moe_expert_ffn_push(self, recv, tile_expert, src_info, wg, wu, wd, staged, tile_count=None, rows_done=None,
+                            stream=None):
+        _check(lib().moe_expert_ffn_push(self.handle, _ptr(recv), _ptr(tile_expert), _ptr(src_info), _ptr(wg), _ptr(wu),
+                                         _ptr(wd), _ptr(staged), _ptr(tile_count), _ptr(rows_done), _stream(stream)),
+               "moe_expert_ffn_push")
+
+    def moe_combine_staged(self, staged, slot_of, topk_w, y, stream=None):
+        _check(lib().moe_combine_staged(self.handle, _ptr(staged), _ptr(slot_of), _ptr(topk_w), _ptr(y), _stream(stream)),
+               "moe_combine_staged")
 
     def moe_combine(self, rows, slot_of, topk_w, y, stream=None):
         _check(lib().moe_combine(self.handle, _ptr(rows), _ptr(slot_of), _ptr(topk_w), _ptr(y), _stream(stream)),

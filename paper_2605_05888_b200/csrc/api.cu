@@ -26,7 +26,9 @@ int check_config(const moe_config_t* c, Geometry* g) {
   if (c->dispatch_mode < 0 || c->dispatch_mode > 3) return MOE_ERR_ARG;
   if (!c->identity_experts && c->F <= 0) return MOE_ERR_ARG;
   if (c->E > 256 || c->K > 32) return MOE_ERR_UNSUPPORTED;
-  if (c->reserved_[0] != 0) return MOE_ERR_ARG;
+  if (c->combine_mode < 0 || c->combine_mode > 1) return MOE_ERR_ARG;
+  if (c->combine_mode == 1 && (c->dtype != MOE_DTYPE_BF16 || c->ffn_kernel != 0 || c->identity_experts))
+    return MOE_ERR_UNSUPPORTED;
   const int eb = c->dtype == MOE_DTYPE_BF16 ? 2 : 4;
   if (((int64_t)c->H * eb) % 16 != 0) return MOE_ERR_ALIGN;
   if (!c->identity_experts && ((int64_t)c->F * eb) % 16 != 0) return MOE_ERR_ALIGN;
@@ -241,6 +243,30 @@ int moe_expert_ffn(moe_plan_t* p, const void* d_recv, const int32_t* d_tile_expe
   return rc == 0 ? MOE_OK : (rc < 0 ? rc : MOE_ERR_CUDA);
 }
 
+int moe_expert_ffn_push(moe_plan_t* p, const void* d_recv, const int32_t* d_tile_expert, const int32_t* d_src_info,
+                        const void* d_wg, const void* d_wu, const void* d_wd, void* d_staged,
+                        const int32_t* d_tile_count, const int32_t* d_rows_done, void* stream) {
+  if (!p || !d_recv || !d_tile_expert || !d_src_info || !d_wg || !d_wu || !d_wd || !d_staged) return MOE_ERR_ARG;
+  if (p->cfg.identity_experts) return MOE_ERR_ARG;
+  if (p->cfg.dtype != MOE_DTYPE_BF16 || p->cfg.ffn_kernel != 0) return MOE_ERR_UNSUPPORTED;
+  if (misaligned(d_recv) || misaligned(d_wg) || misaligned(d_wu) || misaligned(d_wd) || misaligned(d_staged))
+    return MOE_ERR_ALIGN;
+  if ((d_tile_count == nullptr) != (d_rows_done == nullptr)) return MOE_ERR_ARG;
+  p->launches = 0;
+  int rc = launch_ffn_tc(p, d_recv, d_tile_expert, d_wg, d_wu, d_wd, d_staged, d_tile_count, d_rows_done,
+                         (cudaStream_t)stream, nullptr, nullptr, d_src_info);
+  return rc == 0 ? MOE_OK : (rc < 0 ? rc : MOE_ERR_CUDA);
+}
+
+int moe_combine_staged(moe_plan_t* p, const void* d_staged, const int32_t* d_slot_of, const float* d_topk_w, void* d_y,
+                       void* stream) {
+  if (!p) return MOE_ERR_ARG;
+  if (p->cfg.T > 0 && (!d_staged || !d_slot_of || !d_topk_w || !d_y)) return MOE_ERR_ARG;
+  if (misaligned(d_staged) || misaligned(d_y)) return MOE_ERR_ALIGN;
+  p->launches = 0;
+  return launch_combine(p, d_staged, d_slot_of, d_topk_w, d_y, (cudaStream_t)stream, true) ? MOE_ERR_CUDA : MOE_OK;
+}
+
 int moe_combine(moe_plan_t* p, const void* d_rows, const int32_t* d_slot_of, const float* d_topk_w, void* d_y,
                 void* stream) {
   if (!p) return MOE_ERR_ARG;
@@ -281,9 +307,10 @@ int moe_layer(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_b
                                   s.tile_count, s.rows_done, prepared, st))
     return cuda_failed(2);
   mark(p, 2, st);
-  if (overlap) {
-    int rc = launch_ffn_tc(p, s.recv, s.tile_expert, d_wg, d_wu, d_wd, s.out_rows, s.tile_count, s.rows_done, st, d_x,
-                           s.topk_idx);
+  const bool push = c.combine_mode == 1;  // the expert kernel returns every row to its token's position itself
+  if (overlap || push) {
+    int rc = launch_ffn_tc(p, s.recv, s.tile_expert, d_wg, d_wu, d_wd, s.out_rows, s.tile_count, s.rows_done, st,
+                           overlap ? d_x : nullptr, overlap ? s.topk_idx : nullptr, push ? s.src_info : nullptr);
     if (rc != 0) return rc < 0 && rc != MOE_ERR_CUDA ? rc : cuda_failed(3);
   } else if (!p->cfg.identity_experts) {
     int rc = ffn_dispatch(p, s.recv, s.tile_expert, d_wg, d_wu, d_wd, s.out_rows, s.tile_count, s.rows_done, st);
@@ -293,7 +320,7 @@ int moe_layer(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_b
     mark(p, 4, st);
   }
   mark(p, 5, st);
-  if (launch_combine(p, s.out_rows, s.slot_of, s.topk_w, d_y, st)) return cuda_failed(4);
+  if (launch_combine(p, s.out_rows, s.slot_of, s.topk_w, d_y, st, push)) return cuda_failed(4);
   mark(p, 6, st);
   return MOE_OK;
 }

@@ -18,7 +18,7 @@ template <typename XT, int KT>  // KT > 0: K known at compile time; KT == 0: run
 __global__ void __launch_bounds__(kCombThreads)
 combine_kernel(const uint4* __restrict__ rows, const int* __restrict__ slot_of,
                const float* __restrict__ topk_w, int T, int K_rt, int vec_per_row, int runs_per_row,
-               uint4* __restrict__ y) {
+               uint4* __restrict__ y, int staged) {
   constexpr int N = Vec16<XT>::N;
   constexpr int KMAX = KT > 0 ? KT : 1;
   const int K = KT > 0 ? KT : K_rt;
@@ -34,6 +34,8 @@ combine_kernel(const uint4* __restrict__ rows, const int* __restrict__ slot_of,
   if (lane < K) {
     my_slot = slot_of[(size_t)t * K + lane];
     my_w = topk_w[(size_t)t * K + lane];
+    // push-style combine: the experts stored assignment (t, k) at row t*K+k themselves; slot_of only says whether it exists
+    if (staged && my_slot >= 0) my_slot = t * K + lane;
   }
   uint4* dst = y + (size_t)t * vec_per_row;
   const int v0 = v_begin + lane, v1 = v_begin + 32 + lane;
@@ -92,7 +94,7 @@ combine_kernel(const uint4* __restrict__ rows, const int* __restrict__ slot_of,
 
 template <typename XT>
 static int launch_typed(moe_plan* p, const void* rows, const int* slot_of, const float* topk_w, void* y,
-                        cudaStream_t st) {
+                        cudaStream_t st, bool staged) {
   const moe_config_t& c = p->cfg;
   const int vec_per_row = c.H * (int)sizeof(XT) / 16;
   const int runs_per_row = (vec_per_row + kCombRun - 1) / kCombRun;
@@ -100,7 +102,7 @@ static int launch_typed(moe_plan* p, const void* rows, const int* slot_of, const
   const int grid = (int)((warps + kCombThreads / 32 - 1) / (kCombThreads / 32));
 #define MOEHUB_COMBINE(KT)                                                                          \
   launch_pdl(combine_kernel<XT, KT>, dim3(grid), dim3(kCombThreads), 0, st, (const uint4*)rows, slot_of, topk_w, \
-             c.T, c.K, vec_per_row, runs_per_row, (uint4*)y)
+             c.T, c.K, vec_per_row, runs_per_row, (uint4*)y, staged ? 1 : 0)
   switch (c.K) {
     case 1: MOEHUB_COMBINE(1); break;
     case 2: MOEHUB_COMBINE(2); break;
@@ -114,10 +116,10 @@ static int launch_typed(moe_plan* p, const void* rows, const int* slot_of, const
 }
 
 int launch_combine(moe_plan* p, const void* rows, const int* slot_of, const float* topk_w, void* y,
-                   cudaStream_t st) {
+                   cudaStream_t st, bool staged) {
   if (p->cfg.T == 0) return 0;
-  if (p->cfg.dtype == MOE_DTYPE_BF16) return launch_typed<__nv_bfloat16>(p, rows, slot_of, topk_w, y, st);
-  return launch_typed<float>(p, rows, slot_of, topk_w, y, st);
+  if (p->cfg.dtype == MOE_DTYPE_BF16) return launch_typed<__nv_bfloat16>(p, rows, slot_of, topk_w, y, st, staged);
+  return launch_typed<float>(p, rows, slot_of, topk_w, y, st, staged);
 }
 
 }  // namespace moehub

@@ -152,8 +152,9 @@ int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv,
                     int* tile_expert, int* src_info, int* slot_of, int* tile_count, int* rows_done,
                     bool prepared, cudaStream_t st);
 PrepArgs make_prep(moe_plan* p, int* expert_count, int* tile_expert, int* src_info, int* tile_count, int* rows_done);
+// staged: rows holds assignment (t, k) at row t*K+k (push-style combine); slot_of then only tells dropped assignments.
 int launch_combine(moe_plan* p, const void* rows, const int* slot_of, const float* topk_w, void* y,
-                   cudaStream_t st);
+                   cudaStream_t st, bool staged = false);
 int launch_ffn_simt(moe_plan* p, const void* recv, const int* tile_expert, const void* wg,
                     const void* wu, const void* wd, void* out_rows, cudaStream_t st);
 // tile_count / rows_done: availability counters the GEMM1 producer waits on before it reads a tile
@@ -161,7 +162,7 @@ int launch_ffn_simt(moe_plan* p, const void* recv, const int* tile_expert, const
 int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const void* wg,
                   const void* wu, const void* wd, void* out_rows, const int* tile_count,
                   const int* rows_done, cudaStream_t st, const void* overlap_x = nullptr,
-                  const int* overlap_idx = nullptr);
+                  const int* overlap_idx = nullptr, const int* push_src = nullptr);
 
 // ---- element helpers ---------------------------------------------------------------------------
 __device__ __forceinline__ float to_float(float v) { return v; }

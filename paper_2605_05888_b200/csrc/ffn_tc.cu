@@ -432,7 +432,11 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
               tc_wait_ld();
               if (h < H) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) out[(row0 + c + i) * H + h] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                for (int i = 0; i < 16; ++i) {
+                  long long orow = (long long)(row0 + c + i);
+                  if (prm.push_src != nullptr) orow = __ldcg(prm.push_src + row0 + c + i);  // the row's own token position
+                  if (orow >= 0) out[(size_t)orow * H + h] = __float2bfloat16_rn(__uint_as_float(v[i]));
+                }
               }
             }
           }
@@ -461,6 +465,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
           }
         }
       } else {
+        // Push-style combine (paper Section IV-B, all-to-all combine): the expert reads the row's source
+        // information after its final GEMM and stores the result straight to the token's position.
+        if (prm.push_src != nullptr) {
+          const int src = __ldcg(prm.push_src + row);
+          if (src < 0) row_live = false;  // an empty slot: nothing to return
+          else row = (size_t)src;
+        }
         __nv_bfloat16* dst = out + row * H + (size_t)it.nb * 256;
         const int ncols = min(256, H - it.nb * 256);
 #pragma unroll 1
@@ -581,7 +592,7 @@ OrderedParams make_ordered_params(moe_plan* p, const void* x, const int* topk_id
 // dispatches x (ordered scheme, into recv and the plan's own dispatch outputs) on its first CTAs.
 int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const void* wg, const void* wu,
                   const void* wd, void* out_rows, const int* tile_count, const int* rows_done, cudaStream_t st,
-                  const void* overlap_x, const int* overlap_idx) {
+                  const void* overlap_x, const int* overlap_idx, const int* push_src) {
   const moe_config_t& c = p->cfg;
   if (p->P == 0 || c.T == 0) return 0;
   EncodeTiledFn enc;
@@ -607,6 +618,7 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   // default splits there.
   const int fused = c.ffn_split == 2 ? 1 : (c.ffn_split == 1 ? 0 : (c.E <= 64 ? 1 : 0));
   const bool pairs = c.ffn_kernel == 2;  // opt-in: the CTA-pair kernel
+  if (pairs && push_src != nullptr) return MOE_ERR_UNSUPPORTED;
   const int workers = pairs ? grid / 2 : grid;
   if (p->P > kMaxListTiles) return MOE_ERR_UNSUPPORTED;  // the work list lives in the kernel's shared memory
   if ((long long)p->P * (NB1 + NB2) >= (1ll << kThinShift)) return MOE_ERR_UNSUPPORTED;  // item index field of the ring
@@ -644,6 +656,7 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   prm.item_ns = (p->trace && !pairs) ? p->s.item_ns : nullptr;
   prm.hist = nullptr;
   prm.hot_first = 0;
+  prm.push_src = push_src;
   OverlapParams ov = {};
   const bool overlap = overlap_x != nullptr && !pairs;
   if (overlap) {

@@ -315,6 +315,9 @@ struct FfnParams {
   const int* tile_expert;  // [P]
   int P, lag, fused;
   int hot_min;  // > 0: interleave tensor-bound and weight-streaming-bound items (see WorkList)
+  const int* push_src;  // push-style combine: the source info t*K+k of every pool row - the GEMM2 epilogue stores row r
+                        // of the pool at row push_src[r] of `out` (the token's own position) and skips rows whose
+                        // source is negative (empty slots); nullptr: rows stay where they are
   const int* hist;  // rows per expert (the ordered dispatch's counts): the work list is built from them, or nullptr
   int hot_first;    // with hist: experts are walked by descending row count
   int thin;         // the narrow (transposed) form for single tiles of at most 64 rows is in use

@@ -77,6 +77,26 @@ def test_c3_deepseek_like_full_size_skewed(mode):
 
 
 @pytest.mark.parametrize("w", [inputs.C2, inputs.C3, inputs.C4], ids=lambda w: w.name)
+def test_push_combine_full_size(w):
+    """Push-style combine at the benchmark's sizes (every form of the expert kernel's final epilogue: full tiles,
+    short last tiles, narrow single tiles): the same bytes in y as the gather path, and the oracle's output on a
+    row of every used tile."""
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED, combine_mode=1)
+    y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
+    plan.moe_layer(*args, y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    check_sampled_output(w, plan, y, x, wr, bias, wg, wu, wd, 16)
+    gather = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED)
+    y2 = torch.empty_like(y)
+    gather.moe_layer(*args, y2)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y2)
+
+
+@pytest.mark.parametrize("w", [inputs.C2, inputs.C3, inputs.C4], ids=lambda w: w.name)
 def test_overlapped_launch_full_size(w):
     """Dispatch inside the expert kernel's launch (producer CTAs emit the tokens in ascending order, consumer
     CTAs start on a tile when its status counter reaches the rows it will hold) at the benchmark's sizes:

@@ -507,6 +507,62 @@ def test_overlapped_launch_starts_expert_work_before_the_dispatch_ends():
     plan.moe_availability_trace(False)
 
 
+# ------------------------------------------------------------------ push-style combine
+PUSH_CASES = [SMALL[3], SMALL[4], SMALL[5], SMALL[7], SMALL[8],
+              inputs.Workload("three_tiles", T=700, H=320, E=4, R=2, K=2, F=392, dtype=BF16),
+              inputs.Workload("half_tiles", T=900, H=264, E=6, R=3, K=2, F=136, dtype=BF16, zipf_s=1.0, seed=2)]
+
+
+@pytest.mark.parametrize("w", PUSH_CASES, ids=lambda w: w.name)
+def test_push_combine_stages_match_oracle_and_the_gather_path(w):
+    """Section IV-B, all-to-all combine: the expert kernel reads the source information of every row after its
+    final GEMM and stores the result at the token's position t*K+k; the reduction then reads K consecutive rows.
+    Through the C ABI (moe_expert_ffn_push, moe_combine_staged): every staged row is the expert output of its
+    assignment, y matches the oracle, and y is the same bytes as the gather path's."""
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    g = run_stages(w, B.DISPATCH_ATOMIC_PAGED, x, wr, bias, wg, wu, wd)          # the gather path, for comparison
+    plan = g["plan"]
+    staged = torch.full((w.T * w.K, w.H), 7.0, dtype=torch.bfloat16, device="cuda")
+    plan.moe_expert_ffn_push(g["recv"], g["te"], g["src"], Hh.to_dev(wg), Hh.to_dev(wu), Hh.to_dev(wd), staged)
+    y = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+    plan.moe_combine_staged(staged, g["slot"], g["tw"], y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    slot = g["slot"].flatten().long()
+    assert torch.equal(staged, g["out_rows"][slot]), "a staged row is not the expert output of its assignment"
+    assert torch.equal(y, g["y"])
+    Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+
+
+@pytest.mark.parametrize("overlap", [0, 1])
+@pytest.mark.parametrize("mode", [B.DISPATCH_SCAN, B.DISPATCH_ATOMIC_PAGED, B.DISPATCH_ATOMIC_ORDERED])
+@pytest.mark.parametrize("w", [SMALL[3], SMALL[4], SMALL[5]], ids=lambda w: w.name)
+def test_layer_with_push_combine(w, mode, overlap):
+    if overlap and mode != B.DISPATCH_ATOMIC_ORDERED:
+        pytest.skip("the overlapped launch belongs to the ordered dispatch")
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    plan = Hh.make_plan(w, mode, combine_mode=1, overlap=overlap)
+    y = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+    plan.moe_layer(*args, y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+    gather = Hh.make_plan(w, mode)
+    y2 = torch.empty_like(y)
+    gather.moe_layer(*args, y2)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y2)
+
+
+def test_push_combine_is_refused_where_it_is_not_built():
+    with pytest.raises(B.MoeError) as ei:
+        B.moe_workspace_bytes(B.make_config(64, 128, 8, 2, 2, 64, FP32, combine_mode=1))
+    assert ei.value.code == -3
+
+
 # ------------------------------------------------------------------ random small shapes
 def _random_workloads(n, seed):
     rng = np.random.default_rng(seed)
