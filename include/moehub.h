@@ -109,6 +109,18 @@ typedef struct {
                                    the token's own position [t*K+k], the combine kernel then reads
                                    K consecutive rows per token).  Push needs bf16 and the
                                    one-CTA-per-tile tensor-core kernel (ffn_kernel 0)            */
+  int32_t tp_shards;            /* expert + tensor parallelism (Section VII): S > 1 cuts every expert's
+                                   FFN into S slices of its width F (gate/up rows [s*F/S, (s+1)*F/S),
+                                   the matching columns of the down matrix), gives every slice a
+                                   receive region of its own (one registration per TP shard) and
+                                   stores every row to all S of them.  Every stage then sees E*S
+                                   experts and K*S assignments per token: topk_idx / topk_w /
+                                   slot_of are [T, K*S] with entry k*S+s = (expert*S + s, the
+                                   pick's weight), expert_count is [E*S], the pool has
+                                   floor(T*K*S/128) + E*S tiles, and the combine step adds the
+                                   K*S partial rows.  Needs F % S == 0, E*S <= 256, K*S <= 32;
+                                   0 or 1 = none                                               */
+  int32_t reserved_;            /* must be 0                                                  */
   int64_t capacity_rows;        /* mode 1: rows per expert region, multiple of 128, 0 = T
                                    rounded up (overflow-free); modes 0/2: ignored            */
   uint64_t spin_limit;          /* bound (iterations) on the dispatch kernels' waits, 0 = 1<<22 */

@@ -169,10 +169,39 @@ def combine(rows, slot_of, topk_w, bf16_storage=False):
     return y
 
 
-def layer(x, wr, bias, wg, wu, wd, E, R, K, dtype, renormalize=0, identity_experts=False, bf16_storage=False):
+def tp_expand(idx, w, wg, wu, wd, S):
+    """Expert + tensor parallelism as Section VII of the paper puts it: every TP shard of an expert has a receive
+    region of its own and every row is stored to all of them.  Shard s of expert e holds rows [s*F/S, (s+1)*F/S)
+    of the gate and up matrices and the matching columns of the down matrix; it is listed as expert e*S + s.
+    Returns the routing result with every pick listed once per shard (same weight) and the sliced weights."""
+    T, K = idx.shape
+    idx_e = (idx[:, :, None].astype(np.int64) * S + np.arange(S)[None, None, :]).reshape(T, K * S).astype(np.int32)
+    w_e = np.repeat(w, S, axis=1)
+    if wg is None:
+        return idx_e, w_e, None, None, None
+    wg_e, wu_e, wd_e = [], [], []
+    for e in range(len(wg)):
+        for s in range(S):
+            if wg[e] is None:
+                wg_e.append(None), wu_e.append(None), wd_e.append(None)
+                continue
+            Fs = wg[e].shape[0] // S
+            wg_e.append(np.ascontiguousarray(wg[e][s * Fs:(s + 1) * Fs, :]))
+            wu_e.append(np.ascontiguousarray(wu[e][s * Fs:(s + 1) * Fs, :]))
+            wd_e.append(np.ascontiguousarray(wd[e][:, s * Fs:(s + 1) * Fs]))
+    return idx_e, w_e, wg_e, wu_e, wd_e
+
+
+def layer(x, wr, bias, wg, wu, wd, E, R, K, dtype, renormalize=0, identity_experts=False, bf16_storage=False,
+          tp_shards=1):
     """The whole layer: route -> dispatch -> experts -> combine. Returns dict with every stage's output.
-    bf16_storage: the diagnostic restatement (intermediate, expert rows and y rounded to bf16)."""
+    bf16_storage: the diagnostic restatement (intermediate, expert rows and y rounded to bf16).
+    tp_shards = S > 1: every expert is cut into S TP shards (see tp_expand); topk_idx, topk_w, slot_of and the
+    dispatch outputs are then those of the E*S shards, and y adds the shards' partial rows."""
     idx, w, lg = route(x, wr, bias, K, dtype, renormalize)
+    if tp_shards > 1:
+        idx, w, wg, wu, wd = tp_expand(idx, w, wg, wu, wd, tp_shards)
+        E = E * tp_shards
     d = dispatch(x, idx, E, R, dtype)
     if identity_experts:
         rows = identity_ffn(d["recv"], dtype)

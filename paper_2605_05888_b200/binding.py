@@ -34,6 +34,7 @@ class MoeConfig(ctypes.Structure):
                 ("identity_experts", ctypes.c_int32), ("ffn_kernel", ctypes.c_int32), ("ffn_split", ctypes.c_int32),
                 ("ffn_hot_min_tiles", ctypes.c_int32), ("ffn_thin_tiles", ctypes.c_int32),
                 ("overlap", ctypes.c_int32), ("combine_mode", ctypes.c_int32),
+                ("tp_shards", ctypes.c_int32), ("reserved_", ctypes.c_int32),
                 ("capacity_rows", ctypes.c_int64), ("spin_limit", ctypes.c_uint64), ("wait_limit_ns", ctypes.c_uint64)]
 
 
@@ -109,9 +110,9 @@ def _stream(stream) -> int:
 
 def make_config(T, H, E, R, K, F, dtype, renormalize=0, dispatch_mode=DISPATCH_ATOMIC_PAGED, identity_experts=0,
                 ffn_kernel=0, capacity_rows=0, spin_limit=0, ffn_split=0, wait_limit_ns=0,
-                ffn_hot_min_tiles=0, ffn_thin_tiles=0, overlap=0, combine_mode=0) -> MoeConfig:
+                ffn_hot_min_tiles=0, ffn_thin_tiles=0, overlap=0, combine_mode=0, tp_shards=0) -> MoeConfig:
     return MoeConfig(T, H, E, R, K, F, dtype, int(renormalize), dispatch_mode, int(identity_experts), ffn_kernel, int(ffn_split),
-                     int(ffn_hot_min_tiles), int(ffn_thin_tiles), int(overlap), int(combine_mode), capacity_rows, spin_limit, wait_limit_ns)
+                     int(ffn_hot_min_tiles), int(ffn_thin_tiles), int(overlap), int(combine_mode), int(tp_shards), 0, capacity_rows, spin_limit, wait_limit_ns)
 
 
 def moe_pool_tiles(cfg: MoeConfig) -> int:
@@ -254,10 +255,12 @@ class Plan:
         c = self.cfg
         rows = self.P * TILE_ROWS
         el = torch.bfloat16 if c.dtype == DTYPE_BF16 else torch.float32
-        shapes = {0: ((c.T, c.K), torch.int32), 1: ((c.T, c.K), torch.float32), 2: ((rows, c.H), el),
-                  3: ((c.E,), torch.int32), 4: ((self.P,), torch.int32), 5: ((rows,), torch.int32),
-                  6: ((c.T, c.K), torch.int32), 7: ((rows, c.H), el), 8: ((self.P + 2,), torch.int64),
-                  9: ((self.P * ((c.F + 127) // 128 + (c.H + 255) // 256), 4), torch.int64)}
+        tp = max(1, c.tp_shards)                     # with TP shards the stages see E*tp experts, K*tp picks, width F/tp
+        K, E, F = c.K * tp, c.E * tp, c.F // tp
+        shapes = {0: ((c.T, K), torch.int32), 1: ((c.T, K), torch.float32), 2: ((rows, c.H), el),
+                  3: ((E,), torch.int32), 4: ((self.P,), torch.int32), 5: ((rows,), torch.int32),
+                  6: ((c.T, K), torch.int32), 7: ((rows, c.H), el), 8: ((self.P + 2,), torch.int64),
+                  9: ((self.P * ((F + 127) // 128 + (c.H + 255) // 256), 4), torch.int64)}
         shape, dt = shapes[which]
         ptr = self.moe_layer_buffer(which)
         off = ptr - self.workspace.data_ptr()

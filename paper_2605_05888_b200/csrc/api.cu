@@ -13,15 +13,33 @@ constexpr size_t kAlign = 256;
 inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 
 struct Geometry {
+  moe_config_t eff;  // the effective configuration (TP shards folded into E, K and F: see moe_plan)
+  int tp;
   int64_t P, cap_rows;
   int tiles_per_expert, dispatch_tokens, nblk, eb;
   int ord_tokens, ord_nblk;
 };
 
-int check_config(const moe_config_t* c, Geometry* g) {
-  if (!c) return MOE_ERR_ARG;
-  if (c->T < 0 || c->H <= 0 || c->E <= 0 || c->R <= 0 || c->K <= 0) return MOE_ERR_ARG;
-  if (c->K > c->E || c->E % c->R != 0) return MOE_ERR_ARG;
+int check_config(const moe_config_t* user, Geometry* g) {
+  if (!user) return MOE_ERR_ARG;
+  if (user->T < 0 || user->H <= 0 || user->E <= 0 || user->R <= 0 || user->K <= 0) return MOE_ERR_ARG;
+  if (user->K > user->E || user->E % user->R != 0) return MOE_ERR_ARG;
+  // Expert + tensor parallelism (paper Section VII): an expert's FFN is cut into tp_shards slices of its
+  // width F, every slice has a receive region of its own and every row is stored to all of them.  From
+  // here on shard s of expert e is the virtual expert e*S + s of a layer with E*S experts, K*S picks per
+  // token and FFN width F/S (SwiGLU and the down projection are sums over F, so the S partial results of a
+  // pick add up to the expert's output; the combine step adds them with the pick's weight).
+  const int tp = user->tp_shards > 1 ? user->tp_shards : 1;
+  if (user->tp_shards < 0) return MOE_ERR_ARG;
+  if (tp > 1 && (user->identity_experts || user->F % tp != 0)) return MOE_ERR_ARG;
+  if (tp > 1 && user->ffn_kernel == 2) return MOE_ERR_UNSUPPORTED;
+  g->eff = *user;
+  g->eff.E = user->E * tp;
+  g->eff.K = user->K * tp;
+  if (!user->identity_experts) g->eff.F = user->F / tp;
+  g->eff.R = user->R;  // a rank keeps its experts' shards: E*S % R == 0 follows
+  g->tp = tp;
+  const moe_config_t* c = &g->eff;
   if (c->dtype != MOE_DTYPE_FP32 && c->dtype != MOE_DTYPE_BF16) return MOE_ERR_ARG;
   if (c->dispatch_mode < 0 || c->dispatch_mode > 3) return MOE_ERR_ARG;
   if (!c->identity_experts && c->F <= 0) return MOE_ERR_ARG;
@@ -133,7 +151,7 @@ int moe_workspace_bytes(const moe_config_t* cfg, size_t* out_bytes) {
   if (!out_bytes) return MOE_ERR_ARG;
   int rc = check_config(cfg, &g);
   if (rc != MOE_OK) return rc;
-  *out_bytes = carve(*cfg, g, nullptr, nullptr, nullptr);
+  *out_bytes = carve(g.eff, g, nullptr, nullptr, nullptr);
   return MOE_OK;
 }
 
@@ -145,10 +163,13 @@ int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, mo
   if (rc != MOE_OK) return rc;
   if (!d_workspace) return MOE_ERR_ARG;
   if (reinterpret_cast<uintptr_t>(d_workspace) % kAlign != 0) return MOE_ERR_WORKSPACE;
-  if (bytes < carve(*cfg, g, nullptr, nullptr, nullptr)) return MOE_ERR_WORKSPACE;
+  if (bytes < carve(g.eff, g, nullptr, nullptr, nullptr)) return MOE_ERR_WORKSPACE;
   moe_plan* p = new (std::nothrow) moe_plan();
   if (!p) return MOE_ERR_ARG;
-  p->cfg = *cfg;
+  p->cfg = g.eff;
+  p->tp = g.tp;
+  p->route_E = cfg->E;
+  p->route_K = cfg->K;
   p->P = g.P;
   p->cap_rows = g.cap_rows;
   p->tiles_per_expert = g.tiles_per_expert;
@@ -165,7 +186,7 @@ int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, mo
   p->copy_in = p->copy_out = nullptr;
   p->submitted = 0;
   for (int b = 0; b < 2; ++b) p->ev_in[b] = p->ev_done[b] = p->ev_out[b] = nullptr;
-  carve(*cfg, g, (char*)d_workspace, &p->s, &p->counters_bytes);
+  carve(g.eff, g, (char*)d_workspace, &p->s, &p->counters_bytes);
   if (cudaGetDevice(&p->device) != cudaSuccess ||
       cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device) != cudaSuccess) {
     delete p;
@@ -173,7 +194,7 @@ int moe_plan_create(const moe_config_t* cfg, void* d_workspace, size_t bytes, mo
   }
   // The status word must start clean even if a stage other than dispatch is called first.
   if (cudaMemset(p->s.status, 0, p->counters_bytes) != cudaSuccess ||
-      cudaMemset(p->s.hist, 0, sizeof(int) * (size_t)cfg->E) != cudaSuccess ||
+      cudaMemset(p->s.hist, 0, sizeof(int) * (size_t)g.eff.E) != cudaSuccess ||
       cudaMemset(p->s.ord_exit, 0, sizeof(int) * 2) != cudaSuccess ||
       cudaMemset(p->s.gemm1_done, 0, sizeof(int) * (size_t)(g.P + 4)) != cudaSuccess ||
       cudaMemset(p->s.clock_probe, 0, 2 * sizeof(unsigned long long)) != cudaSuccess) {

@@ -76,7 +76,10 @@ __device__ __forceinline__ void prep_reset(const PrepArgs& a, int gtid, int gthr
 }  // namespace moehub
 
 struct moe_plan {
-  moe_config_t cfg;
+  moe_config_t cfg;          // the EFFECTIVE configuration: with tp_shards = S, E, K and F here are E*S, K*S and F/S
+                             // (every expert's S shards are S virtual experts, every pick S assignments)
+  int tp;                    // TP shards per expert (1: none)
+  int route_E, route_K;      // what the router works with: the experts it scores and the picks per token
   int64_t P;                 // pool tiles
   int64_t cap_rows;          // mode 1: rows per expert
   int tiles_per_expert;      // paged tile-table width

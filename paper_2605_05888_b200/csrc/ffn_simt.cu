@@ -16,8 +16,8 @@ constexpr int kSimtBK = 16;
 template <typename XT, bool SWIGLU>
 __global__ void __launch_bounds__(kSimtThreads)
 ffn_simt_kernel(const XT* __restrict__ A, int lda, const int* __restrict__ tile_expert,
-                const XT* __restrict__ B1, const XT* __restrict__ B2, size_t expert_stride, int N, int Kd,
-                XT* __restrict__ C, int ldc) {
+                const XT* __restrict__ B1, const XT* __restrict__ B2, size_t expert_stride, int tp,
+                size_t shard_offset, int ldb, int N, int Kd, XT* __restrict__ C, int ldc) {
   const int p = blockIdx.y;
   pdl_wait();
   pdl_trigger();
@@ -25,8 +25,10 @@ ffn_simt_kernel(const XT* __restrict__ A, int lda, const int* __restrict__ tile_
   if (e < 0) return;
   const int n0 = blockIdx.x * kSimtBN;
   const size_t row0 = (size_t)p * kTileRows;
-  const XT* b1 = B1 + (size_t)e * expert_stride;
-  const XT* b2 = SWIGLU ? B2 + (size_t)e * expert_stride : nullptr;
+  // e is a virtual expert: shard e % tp of expert e / tp (tp = 1: the expert itself)
+  const size_t base = (size_t)(e / tp) * expert_stride + (size_t)(e % tp) * shard_offset;
+  const XT* b1 = B1 + base;
+  const XT* b2 = SWIGLU ? B2 + base : nullptr;
   __shared__ float As[kSimtBK][kTileRows + 1];
   __shared__ float Bs[kSimtBK][kSimtBN + 1];
   __shared__ float Bs2[SWIGLU ? kSimtBK : 1][kSimtBN + 1];
@@ -51,8 +53,8 @@ ffn_simt_kernel(const XT* __restrict__ A, int lda, const int* __restrict__ tile_
       const int idx = threadIdx.x + i * kSimtThreads;
       const int r = idx / kSimtBK, kk = idx % kSimtBK;
       const bool ok = (n0 + r < N) && (k0 + kk < Kd);
-      Bs[kk][r] = ok ? to_float(b1[(size_t)(n0 + r) * Kd + k0 + kk]) : 0.0f;
-      if (SWIGLU) Bs2[kk][r] = ok ? to_float(b2[(size_t)(n0 + r) * Kd + k0 + kk]) : 0.0f;
+      Bs[kk][r] = ok ? to_float(b1[(size_t)(n0 + r) * ldb + k0 + kk]) : 0.0f;
+      if (SWIGLU) Bs2[kk][r] = ok ? to_float(b2[(size_t)(n0 + r) * ldb + k0 + kk]) : 0.0f;
     }
     __syncthreads();
 #pragma unroll
@@ -91,15 +93,18 @@ template <typename XT>
 static int launch_typed(moe_plan* p, const void* recv, const int* tile_expert, const void* wg,
                         const void* wu, const void* wd, void* out_rows, cudaStream_t st) {
   const moe_config_t& c = p->cfg;
-  const size_t stride = (size_t)c.F * c.H;
+  // c.F is a shard's width; a whole expert's matrices are tp times that.  Gate/up rows of a shard are
+  // contiguous ([F/tp, H] at offset s*F/tp*H); a shard of the down matrix is a column slice of it (row pitch: the full width).
+  const int tp = p->tp;
+  const size_t stride = (size_t)c.F * tp * c.H;
   mark(p, 3, st);
   dim3 g1((c.F + kSimtBN - 1) / kSimtBN, (unsigned)p->P);
   launch_pdl(ffn_simt_kernel<XT, true>, g1, dim3(kSimtThreads), 0, st, (const XT*)recv, c.H, tile_expert,
-             (const XT*)wg, (const XT*)wu, stride, c.F, c.H, (XT*)p->s.inter, c.F);
+             (const XT*)wg, (const XT*)wu, stride, tp, (size_t)c.F * c.H, c.H, c.F, c.H, (XT*)p->s.inter, c.F);
   mark(p, 4, st);
   dim3 g2((c.H + kSimtBN - 1) / kSimtBN, (unsigned)p->P);
   launch_pdl(ffn_simt_kernel<XT, false>, g2, dim3(kSimtThreads), 0, st, (const XT*)p->s.inter, c.F, tile_expert,
-             (const XT*)wd, (const XT*)nullptr, stride, c.H, c.F, (XT*)out_rows, c.H);
+             (const XT*)wd, (const XT*)nullptr, stride, tp, (size_t)c.F, c.F * tp, c.H, c.F, (XT*)out_rows, c.H);
   p->launches += 2;
   return (int)cudaGetLastError();
 }

@@ -298,13 +298,13 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
               tma_load_3d_hint(b_dst, &map_bg, full, kb * kBK, it.nb * 128, it.e, pol_stream);
               tma_load_3d_hint(b_dst + kBBytes / 2, &map_bu, full, kb * kBK, it.nb * 128, it.e, pol_stream);
             } else {
-              tma_load_3d_hint(b_dst, &map_bd, full, kb * kBK, it.nb * 256, it.e, pol_stream);
+              tma_load_4d_hint(b_dst, &map_bd, full, kb * kBK, it.nb * 256, it.e % prm.tp, it.e / prm.tp, pol_stream);
             }
           } else if (it.type == 0) {
             tma_load_3d(b_dst, &map_bg, full, kb * kBK, it.nb * 128, it.e);
             tma_load_3d(b_dst + kBBytes / 2, &map_bu, full, kb * kBK, it.nb * 128, it.e);
           } else {
-            tma_load_3d(b_dst, &map_bd, full, kb * kBK, it.nb * 256, it.e);
+            tma_load_4d(b_dst, &map_bd, full, kb * kBK, it.nb * 256, it.e % prm.tp, it.e / prm.tp);
           }
 #pragma unroll
           for (int s = 0; s < kStages; ++s)
@@ -590,6 +590,20 @@ OrderedParams make_ordered_params(moe_plan* p, const void* x, const int* topk_id
 
 // overlap_x / overlap_idx != nullptr: the overlapped form - the launch that runs the GEMM1 items also
 // dispatches x (ordered scheme, into recv and the plan's own dispatch outputs) on its first CTAs.
+// The down matrices [E, H, F*tp] seen as [E, tp, H, F]: shard s of an expert is the column slice [s*F, (s+1)*F).
+// Box [1, 1, box_rows, 64].
+static int make_map_wd(EncodeTiledFn enc, CUtensorMap* m, const void* base, uint64_t experts, uint64_t tp, uint64_t rows,
+                       uint64_t cols, uint32_t box_rows) {
+  cuuint64_t dims[4] = {cols, rows, tp, experts};
+  cuuint64_t strides[3] = {cols * tp * 2, cols * 2, rows * cols * tp * 2};
+  cuuint32_t box[4] = {(cuuint32_t)kBK, box_rows, 1, 1};
+  cuuint32_t estr[4] = {1, 1, 1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MOE_OK : MOE_ERR_CUDA;
+}
+
 int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const void* wg, const void* wu,
                   const void* wd, void* out_rows, const int* tile_count, const int* rows_done, cudaStream_t st,
                   const void* overlap_x, const int* overlap_idx, const int* push_src) {
@@ -604,7 +618,12 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   if ((rc = make_map_3d(enc, &bg, wg, c.E, c.F, c.H, 128)) != MOE_OK) return rc;
   if ((rc = make_map_3d(enc, &bu, wu, c.E, c.F, c.H, 128)) != MOE_OK) return rc;
   if ((rc = make_map_2d(enc, &a2, p->s.inter, pool_rows, c.F, kTileRows)) != MOE_OK) return rc;
-  if ((rc = make_map_3d(enc, &bd, wd, c.E, c.H, c.F, c.ffn_kernel == 2 ? 128 : 256)) != MOE_OK) return rc;
+  if (c.ffn_kernel == 2) {  // the pair kernel: 3-D map, no TP shards
+    if (p->tp != 1) return MOE_ERR_UNSUPPORTED;
+    if ((rc = make_map_3d(enc, &bd, wd, c.E, c.H, c.F, 128)) != MOE_OK) return rc;
+  } else if ((rc = make_map_wd(enc, &bd, wd, c.E / p->tp, p->tp, c.H, c.F, 256)) != MOE_OK) {
+    return rc;
+  }
   CUtensorMap a1t, a2t;  // the first kThinRows rows of a tile, for tiles computed the other way round
   if ((rc = make_map_2d(enc, &a1t, recv, pool_rows, c.H, kThinRows)) != MOE_OK) return rc;
   if ((rc = make_map_2d(enc, &a2t, p->s.inter, pool_rows, c.F, kThinRows)) != MOE_OK) return rc;
@@ -640,6 +659,7 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   prm.hot_min = (fused || pairs || c.ffn_hot_min_tiles <= 0) ? 0 : c.ffn_hot_min_tiles;
   prm.cold_below = prm.hot_min > 0 ? prm.hot_min : 3;
   prm.thin = c.ffn_thin_tiles >= 0;
+  prm.tp = p->tp;
   prm.E = c.E;
   prm.F = c.F;
   prm.H = c.H;

@@ -22,8 +22,10 @@ namespace moehub {
 // in shared memory.
 // s_hist (shared memory, [E], or nullptr): every pick is also counted per expert.
 template <int EP>
+// tp > 1 (expert + tensor parallelism, paper Section VII): every pick is listed once per TP shard, as the
+// virtual expert e*tp + s with the pick's weight, so that the dispatch stores the row into every shard's region.
 __device__ __forceinline__ void select_topk(const float* ls, int tvalid, int t0, int E, int K, int renorm,
-                                            int* __restrict__ topk_idx, float* __restrict__ topk_w, int* s_hist) {
+                                            int* __restrict__ topk_idx, float* __restrict__ topk_w, int* s_hist, int tp) {
   constexpr int NJ = (EP + 31) / 32;
   const int warp = threadIdx.x / 32, lane = threadIdx.x % 32;
   for (int tl = warp; tl < tvalid; tl += blockDim.x / 32) {
@@ -70,9 +72,12 @@ __device__ __forceinline__ void select_topk(const float* ls, int tvalid, int t0,
       p = p / s;
     }
     if (lane < K) {
-      topk_idx[(size_t)(t0 + tl) * K + lane] = my_e;
-      topk_w[(size_t)(t0 + tl) * K + lane] = p;
-      if (s_hist != nullptr) atomicAdd(&s_hist[my_e], 1);
+      for (int sh = 0; sh < tp; ++sh) {
+        const size_t o = ((size_t)(t0 + tl) * K + lane) * tp + sh;
+        topk_idx[o] = my_e * tp + sh;
+        topk_w[o] = p;
+        if (s_hist != nullptr) atomicAdd(&s_hist[my_e * tp + sh], 1);
+      }
     }
   }
 }
@@ -142,7 +147,7 @@ template <typename XT, int TMT>
 __global__ void __launch_bounds__(kWideThreads)
 route_wide_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias, int T,
                   int H, int E, int K, int renorm, int* __restrict__ topk_idx, float* __restrict__ topk_w,
-                  const PrepArgs prep) {
+                  const PrepArgs prep, int tp) {
   constexpr int TB = 8 * TMT;  // tokens per CTA: 4 warps x 2 lane groups x TMT
   extern __shared__ __align__(16) float smem[];
   __shared__ int s_hist[kRouteMaxExperts];
@@ -254,7 +259,7 @@ route_wide_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const flo
     }
   }
   __syncthreads();
-  select_topk<kWideEP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w, prep.hist ? s_hist : nullptr);
+  select_topk<kWideEP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w, prep.hist ? s_hist : nullptr, tp);
   route_prep_end(prep, s_hist);
 }
 
@@ -269,7 +274,7 @@ static int launch_wide_tmt(moe_plan* p, const void* x, const void* wr, const flo
   const moe_config_t& c = p->cfg;
   p->launches += 1;
   return (int)launch_maybe_pdl(false, kern, dim3((c.T + 8 * TMT - 1) / (8 * TMT)), dim3(kWideThreads), smem, st,
-                               (const XT*)x, (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w, prep);
+                               (const XT*)x, (const XT*)wr, bias, c.T, c.H, p->route_E, p->route_K, c.renormalize, topk_idx, topk_w, prep, p->tp);
 }
 
 template <typename XT>
@@ -367,7 +372,7 @@ template <typename XT, bool SWAP, int EW, int TWP, int HC>
 __global__ void __launch_bounds__(32 * (EW * TWP + kNarrowFillWarps))
 route_narrow_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const float* __restrict__ bias, int T,
                     int H, int E, int K, int renorm, int* __restrict__ topk_idx, float* __restrict__ topk_w,
-                    const PrepArgs prep) {
+                    const PrepArgs prep, int tp) {
   __shared__ int s_hist[kRouteMaxExperts];
   constexpr int TN = 2;                    // experts per lane
   constexpr int G = SWAP ? 16 : 2;         // expert groups per warp
@@ -477,7 +482,7 @@ route_narrow_kernel(const XT* __restrict__ x, const XT* __restrict__ wr, const f
     }
   }
   __syncthreads();
-  select_topk<EP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w, prep.hist ? s_hist : nullptr);
+  select_topk<EP>(ls, tvalid, t0, E, K, renorm, topk_idx, topk_w, prep.hist ? s_hist : nullptr, tp);
   route_prep_end(prep, s_hist);
 }
 
@@ -493,7 +498,7 @@ static int launch_narrow(moe_plan* p, const void* x, const void* wr, const float
   const moe_config_t& c = p->cfg;
   p->launches += 1;
   return (int)launch_maybe_pdl(false, kern, dim3((c.T + TB - 1) / TB), dim3(32 * (EW * TWP + kNarrowFillWarps)), smem, st,
-                               (const XT*)x, (const XT*)wr, bias, c.T, c.H, c.E, c.K, c.renormalize, topk_idx, topk_w, prep);
+                               (const XT*)x, (const XT*)wr, bias, c.T, c.H, p->route_E, p->route_K, c.renormalize, topk_idx, topk_w, prep, p->tp);
 }
 
 template <typename XT>
@@ -503,10 +508,11 @@ static int launch_typed(moe_plan* p, const void* x, const void* wr, const float*
   // 16 tokens x 2 expert groups per warp, two compute warps per CTA (32 tokens: T = 4096 gives 128
   // CTAs); with many experts 2 tokens x 16 groups, so that the chains still spread over the SMs.
   constexpr int HL = sizeof(XT) == 2 ? 256 : 128;  // h per chunk
-  if (c.E <= 8) return launch_narrow<XT, false, 2, 2, HL>(p, x, wr, bias, topk_idx, topk_w, prep, st);   // 32 tokens per CTA
-  if (c.E <= 16) return launch_narrow<XT, false, 4, 2, HL>(p, x, wr, bias, topk_idx, topk_w, prep, st);  // 32 tokens per CTA
-  if (c.E <= 32) return launch_narrow<XT, true, 1, 4, HL / 2>(p, x, wr, bias, topk_idx, topk_w, prep, st);  // 8 tokens per CTA
-  if (c.E <= 64) return launch_narrow<XT, true, 2, 2, HL / 2>(p, x, wr, bias, topk_idx, topk_w, prep, st);  // 4 tokens per CTA
+  const int E = p->route_E;  // the experts the router scores (the plan's E counts every TP shard of an expert)
+  if (E <= 8) return launch_narrow<XT, false, 2, 2, HL>(p, x, wr, bias, topk_idx, topk_w, prep, st);   // 32 tokens per CTA
+  if (E <= 16) return launch_narrow<XT, false, 4, 2, HL>(p, x, wr, bias, topk_idx, topk_w, prep, st);  // 32 tokens per CTA
+  if (E <= 32) return launch_narrow<XT, true, 1, 4, HL / 2>(p, x, wr, bias, topk_idx, topk_w, prep, st);  // 8 tokens per CTA
+  if (E <= 64) return launch_narrow<XT, true, 2, 2, HL / 2>(p, x, wr, bias, topk_idx, topk_w, prep, st);  // 4 tokens per CTA
   return launch_wide<XT>(p, x, wr, bias, topk_idx, topk_w, prep, st);
 }
 

@@ -193,8 +193,8 @@ def oracle_inputs(w: inputs.Workload, with_experts=True):
     return x, wr, bias, wg, wu, wd
 
 
-def oracle_layer_for(w: inputs.Workload, x, wr, bias, wg, wu, wd, bf16_storage=False):
+def oracle_layer_for(w: inputs.Workload, x, wr, bias, wg, wu, wd, bf16_storage=False, tp_shards=1):
     ws = (None, None, None) if wg is None else ([wg[e] for e in range(w.E)], [wu[e] for e in range(w.E)],
                                                  [wd[e] for e in range(w.E)])
     return oracle.layer(x, wr, bias, *ws, w.E, w.R, w.K, w.dtype, identity_experts=w.identity_experts,
-                        bf16_storage=bf16_storage)
+                        bf16_storage=bf16_storage, tp_shards=tp_shards)

@@ -563,6 +563,63 @@ def test_push_combine_is_refused_where_it_is_not_built():
     assert ei.value.code == -3
 
 
+# ------------------------------------------------------------------ expert + tensor parallelism
+TP_CASES = [(inputs.Workload("tp_bf16", T=333, H=264, E=12, R=3, K=3, F=400, dtype=BF16), 2),
+            (inputs.Workload("tp_bf16_4", T=700, H=320, E=4, R=2, K=2, F=1024, dtype=BF16, zipf_s=1.0), 4),
+            (inputs.Workload("tp_many", T=300, H=256, E=64, R=8, K=8, F=256, dtype=BF16, zipf_s=1.0), 4),
+            (inputs.Workload("tp_fp32", T=130, H=128, E=8, R=2, K=2, F=192, dtype=FP32), 3)]
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("case", TP_CASES, ids=lambda c: f"{c[0].name}_S{c[1]}")
+def test_tp_shards_layer_matches_oracle(case, mode):
+    """Section VII: one receive region per TP shard, every row stored to each.  Routing (every pick listed once per
+    shard), dispatch contents of the E*S regions and the output against the oracle's TP layer - which itself equals
+    the plain layer - in every dispatch scheme; the output also agrees with the same plan without shards."""
+    w, S = case
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd, tp_shards=S)
+    args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    plan = Hh.make_plan(w, mode, tp_shards=S)
+    assert plan.P == (w.T * w.K * S // 128 + w.E * S if mode != B.DISPATCH_ATOMIC_STATIC else plan.P)
+    y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
+    plan.moe_layer(*args, y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    Hh.check_route(plan.layer_tensor(0), plan.layer_tensor(1), ref["topk_idx"], ref["topk_w"])
+    ws = w.with_(E=w.E * S, K=w.K * S)
+    Hh.check_dispatch(ws, plan.P, x, ref["topk_idx"], ref, plan.layer_tensor(2), plan.layer_tensor(3),
+                      plan.layer_tensor(4), plan.layer_tensor(5), plan.layer_tensor(6))
+    Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+    plain = Hh.make_plan(w, mode)
+    y2 = torch.empty_like(y)
+    plain.moe_layer(*args, y2)
+    torch.cuda.synchronize()
+    Hh.assert_output_close(Hh.to_host_f64(y), Hh.to_host_f64(y2), w.dtype, "with and without TP shards")
+
+
+def test_tp_shards_with_overlap_and_push_combine():
+    w, S = TP_CASES[1]
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd, tp_shards=S)
+    args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, tp_shards=S, overlap=1, combine_mode=1)
+    y = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+    plan.moe_layer(*args, y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
+
+
+def test_tp_shards_limits_are_refused_on_the_host():
+    for cfg, code in [(B.make_config(64, 128, 8, 2, 2, 100, BF16, tp_shards=3), -1),     # F % S != 0
+                      (B.make_config(64, 128, 128, 2, 2, 64, BF16, tp_shards=4), -3),    # E*S > 256
+                      (B.make_config(64, 128, 64, 2, 16, 64, BF16, tp_shards=4), -3)]:   # K*S > 32
+        with pytest.raises(B.MoeError) as ei:
+            B.moe_workspace_bytes(cfg)
+        assert ei.value.code == code
+
+
 # ------------------------------------------------------------------ random small shapes
 def _random_workloads(n, seed):
     rng = np.random.default_rng(seed)

@@ -327,3 +327,29 @@ def test_inputs_are_slice_consistent_and_bf16_rounding_is_rne():
     big = np.random.default_rng(0).standard_normal(10000).astype(np.float32)
     t = torch.from_numpy(big).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
     assert np.array_equal(inputs.fp32_to_bf16_bits(big), t)
+
+
+# ---------------------------------------------------------------- expert + tensor parallelism (Section VII)
+@pytest.mark.parametrize("dtype", [FP32, BF16])
+@pytest.mark.parametrize("S", [2, 4])
+def test_tp_shards_change_the_bookkeeping_but_not_the_result(S, dtype):
+    """SwiGLU acts per FFN column and the down projection is a sum over FFN columns, so cutting an expert into S
+    slices of its width and adding the slices' outputs gives the expert's output: the layer with TP shards must
+    equal the plain layer (fp64: to rounding).  A slice taken from the wrong matrix axis, a pick's weight not
+    carried to its shards, or a row missing from a shard's region breaks the equality.  The bookkeeping is that
+    of E*S experts: every shard of a picked expert receives the row."""
+    w = inputs.Workload("tp", T=37, H=24, E=6, R=3, K=2, F=16 * S, dtype=dtype, zipf_s=1.0, seed=4)
+    x = inputs.make_x(w)
+    wr, bias = inputs.make_router(w)
+    wg, wu, wd = (list(a) for a in inputs.make_all_expert_weights(w))
+    plain = oracle.layer(x, wr, bias, wg, wu, wd, w.E, w.R, w.K, dtype)
+    tp = oracle.layer(x, wr, bias, wg, wu, wd, w.E, w.R, w.K, dtype, tp_shards=S)
+    assert np.abs(tp["y"] - plain["y"]).max() <= 1e-12 * np.abs(plain["y"]).max()
+    assert tp["topk_idx"].shape == (w.T, w.K * S)
+    assert np.array_equal(tp["topk_idx"] // S, np.repeat(plain["topk_idx"], S, axis=1))
+    assert np.array_equal(tp["topk_idx"] % S, np.tile(np.arange(S), (w.T, w.K)))
+    assert np.array_equal(tp["topk_w"], np.repeat(plain["topk_w"], S, axis=1))
+    assert np.array_equal(tp["count"], np.repeat(plain["count"], S))            # every shard gets every row of its expert
+    assert tp["count"].sum() == w.T * w.K * S
+    rows = tp["recv"][tp["slot_of"].ravel()]
+    assert rows.tobytes() == np.repeat(x, w.K * S, axis=0).tobytes()
