@@ -237,6 +237,40 @@ int moe_expert_ffn_push(moe_plan_t* plan, const void* d_recv, const int32_t* d_t
 int moe_combine_staged(moe_plan_t* plan, const void* d_staged, const int32_t* d_slot_of,
                        const float* d_topk_w, void* d_y, void* stream);
 
+/* Dispatch across GPUs - real expert parallelism, the paper's own setting (Section III-B: producers send
+ * without knowing the destination's layout; Section IV-B: the CONSUMER's allocation pointers hand out the
+ * rows).  Rank r of cfg->R holds cfg->T tokens (its share of the batch) and the experts
+ * [r*E/R, (r+1)*E/R); cfg->E counts all experts.  Every rank owns, in its own memory, one static region of
+ * cap_rows rows per local expert plus the counters below, and makes them reachable by the other ranks
+ * (CUDA IPC, a symmetric-memory allocator, or - on one GPU - plain local pointers).  The call dispatches THIS
+ * rank's tokens: for every token block one system-scope atomicAdd per touched expert on the owner's
+ * row_pointer, the rows by plain 16-byte stores into the owner's region, then system-scope release
+ * increments of the owner's tile and global counters.  Nothing but ordinary loads, stores and atomics
+ * touches another GPU's memory (no TMA, no bulk copy, no multicast, no library kernel), and the kernel waits
+ * for nobody, so no two ranks need to run at the same time.
+ *
+ * Before any rank dispatches, every rank clears ITS OWN row_pointer, tile_count and rows_done and fills its
+ * src_info with -1, and the ranks synchronise (host barrier or events): that start state is the caller's job.
+ * h_peers: HOST array [R] of device pointers valid on the calling GPU, entry r describing rank r's buffers:
+ *   recv [E/R * cap_rows, H] (dtype), row_pointer [E/R], tile_count [E/R * cap_rows/128],
+ *   src_info [E/R * cap_rows] (receives (source rank * T + t) * K + k), rows_done [1] (assignments addressed
+ *   to this rank, dropped ones included).
+ * cap_rows: multiple of 128; an assignment beyond it is dropped and reported (MOE_ERR_OVERFLOW).
+ * out: d_slot_of [T,K] = owner rank * (E/R * cap_rows) + row in the owner's regions, or -1;
+ *      d_status [2] device status (code, detail) of this call.
+ * Limits: R <= MOE_EP_MAX_RANKS, E <= 256, K <= 32.  Not yet measured on more than one GPU. */
+#define MOE_EP_MAX_RANKS 32
+typedef struct {
+  void* recv;
+  int32_t* row_pointer;
+  int32_t* tile_count;
+  int32_t* src_info;
+  int32_t* rows_done;
+} moe_ep_peer_t;
+int moe_dispatch_ep(const moe_config_t* cfg, int32_t rank, const moe_ep_peer_t* h_peers, int64_t cap_rows,
+                    const void* d_x, const int32_t* d_topk_idx, int32_t* d_slot_of, int32_t* d_status,
+                    void* stream);
+
 /* Steps 4+5 (Section II-A, combine and scaling): y[t,:] = sum_k w[t,k]*rows[slot_of[t,k],:],
  * k ascending, fp32 accumulation, rounded once to dtype.  Assignments with slot -1 add 0.
  * in: d_rows [P*128,H] (dtype), d_slot_of [T,K], d_topk_w [T,K].  out: d_y [T,H] (dtype). */

@@ -21,7 +21,7 @@ DISPATCH_SCAN, DISPATCH_ATOMIC_STATIC, DISPATCH_ATOMIC_PAGED, DISPATCH_ATOMIC_OR
 TILE_ROWS = 128
 STAGES = ["route", "dispatch", "worklist", "gemm1", "gemm2", "combine"]
 
-EXPORTS = ["moe_dispatch_noalloc", "moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
+EXPORTS = ["moe_dispatch_noalloc", "moe_dispatch_ep", "moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
            "moe_dispatch", "moe_expert_ffn", "moe_expert_ffn_push", "moe_combine", "moe_combine_staged", "moe_layer", "moe_layer_host", "moe_layer_host_submit", "moe_layer_host_wait", "moe_layer_timed",
            "moe_layer_buffer", "moe_availability_trace",
            "moe_ffn_clock_mhz", "moe_last_launch_count", "moe_last_status", "moe_last_cuda_error", "moe_strerror"]
@@ -36,6 +36,12 @@ class MoeConfig(ctypes.Structure):
                 ("overlap", ctypes.c_int32), ("combine_mode", ctypes.c_int32),
                 ("tp_shards", ctypes.c_int32), ("reserved_", ctypes.c_int32),
                 ("capacity_rows", ctypes.c_int64), ("spin_limit", ctypes.c_uint64), ("wait_limit_ns", ctypes.c_uint64)]
+
+
+class EpPeer(ctypes.Structure):
+    """moe_ep_peer_t: one rank's receive buffers as device pointers valid on the calling GPU."""
+    _fields_ = [("recv", ctypes.c_void_p), ("row_pointer", ctypes.c_void_p), ("tile_count", ctypes.c_void_p),
+                ("src_info", ctypes.c_void_p), ("rows_done", ctypes.c_void_p)]
 
 
 class MoeError(RuntimeError):
@@ -60,6 +66,7 @@ def lib() -> ctypes.CDLL:
         L.moe_route.argtypes = [vp, vp, vp, fp, i32p, fp, vp]
         L.moe_dispatch.argtypes = [vp, vp, i32p, vp, i32p, i32p, i32p, i32p, i32p, i32p, vp]
         L.moe_dispatch_noalloc.argtypes = [cfgp, vp, i32p, vp, i32p, i32p, i32p, i32p, i32p, vp]
+        L.moe_dispatch_ep.argtypes = [cfgp, ctypes.c_int32, ctypes.POINTER(EpPeer), ctypes.c_int64, vp, i32p, i32p, i32p, vp]
         L.moe_expert_ffn.argtypes = [vp, vp, i32p, vp, vp, vp, vp, i32p, i32p, vp]
         L.moe_combine.argtypes = [vp, vp, i32p, fp, vp, vp]
         L.moe_expert_ffn_push.argtypes = [vp, vp, i32p, i32p, vp, vp, vp, vp, i32p, i32p, vp]
@@ -135,6 +142,17 @@ def moe_dispatch_noalloc(cfg: MoeConfig, x, topk_idx, recv, expert_count, tile_e
     _check(lib().moe_dispatch_noalloc(ctypes.byref(cfg), _ptr(x), _ptr(topk_idx), _ptr(recv), _ptr(expert_count),
                                       _ptr(tile_expert), _ptr(src_info), _ptr(slot_of), _ptr(status),
                                       _stream(stream)), "moe_dispatch_noalloc")
+
+
+def moe_dispatch_ep(cfg: MoeConfig, rank: int, peers, cap_rows: int, x, topk_idx, slot_of, status, stream=None) -> None:
+    """Dispatch of THIS rank's tokens into the owning ranks' receive regions (real expert parallelism).
+    peers: one dict per rank with the tensors (or device pointers valid on this GPU) recv, row_pointer, tile_count,
+    src_info, rows_done.  cfg.T is this rank's token count, cfg.E the experts of all ranks."""
+    table = (EpPeer * len(peers))()
+    for r, q in enumerate(peers):
+        table[r] = EpPeer(*(_ptr(q[k]) for k in ("recv", "row_pointer", "tile_count", "src_info", "rows_done")))
+    _check(lib().moe_dispatch_ep(ctypes.byref(cfg), rank, table, cap_rows, _ptr(x), _ptr(topk_idx), _ptr(slot_of),
+                                 _ptr(status), _stream(stream)), "moe_dispatch_ep")
 
 
 class Plan:
