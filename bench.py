@@ -31,6 +31,9 @@ UNIT = "tokens/s"
 WORKLOADS = {"c1": inputs.C1, "c2": inputs.C2, "c3": inputs.C3, "c4": inputs.C4,
              # a quarter-size C2 (same kernels, 0.7 GB of weights) for ncu captures that must stay small
              "c2_small": inputs.C2.with_(name="mixtral_like_bf16_small", T=2048, E=4, R=4, F=7168),
+             # a reduced DeepSeek-V3-like layer (same H, F, top-8 and Zipf bias; 32 experts, 1024 tokens: 2.8 GB of
+             # weights) for ncu captures of the expert kernel in its skewed, weight-streaming regime
+             "c3_small": inputs.C3.with_(name="deepseek_v3_like_bf16_small", T=1024, E=32, R=4),
              # the other two shapes of the paper's Table II
              "phi35": inputs.PHI35, "qwen64": inputs.QWEN64,
              # dispatch/combine-only sweep points (identity experts)
