@@ -135,6 +135,7 @@ class ClockSampler(threading.Thread):
     def __init__(self, index: int):
         super().__init__(daemon=True)
         self.samples, self.reasons, self.max_mhz = [], set(), None
+        self.power_w, self.power_limit_w = [], None
         self._stop_evt = threading.Event()
         self.ok = False
         try:
@@ -143,6 +144,10 @@ class ClockSampler(threading.Thread):
             pynvml.nvmlInit()
             self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
             self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            try:
+                self.power_limit_w = pynvml.nvmlDeviceGetEnforcedPowerLimit(self.h) / 1000.0
+            except Exception:
+                self.power_limit_w = None
             self.ok = True
         except Exception:
             self.ok = False
@@ -166,6 +171,10 @@ class ClockSampler(threading.Thread):
                         self.reasons.add(name)
             except Exception:
                 pass
+            try:  # board power (NVML averages it over a window of its own, so short runs under-read)
+                self.power_w.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+            except Exception:
+                pass
             self._stop_evt.wait(0.005)
 
     def stop(self) -> dict:
@@ -174,7 +183,8 @@ class ClockSampler(threading.Thread):
             self.join(1.0)
         med = float(np.median(self.samples)) if self.samples else None
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                "samples": len(self.samples),
+                "power_w_max": (round(max(self.power_w), 1) if self.power_w else None), "power_limit_w": self.power_limit_w}
 
 
 def max_over_ranks(values: list[float], device: str = "cpu") -> list[float]:
