@@ -271,6 +271,30 @@ int moe_dispatch_ep(const moe_config_t* cfg, int32_t rank, const moe_ep_peer_t* 
                     const void* d_x, const int32_t* d_topk_idx, int32_t* d_slot_of, int32_t* d_status,
                     void* stream);
 
+/* After every rank's moe_dispatch_ep has completed (host barrier): the owner's tile table from its allocation
+ * pointers, in the form moe_expert_ffn takes for static regions of cap_rows rows - expert e of this rank holds
+ * min(row_pointer[e], cap_rows) rows in the first tiles of region e, the region's other tiles are unused.
+ * in: d_row_pointer [experts_local].  out: d_expert_count [experts_local], d_tile_expert
+ * [experts_local * cap_rows/128] (local expert index, or -1).  One small launch on `stream`. */
+int moe_ep_tiles(int32_t experts_local, int64_t cap_rows, const int32_t* d_row_pointer,
+                 int32_t* d_expert_count, int32_t* d_tile_expert, void* stream);
+
+/* The combine direction across GPUs (Section IV-B, all-to-all combine): the owner reads the source
+ * information of every result row and stores the row at the token's own position - row t*K+k of the SOURCE
+ * rank's staging buffer [T*K, H] - with plain 16-byte peer stores, then raises that rank's counter of returned
+ * rows with a system-scope release add.  The source rank then runs moe_combine_staged on its staging buffer
+ * (after a host barrier, or once rows_back has reached the number of its assignments that were not dropped).
+ * cfg as for moe_dispatch_ep (T = tokens per rank, E = all experts).  h_staging, h_rows_back: HOST arrays [R]
+ * of device pointers valid on the calling GPU (rank r's staging buffer; its int32 counter, zero before the
+ * step).  in: d_out_rows [E/R * cap_rows, H] (this rank's expert outputs, same rows as its receive regions),
+ * d_src_info [E/R * cap_rows], d_expert_count [E/R] (from moe_ep_tiles).  out: d_status [2]; a row without
+ * valid source information is reported as MOE_ERR_INTERNAL and not sent.  Same rule as the dispatch: only
+ * ordinary loads, stores and atomics touch peer memory, and the kernel waits for nobody.  Not yet measured on
+ * more than one GPU. */
+int moe_combine_ep(const moe_config_t* cfg, void* const* h_staging, int32_t* const* h_rows_back,
+                   int64_t cap_rows, const void* d_out_rows, const int32_t* d_src_info,
+                   const int32_t* d_expert_count, int32_t* d_status, void* stream);
+
 /* Steps 4+5 (Section II-A, combine and scaling): y[t,:] = sum_k w[t,k]*rows[slot_of[t,k],:],
  * k ascending, fp32 accumulation, rounded once to dtype.  Assignments with slot -1 add 0.
  * in: d_rows [P*128,H] (dtype), d_slot_of [T,K], d_topk_w [T,K].  out: d_y [T,H] (dtype). */

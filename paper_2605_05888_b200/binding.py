@@ -21,7 +21,7 @@ DISPATCH_SCAN, DISPATCH_ATOMIC_STATIC, DISPATCH_ATOMIC_PAGED, DISPATCH_ATOMIC_OR
 TILE_ROWS = 128
 STAGES = ["route", "dispatch", "worklist", "gemm1", "gemm2", "combine"]
 
-EXPORTS = ["moe_dispatch_noalloc", "moe_dispatch_ep", "moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
+EXPORTS = ["moe_dispatch_noalloc", "moe_dispatch_ep", "moe_ep_tiles", "moe_combine_ep", "moe_pool_tiles", "moe_workspace_bytes", "moe_plan_create", "moe_plan_destroy", "moe_route",
            "moe_dispatch", "moe_expert_ffn", "moe_expert_ffn_push", "moe_combine", "moe_combine_staged", "moe_layer", "moe_layer_host", "moe_layer_host_submit", "moe_layer_host_wait", "moe_layer_timed",
            "moe_layer_buffer", "moe_availability_trace",
            "moe_ffn_clock_mhz", "moe_last_launch_count", "moe_last_status", "moe_last_cuda_error", "moe_strerror"]
@@ -67,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.moe_dispatch.argtypes = [vp, vp, i32p, vp, i32p, i32p, i32p, i32p, i32p, i32p, vp]
         L.moe_dispatch_noalloc.argtypes = [cfgp, vp, i32p, vp, i32p, i32p, i32p, i32p, i32p, vp]
         L.moe_dispatch_ep.argtypes = [cfgp, ctypes.c_int32, ctypes.POINTER(EpPeer), ctypes.c_int64, vp, i32p, i32p, i32p, vp]
+        L.moe_ep_tiles.argtypes = [ctypes.c_int32, ctypes.c_int64, i32p, i32p, i32p, vp]
+        L.moe_combine_ep.argtypes = [cfgp, ctypes.POINTER(vp), ctypes.POINTER(vp), ctypes.c_int64, vp, i32p, i32p, i32p, vp]
         L.moe_expert_ffn.argtypes = [vp, vp, i32p, vp, vp, vp, vp, i32p, i32p, vp]
         L.moe_combine.argtypes = [vp, vp, i32p, fp, vp, vp]
         L.moe_expert_ffn_push.argtypes = [vp, vp, i32p, i32p, vp, vp, vp, vp, i32p, i32p, vp]
@@ -153,6 +155,23 @@ def moe_dispatch_ep(cfg: MoeConfig, rank: int, peers, cap_rows: int, x, topk_idx
         table[r] = EpPeer(*(_ptr(q[k]) for k in ("recv", "row_pointer", "tile_count", "src_info", "rows_done")))
     _check(lib().moe_dispatch_ep(ctypes.byref(cfg), rank, table, cap_rows, _ptr(x), _ptr(topk_idx), _ptr(slot_of),
                                  _ptr(status), _stream(stream)), "moe_dispatch_ep")
+
+
+def moe_ep_tiles(experts_local: int, cap_rows: int, row_pointer, expert_count, tile_expert, stream=None) -> None:
+    """The owner's tile table (static regions of cap_rows rows) from its allocation pointers."""
+    _check(lib().moe_ep_tiles(experts_local, cap_rows, _ptr(row_pointer), _ptr(expert_count), _ptr(tile_expert),
+                              _stream(stream)), "moe_ep_tiles")
+
+
+def moe_combine_ep(cfg: MoeConfig, staging, rows_back, cap_rows: int, out_rows, src_info, expert_count, status,
+                   stream=None) -> None:
+    """The owner's result rows back to their source ranks' staging buffers.  staging, rows_back: one tensor (or
+    device pointer valid on this GPU) per rank."""
+    n = len(staging)
+    st = (ctypes.c_void_p * n)(*(_ptr(t) for t in staging))
+    rb = (ctypes.c_void_p * n)(*(_ptr(t) for t in rows_back))
+    _check(lib().moe_combine_ep(ctypes.byref(cfg), st, rb, cap_rows, _ptr(out_rows), _ptr(src_info), _ptr(expert_count),
+                                _ptr(status), _stream(stream)), "moe_combine_ep")
 
 
 class Plan:

@@ -122,7 +122,103 @@ dispatch_ep_kernel(const uint4* __restrict__ x, const int* __restrict__ topk_idx
   }
 }
 
+// The owner's tile table from its allocation pointers, once every producer has finished: region e holds
+// min(row_pointer[e], cap_rows) rows in its first tiles; the other tiles of the region are unused.
+__global__ void ep_tiles_kernel(const int* __restrict__ row_pointer, int epr, int cap_rows, int* __restrict__ expert_count,
+                                int* __restrict__ tile_expert) {
+  const int tiles_per = cap_rows / kTileRows;
+  const int tile = blockIdx.x * blockDim.x + threadIdx.x;
+  if (tile >= epr * tiles_per) return;
+  const int e = tile / tiles_per, i = tile % tiles_per;
+  const int cnt = max(0, min(row_pointer[e], cap_rows));
+  tile_expert[tile] = i * kTileRows < cnt ? e : -1;
+  if (i == 0) expert_count[e] = cnt;
+}
+
+// The combine direction (Section IV-B, all-to-all combine): the owner reads every result row's source
+// information (source rank, token, k) and stores the row at the token's own position, row t*K+k of the source
+// rank's staging buffer [T*K, H] - plain 16-byte peer stores again.  After a CTA's stores are visible
+// system-wide it raises the source rank's counter of returned rows by the rows it sent there, so that rank
+// knows its T*K rows (minus dropped ones) are back without hearing from anybody.
+struct EpStaging {
+  uint4* staging[kEpMaxRanks];
+  int* rows_back[kEpMaxRanks];
+};
+
+__global__ void __launch_bounds__(kEpThreads)
+combine_ep_kernel(const uint4* __restrict__ out_rows, const int* __restrict__ src_info, const int* __restrict__ expert_count,
+                  int cap_rows, int vec_per_row, int rows_per_rank /* T*K */, int R, const EpStaging peers,
+                  int* __restrict__ status) {
+  __shared__ int s_sent[kEpMaxRanks];
+  const int tiles_per = cap_rows / kTileRows;
+  const int e = blockIdx.x / tiles_per, i = blockIdx.x % tiles_per;
+  const int rows = min(kTileRows, expert_count[e] - i * kTileRows);
+  if (rows <= 0) return;
+  const int lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+  if (threadIdx.x < kEpMaxRanks) s_sent[threadIdx.x] = 0;
+  __syncthreads();
+  const size_t row0 = (size_t)e * cap_rows + (size_t)i * kTileRows;
+  for (int r = warp; r < rows; r += kEpThreads / 32) {
+    const int src = src_info[row0 + r];
+    const int dst = src / rows_per_rank;
+    if (src < 0 || dst >= R) {  // a row nobody registered: report it, send nothing
+      if (lane == 0) set_status(status, MOE_ERR_INTERNAL, 301);
+      continue;
+    }
+    const uint4* from = out_rows + (row0 + r) * vec_per_row;
+    uint4* to = peers.staging[dst] + (size_t)(src % rows_per_rank) * vec_per_row;
+    for (int v = lane; v < vec_per_row; v += 32) to[v] = __ldg(from + v);
+    if (lane == 0) atomicAdd(&s_sent[dst], 1);
+  }
+  __threadfence_system();
+  __syncthreads();
+  if (threadIdx.x < R && s_sent[threadIdx.x] != 0)
+    asm volatile("red.release.sys.global.add.s32 [%0], %1;" ::"l"(peers.rows_back[threadIdx.x]), "r"(s_sent[threadIdx.x]) : "memory");
+}
+
 }  // namespace moehub
+
+extern "C" int moe_ep_tiles(int32_t experts_local, int64_t cap_rows, const int32_t* d_row_pointer, int32_t* d_expert_count,
+                            int32_t* d_tile_expert, void* stream) {
+  using namespace moehub;
+  if (experts_local <= 0 || cap_rows <= 0 || cap_rows % kTileRows != 0) return MOE_ERR_ARG;
+  if (!d_row_pointer || !d_expert_count || !d_tile_expert) return MOE_ERR_ARG;
+  if ((int64_t)experts_local * cap_rows >= (1ll << 31)) return MOE_ERR_UNSUPPORTED;
+  const int tiles = experts_local * (int)(cap_rows / kTileRows);
+  ep_tiles_kernel<<<(tiles + 127) / 128, 128, 0, (cudaStream_t)stream>>>(d_row_pointer, experts_local, (int)cap_rows,
+                                                                        d_expert_count, d_tile_expert);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
+
+extern "C" int moe_combine_ep(const moe_config_t* cfg, void* const* h_staging, int32_t* const* h_rows_back, int64_t cap_rows,
+                              const void* d_out_rows, const int32_t* d_src_info, const int32_t* d_expert_count,
+                              int32_t* d_status, void* stream) {
+  using namespace moehub;
+  if (!cfg || !h_staging || !h_rows_back || !d_status) return MOE_ERR_ARG;
+  const moe_config_t& c = *cfg;
+  if (c.T < 0 || c.H <= 0 || c.E <= 0 || c.R <= 0 || c.K <= 0 || c.E % c.R != 0) return MOE_ERR_ARG;
+  if (cap_rows <= 0 || cap_rows % kTileRows != 0) return MOE_ERR_ARG;
+  if (c.dtype != MOE_DTYPE_FP32 && c.dtype != MOE_DTYPE_BF16) return MOE_ERR_ARG;
+  if (c.R > kEpMaxRanks) return MOE_ERR_UNSUPPORTED;
+  if (!d_out_rows || !d_src_info || !d_expert_count) return MOE_ERR_ARG;
+  const int eb = c.dtype == MOE_DTYPE_BF16 ? 2 : 4;
+  if (((int64_t)c.H * eb) % 16 != 0 || (reinterpret_cast<uintptr_t>(d_out_rows) & 15)) return MOE_ERR_ALIGN;
+  if ((int64_t)c.R * c.T * c.K >= (1ll << 31) || (int64_t)(c.E / c.R) * cap_rows >= (1ll << 31)) return MOE_ERR_UNSUPPORTED;
+  EpStaging peers = {};
+  for (int r = 0; r < c.R; ++r) {
+    if (!h_staging[r] || !h_rows_back[r]) return MOE_ERR_ARG;
+    if (reinterpret_cast<uintptr_t>(h_staging[r]) & 15) return MOE_ERR_ALIGN;
+    peers.staging[r] = (uint4*)h_staging[r];
+    peers.rows_back[r] = h_rows_back[r];
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  if (cudaMemsetAsync(d_status, 0, 2 * sizeof(int), st) != cudaSuccess) return MOE_ERR_CUDA;
+  if (c.T == 0) return MOE_OK;  // with no tokens per rank nothing was dispatched
+  const int tiles = (c.E / c.R) * (int)(cap_rows / kTileRows);
+  combine_ep_kernel<<<tiles, kEpThreads, 0, st>>>((const uint4*)d_out_rows, d_src_info, d_expert_count, (int)cap_rows,
+                                                  c.H * eb / 16, c.T * c.K, c.R, peers, d_status);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ERR_CUDA;
+}
 
 extern "C" int moe_dispatch_ep(const moe_config_t* cfg, int32_t rank, const moe_ep_peer_t* h_peers, int64_t cap_rows,
                                const void* d_x, const int32_t* d_topk_idx, int32_t* d_slot_of, int32_t* d_status,

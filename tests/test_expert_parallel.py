@@ -155,3 +155,64 @@ def test_peer_dispatch_reports_a_full_region():
     s = so.cpu().numpy().ravel()
     assert (s >= 0).sum() == 128 and (s == -1).sum() == T - 128
     assert int(bufs[1]["rows_done"][0]) == T and torch.all(guard[2 * 128:] == 5.0)
+
+
+def ep_layer_problem(T, H, E, K, F, R, dtype):
+    import parity_helpers as Hh
+    w = inputs.Workload("ep_layer", T=T, H=H, E=E, R=R, K=K, F=F, dtype=dtype, zipf_s=0.8, seed=11)
+    return (w,) + Hh.oracle_inputs(w)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("R,dtype", [(2, inputs.BF16), (4, inputs.BF16), (2, inputs.FP32)])
+def test_expert_parallel_layer_ranks_run_phase_by_phase_on_one_gpu(R, dtype):
+    """The whole destination-agnostic layer over R ranks - route, peer dispatch, experts on the owner, result rows
+    pushed back to the source rank's staging buffer, weighted sum - against the oracle's plain layer on the whole
+    batch.  The ranks are objects in one process and run phase by phase; every peer pointer is local memory."""
+    import parity_helpers as Hh
+    T, H, E, K, F = 384, 256, 8, 2, 128
+    w, x, wr, bias, wg, wu, wd = ep_layer_problem(T, H, E, K, F, R, dtype)
+    Tl, epr = T // R, E // R
+    ranks = [ep.EpRank(r, R, Tl, H, E, K, F, dtype) for r in range(R)]
+    xs = [Hh.to_dev(np.ascontiguousarray(x[r * Tl:(r + 1) * Tl]), dtype) for r in range(R)]
+    dwr, dbias = Hh.to_dev(wr, dtype), Hh.to_dev(bias)
+    shard = lambda m: [Hh.to_dev(np.ascontiguousarray(m[r * epr:(r + 1) * epr]), dtype) for r in range(R)]
+    ys = [torch.empty((Tl, H), dtype=ranks[0].el, device="cuda") for _ in range(R)]
+    ref = Hh.oracle_layer_for(w, x, wr, bias, wg, wu, wd)
+    for _ in range(2):                       # a second step finds every counter back in its start state
+        for y in ys:
+            y.zero_()
+        ep.run_in_process(ranks, xs, dwr, dbias, shard(wg), shard(wu), shard(wd), ys)
+        got = np.concatenate([Hh.to_host_f64(y) for y in ys])
+        Hh.assert_output_close(got, ref["y"], dtype, f"EP layer, R = {R}")
+    for r, rk in enumerate(ranks):
+        assert int(rk.own["rows_back"][0]) == Tl * K
+        assert np.array_equal(rk.expert_count.cpu().numpy(), ref["count"][r * epr:(r + 1) * epr])
+        assert int(rk.own["rows_done"][0]) == ref["rank_count"][r]
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("R", [2, 3])
+def test_expert_parallel_layer_one_process_per_rank_through_cuda_ipc(R):
+    """The same layer with one PROCESS per rank: the ranks exchange CUDA IPC handles of their receive and staging
+    buffers over gloo and write into one another's memory with the peer kernels.  All processes share the one
+    visible GPU, which is legal because no kernel waits for another rank's kernel; each rank checks its own tokens
+    against the oracle and the exit codes carry the verdict."""
+    import subprocess
+    T, H, E, K, F = 96 * R, 256, 4 * R, 2, 128
+    port = free_port()
+    procs = []
+    for r in range(R):
+        env = dict(os.environ, RANK=str(r), WORLD_SIZE=str(R), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.join(ROOT, "tests", "ep_worker.py"),
+                                       *(str(v) for v in (T, H, E, K, F, inputs.BF16))], env=env,
+                                      stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True))
+    outs = []
+    for p in procs:
+        try:
+            out, _ = p.communicate(timeout=300)
+        except subprocess.TimeoutExpired:
+            p.kill()
+            out, _ = p.communicate()
+        outs.append(out)
+    assert [p.returncode for p in procs] == [0] * R, "\n".join(o[-2000:] for o in outs)
