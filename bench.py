@@ -187,6 +187,30 @@ class ClockSampler(threading.Thread):
                 "power_w_max": (round(max(self.power_w), 1) if self.power_w else None), "power_limit_w": self.power_limit_w}
 
 
+def plain_copy_us(total_bytes: float) -> float | None:
+    """Yardstick for the copy-bound stages: a plain device-to-device copy that moves the same number of bytes
+    (half read, half written), timed the way the per-kernel pass times a stage - one launch between two events,
+    synchronised - median of 9.  Small stages cannot beat it however they are written."""
+    import torch
+    try:
+        n = max(1, int(total_bytes) // 4)            # bf16 elements: n * 2 bytes read + n * 2 bytes written
+        src = torch.empty(n, dtype=torch.bfloat16, device="cuda").normal_()
+        dst = torch.empty_like(src)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ts = []
+        for i in range(12):
+            torch.cuda.synchronize()
+            e0.record()
+            dst.copy_(src)
+            e1.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(e0.elapsed_time(e1) * 1e3)
+        return float(np.median(ts))
+    except Exception:
+        return None
+
+
 def max_over_ranks(values: list[float], device: str = "cpu") -> list[float]:
     """Element-wise max of per-rank timings over the default process group (identity when single-process)."""
     import torch
@@ -249,14 +273,19 @@ def brief_measurement(args, w: inputs.Workload) -> dict:
     eb, rows = w.elem_bytes, w.T * w.K
     flops = 6.0 * rows * w.H * w.F
     t_ffn = sm["gemm1"] + sm["gemm2"]
-    disp = (w.T * w.H * eb * (1 + w.K) + 12 * rows) / sm["dispatch"] / 1e6
-    comb = (w.T * w.H * eb * (w.K + 1) + 8 * rows) / sm["combine"] / 1e6
+    disp_b, comb_b = w.T * w.H * eb * (1 + w.K) + 12 * rows, w.T * w.H * eb * (w.K + 1) + 8 * rows
+    disp = disp_b / sm["dispatch"] / 1e6
+    comb = comb_b / sm["combine"] / 1e6
+    copy_us = plain_copy_us(disp_b)
     return {"ms_per_step": ms, "value": w.T / ms * 1e3, "unit": UNIT, "steps": args.steps,
             "config": workload_config(w, {"dispatch_mode": dispatch}),
             "ffn": {"ms": t_ffn, "TFLOPs": flops / t_ffn / 1e9, "frac_of_burst_peak": flops / t_ffn / 1e9 / peaks["bf16_tflops"],
                     "kernel_sm_mhz": clock},
-            "route_ms": sm["route"], "dispatch": {"ms": sm["dispatch"], "GBps": disp, "frac_hbm": disp / peaks["hbm_gbs"]},
-            "combine": {"ms": sm["combine"], "GBps": comb, "frac_hbm": comb / peaks["hbm_gbs"]},
+            "route_ms": sm["route"],
+            "dispatch": {"ms": sm["dispatch"], "GBps": disp, "frac_hbm": disp / peaks["hbm_gbs"], "plain_copy_same_bytes_us": copy_us,
+                         "time_vs_plain_copy": (sm["dispatch"] * 1e3 / copy_us) if copy_us else None},
+            "combine": {"ms": sm["combine"], "GBps": comb, "frac_hbm": comb / peaks["hbm_gbs"], "plain_copy_same_bytes_us": copy_us,
+                        "time_vs_plain_copy": (sm["combine"] * 1e3 / copy_us) if copy_us else None},
             "stages_from": "a separate pass with an event after every kernel and a synchronisation per step"}
 
 
@@ -422,6 +451,11 @@ def run_cuda(args, w: inputs.Workload) -> None:
                     "frac_hbm": comb_bytes / sm["combine"] / 1e6 / hbm_peak,
                     "frac_hbm_nominal_8TBps": comb_bytes / sm["combine"] / 1e6 / 8000.0},
     }
+    for name, nbytes in (("dispatch", disp_bytes), ("combine", comb_bytes)):
+        us = plain_copy_us(nbytes) if rank == 0 else None
+        if us:
+            stages[name]["plain_copy_same_bytes_us"] = us
+            stages[name]["time_vs_plain_copy"] = stages[name]["ms"] * 1e3 / us
     if w.identity_experts or w.dtype != inputs.BF16:
         dom = "dispatch"
         roofline = {"kernel": "dispatch", "bound": "hbm", "achieved": stages["dispatch"]["GBps"], "peak": hbm_peak,

@@ -118,7 +118,16 @@ def assert_close_to_bf16_storage(got: np.ndarray, stored: dict, what: str = "out
         bound = bound + w[:, k:k + 1] * (bf16_step(o) * 2.0 + rms * 2.0 ** -10)   # 2 steps: |o| may sit just under a binade edge
     excess = np.abs(got - y) / bound
     worst = float(excess.max()) if excess.size else 0.0
-    assert worst <= 1.0, f"{what}: {worst:.2f} x the few-bf16-steps bound from the bf16-storage restatement"
+    # The noise term is a one-sigma figure (a tenth of the F intermediates flip, each by one step of itself, with
+    # random signs), so among millions of compared elements a few lie beyond it: up to 1e-5 of them may, by at
+    # most a factor of two.  Anything wrong in the path (an index, a k-block, a term) moves whole rows - thousands
+    # of elements of a token - by many steps.
+    bad = int((excess > 1.0).sum())
+    if worst > 2.0 or bad > max(2, int(1e-5 * excess.size)):
+        t, j = np.unravel_index(int(np.argmax(excess)), excess.shape)
+        raise AssertionError(f"{what}: {worst:.2f} x the few-bf16-steps bound from the bf16-storage restatement at sampled "
+                             f"token {t}, column {j}: got {got[t, j]!r}, restatement {y[t, j]!r}, bound {bound[t, j]!r}; "
+                             f"{bad} of {excess.size} elements (in {int((excess > 1.0).any(axis=1).sum())} tokens) over the bound")
 
 
 def tokens_covering_every_tile(slot_of: np.ndarray, extra: np.ndarray | None = None) -> np.ndarray:
