@@ -106,6 +106,7 @@ def test_overlapped_launch_full_size(w):
     plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, overlap=1)
     y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
     args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    plan.layer_tensor(2).fill_(1.0e30)     # a row consumed before it was stored would show in y
     plan.moe_layer(*args, y)
     torch.cuda.synchronize()
     assert plan.moe_last_status() == (0, 0)

@@ -440,6 +440,8 @@ def test_overlapped_dispatch_and_experts_match_oracle(w, split):
     y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
     args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
     for _ in range(2):      # twice: the second call meets the counters as the first one left them
+        # a row that a consumer read before its producer had stored it would show: the pool holds 1e30 everywhere
+        plan.layer_tensor(2).fill_(1.0e30)
         plan.moe_layer(*args, y)
         torch.cuda.synchronize()
         assert plan.moe_last_status() == (0, 0)
