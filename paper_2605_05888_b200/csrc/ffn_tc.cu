@@ -129,7 +129,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
   ClockProbe probe(prm.clock_probe);
   const unsigned long long wait_ns = prm.wait_ns;
 
-  const int NB1 = (F + 127) / 128;
+  const int NB1 = (F + 127) / 128, NB2 = (H + 255) / 256;
   const int KB1 = (H + kBK - 1) / kBK, KB2 = (F + kBK - 1) / kBK;
   int item_begin = 0, item_end = wl.seg_start[nseg];
   if (phase == 1) item_end = wl.n1;
@@ -174,8 +174,16 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
     it.m = m;
     it.cold = m < prm.cold_below;
     const int local = item - wl.seg_start[lo];
-    it.nb = local / m;
-    it.tile = wl.tiles[wl.estart[it.e] + local % m];
+    if (prm.band > 0 && m > prm.band) {
+      const int per_band = (it.type == 0 ? NB1 : NB2) * prm.band;  // every band but the last is full
+      const int j = local / per_band, rem = local - j * per_band;
+      const int bz = min(prm.band, m - j * prm.band);
+      it.nb = rem / bz;
+      it.tile = wl.tiles[wl.estart[it.e] + j * prm.band + rem % bz];
+    } else {
+      it.nb = local / m;
+      it.tile = wl.tiles[wl.estart[it.e] + local % m];
+    }
     return it;
   };
   volatile int* item_ring = sh->item_ring;
@@ -676,6 +684,7 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
   prm.item_ns = (p->trace && !pairs) ? p->s.item_ns : nullptr;
   prm.hist = nullptr;
   prm.hot_first = 0;
+  prm.band = 0;
   prm.push_src = push_src;
   OverlapParams ov = {};
   const bool overlap = overlap_x != nullptr && !pairs;
@@ -703,11 +712,15 @@ int launch_ffn_tc(moe_plan* p, const void* recv, const int* tile_expert, const v
       ovp = ov;
       prm.hist = p->s.hist;
       prm.hot_first = 1;
+      // Bands re-read an expert's gate and up matrices once per band: only where they stay in L2 meanwhile
+      // (58.7 MB on the DeepSeek-like layer; the Mixtral-like layer's 235 MB would be streamed again and again).
+      prm.band = (size_t)2 * c.F * c.H * 2 <= ((size_t)64 << 20) ? 4 : 0;
       return launch_pdl(ffn_tc_kernel, dim3(grid + ov.n_dispatch), dim3(kTcThreads), kTcSmem, st, a1, bg, bu, a2, bd, a1t, a2t, prm,
                         ovp) == cudaSuccess ? 0 : MOE_ERR_CUDA;
     }
     prm.hist = nullptr;
     prm.hot_first = 0;
+    prm.band = 0;
     return launch_pdl(ffn_tc_kernel, dim3(grid), dim3(kTcThreads), kTcSmem, st, a1, bg, bu, a2, bd, a1t, a2t, prm, ovp) == cudaSuccess
                ? 0 : MOE_ERR_CUDA;
   };

@@ -332,6 +332,9 @@ struct FfnParams {
                         // source is negative (empty slots); nullptr: rows stay where they are
   const int* hist;  // rows per expert (the ordered dispatch's counts): the work list is built from them, or nullptr
   int hot_first;    // with hist: experts are walked by descending row count
+  int band;         // > 0 (the launch that carries the dispatch): an expert's items go band by band of this many tiles
+                    // (column-block-major inside a band), so the first items need only the expert's first tiles,
+                    // which the token-ordered dispatch completes first; 0: column-block-major over all its tiles
   int thin;         // the narrow (transposed) form for single tiles of at most 64 rows is in use
   int cold_below;   // experts with fewer tiles than this stream their weights once: their loads are evict-first
   int phase, E, F, H;
