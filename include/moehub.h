@@ -147,7 +147,9 @@ int moe_plan_destroy(moe_plan_t* plan);
  * ascending fp32 FMA chain, softmax over the E experts, the K largest logits (lowest index
  * wins ties), in descending order.
  * d_x [T,H], d_wr [E,H] (dtype); d_bias [E] fp32 or NULL;
- * out: d_topk_idx [T,K] int32, d_topk_w [T,K] fp32. */
+ * out: d_topk_idx [T,K] int32, d_topk_w [T,K] fp32.
+ * An empty batch (T = 0) is legal in every call of this header: the per-token pointers may then be NULL,
+ * no kernel touches a row, and the dispatch outputs get their start state (counts 0, no tile owned). */
 int moe_route(moe_plan_t* plan, const void* d_x, const void* d_wr, const float* d_bias,
               int32_t* d_topk_idx, float* d_topk_w, void* stream);
 

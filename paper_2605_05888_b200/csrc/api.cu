@@ -227,7 +227,8 @@ int moe_plan_destroy(moe_plan_t* plan) {
 
 int moe_route(moe_plan_t* p, const void* d_x, const void* d_wr, const float* d_bias, int32_t* d_topk_idx,
               float* d_topk_w, void* stream) {
-  if (!p || !d_wr || !d_topk_idx || !d_topk_w || (!d_x && p->cfg.T > 0)) return MOE_ERR_ARG;
+  if (!p || !d_wr) return MOE_ERR_ARG;
+  if (p->cfg.T > 0 && (!d_x || !d_topk_idx || !d_topk_w)) return MOE_ERR_ARG;  // an empty batch has no rows to point at
   if (misaligned(d_x) || misaligned(d_wr)) return MOE_ERR_ALIGN;
   p->launches = 0;
   return launch_route(p, d_x, d_wr, d_bias, d_topk_idx, d_topk_w, nullptr, (cudaStream_t)stream) ? MOE_ERR_CUDA : MOE_OK;

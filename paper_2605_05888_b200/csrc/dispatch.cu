@@ -390,10 +390,10 @@ PrepArgs make_prep(moe_plan* p, int* expert_count, int* tile_expert, int* src_in
   add(rows_done, 1, 0);
   add(tile_count, P, 0);
   add(p->s.gemm1_done, P + 4, 0);
-  if (c.dispatch_mode == MOE_DISPATCH_ATOMIC_ORDERED) {
+  if (c.dispatch_mode == MOE_DISPATCH_ATOMIC_ORDERED && c.T > 0) {
     add(p->s.row_pointer, c.E, 0);  // expert_count, tile_expert and the empty slots' source info are written by the dispatch
     a.hist = p->s.hist;
-  } else {
+  } else {  // (an empty batch in the ordered scheme launches no dispatch: its outputs get their start state here)
     add(expert_count, c.E, 0);
     add(tile_expert, P, -1);
     add(src_info, (long long)P * kTileRows, -1);

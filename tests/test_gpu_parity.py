@@ -656,6 +656,61 @@ def test_random_small_layers_match_oracle(w):
         Hh.assert_output_close(Hh.to_host_f64(y), ref["y"], w.dtype)
 
 
+@pytest.mark.parametrize("w", [w for w in _random_workloads(24, 2024) if w.dtype == BF16][:10],
+                         ids=lambda w: f"{w.name}_T{w.T}_H{w.H}_E{w.E}_K{w.K}_F{w.F}")
+def test_random_small_layers_variants_agree_bit_for_bit(w):
+    """The variants of the bf16 layer do the same arithmetic in the same order per output element - ordered
+    dispatch with the dispatch inside the expert launch, push-style combine, both together - so on the same
+    seeded random shapes their y must equal the plain ordered layer's y bit for bit (which the test above holds
+    against the oracle)."""
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    ys = []
+    for kw in ({}, {"overlap": 1}, {"combine_mode": 1}, {"overlap": 1, "combine_mode": 1}):
+        plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, **kw)
+        y = torch.full((w.T, w.H), 7.0, dtype=torch.bfloat16, device="cuda")
+        for _ in range(2):
+            plan.moe_layer(*args, y)
+        torch.cuda.synchronize()
+        assert plan.moe_last_status() == (0, 0), kw
+        ys.append(y)
+    for kw, y in zip(("overlap", "push", "overlap + push"), ys[1:]):
+        assert torch.equal(y, ys[0]), kw
+
+
+@pytest.mark.parametrize("mode", MODES)
+@pytest.mark.parametrize("dtype", [BF16, FP32])
+def test_empty_batch_is_a_legal_call(mode, dtype):
+    """T = 0: every entry point accepts it, launches nothing that could touch a row, reports no error."""
+    w = inputs.Workload("empty", T=0, H=128, E=8, R=2, K=2, F=128, dtype=dtype)
+    _, wr, bias, wg, wu, wd = Hh.oracle_inputs(w.with_(T=4))
+    plan = Hh.make_plan(w, mode)
+    el = Hh.el_dtype(w)
+    x = torch.empty((0, w.H), dtype=el, device="cuda")
+    y = torch.empty((0, w.H), dtype=el, device="cuda")
+    idx = torch.empty((0, w.K), dtype=torch.int32, device="cuda")
+    tw = torch.empty((0, w.K), dtype=torch.float32, device="cuda")
+    dwr, dwg, dwu, dwd = (Hh.to_dev(a) for a in (wr, wg, wu, wd))
+    plan.moe_route(x, dwr, None, idx, tw)
+    rows = plan.P * 128
+    recv = torch.full((rows, w.H), 3.0, dtype=el, device="cuda")
+    cnt = torch.full((w.E,), 9, dtype=torch.int32, device="cuda")
+    te = torch.full((plan.P,), 9, dtype=torch.int32, device="cuda")
+    src = torch.full((rows,), 9, dtype=torch.int32, device="cuda")
+    slot = torch.empty((0, w.K), dtype=torch.int32, device="cuda")
+    plan.moe_dispatch(x, idx, recv, cnt, te, src, slot)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    assert cnt.eq(0).all() and te.eq(-1).all() and recv.eq(3.0).all()      # nobody owns a tile, no row was written
+    out_rows = torch.full((rows, w.H), 5.0, dtype=el, device="cuda")
+    plan.moe_expert_ffn(recv, te, dwg, dwu, dwd, out_rows)
+    plan.moe_combine(out_rows, slot, tw, y)
+    plan.moe_layer(x, dwr, None, dwg, dwu, dwd, y)
+    torch.cuda.synchronize()
+    assert plan.moe_last_status() == (0, 0)
+    assert out_rows.eq(5.0).all()                                          # no tile, no expert work
+
+
 def test_pipelined_host_steps_match_single_steps():
     """moe_layer_host_submit / _wait with two steps in flight: five batches, each result identical to
     the same batch run alone through moe_layer (bit for bit: same kernels, same order)."""
