@@ -27,6 +27,9 @@ SMALL = [
     inputs.Workload("k_equals_e", T=50, H=64, E=4, R=2, K=4, F=64, dtype=FP32),
     inputs.Workload("one_token", T=1, H=128, E=8, R=1, K=2, F=128, dtype=BF16),
     inputs.Workload("top1", T=130, H=128, E=16, R=4, K=1, F=136, dtype=BF16, zipf_s=1.2),
+    # the limits of the entry points: K = 32 picks per token, with 64 and with 256 experts
+    inputs.Workload("max_k", T=70, H=128, E=64, R=4, K=32, F=64, dtype=BF16),
+    inputs.Workload("max_e_max_k", T=45, H=64, E=256, R=8, K=32, F=64, dtype=BF16, zipf_s=1.0),
 ]
 
 
@@ -104,7 +107,7 @@ def test_tensor_core_ffn_forms_match_oracle(w, split, kernel):
 
 
 @pytest.mark.parametrize("mode", MODES)
-@pytest.mark.parametrize("w", [inputs.C1, SMALL[3], SMALL[5], inputs.C5(512), inputs.C5(256, 1.2)],
+@pytest.mark.parametrize("w", [inputs.C1, SMALL[3], SMALL[5], SMALL[9], SMALL[10], inputs.C5(512), inputs.C5(256, 1.2)],
                          ids=lambda w: w.name)
 def test_fused_layer_matches_oracle(w, mode):
     x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
@@ -424,7 +427,8 @@ def test_consumer_wait_runs_out_and_reports_it(kernel):
 OVERLAP_CASES = [SMALL[3], SMALL[4], SMALL[5], SMALL[7],
                  inputs.Workload("three_tiles", T=700, H=320, E=4, R=2, K=2, F=392, dtype=BF16),
                  inputs.Workload("many_items", T=2100, H=520, E=12, R=3, K=3, F=1032, dtype=BF16, seed=5, zipf_s=1.0),
-                 inputs.Workload("long_rows", T=260, H=9216, E=8, R=2, K=2, F=128, dtype=BF16)]   # rows of 18 KB: two chunks per row
+                 inputs.Workload("long_rows", T=260, H=9216, E=8, R=2, K=2, F=128, dtype=BF16),
+                 inputs.Workload("max_k_overlapped", T=70, H=128, E=64, R=4, K=32, F=64, dtype=BF16)]   # rows of 18 KB: two chunks per row
 
 
 @pytest.mark.parametrize("split", [1, 2])
