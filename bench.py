@@ -177,6 +177,13 @@ class ClockSampler(threading.Thread):
                 pass
             self._stop_evt.wait(0.005)
 
+    def energy_mj(self):
+        """The board's energy counter (millijoules since the driver was loaded), or None."""
+        try:
+            return float(self.nv.nvmlDeviceGetTotalEnergyConsumption(self.h)) if self.ok else None
+        except Exception:
+            return None
+
     def stop(self) -> dict:
         self._stop_evt.set()
         if self.is_alive():
@@ -352,13 +359,20 @@ def run_cuda(args, w: inputs.Workload) -> None:
     plan.moe_ffn_clock_mhz(reset=True)
     sampler.start()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    mj0 = sampler.energy_mj()
     e0.record(stream)
     for _ in range(args.steps):
         step()
     e1.record(stream)
     torch.cuda.synchronize()
+    mj1 = sampler.energy_mj()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop()
+    if mj0 is not None and mj1 is not None and mj1 > mj0:
+        # NVML's energy counter over the timed region (it advances in steps of some tens of milliseconds, so
+        # short regions read coarsely): joules per layer and the mean board power they imply.
+        clocks["energy_j_per_step"] = round((mj1 - mj0) / 1e3 / args.steps, 3)
+        clocks["mean_power_w"] = round((mj1 - mj0) / ms_total, 1)
     # SM clock the tensor-core expert kernel really ran at (cycles / time measured inside the kernel): THE clock
     # of the dominant kernel.  sm_mhz is what NVML returned when polled every 5 ms during the timed region; a
     # region of tens of milliseconds gives it a handful of samples, taken mostly between kernels.
