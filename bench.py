@@ -556,6 +556,9 @@ def run_cuda(args, w: inputs.Workload) -> None:
         cpu = {"value": n / secs, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": f"first {n} of {w.T} tokens, whole layer, {secs:.1f} s"}
 
+    if clocks.get("mean_power_w") and clocks.get("power_limit_w") and clocks["mean_power_w"] >= 0.93 * clocks["power_limit_w"]:
+        roofline["power_note"] = ("the board ran at its power limit during the timed region (clocks.mean_power_w of "
+                                  "clocks.power_limit_w): the kernel's clock, and with it both fractions, are set by the energy per step")
     h2d = w.T * w.H * eb
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
