@@ -7,6 +7,8 @@
 // the token's slots and weights once and broadcast them by shuffle; for every chunk the K row loads
 // are issued together, the sum runs in fp32 in ascending k (so the result is deterministic), and is
 // rounded once to the storage type.
+#include <climits>
+
 #include "common.cuh"
 
 namespace moehub {
@@ -18,7 +20,7 @@ template <typename XT, int KT>  // KT > 0: K known at compile time; KT == 0: run
 __global__ void __launch_bounds__(kCombThreads)
 combine_kernel(const uint4* __restrict__ rows, const int* __restrict__ slot_of,
                const float* __restrict__ topk_w, int T, int K_rt, int vec_per_row, int runs_per_row,
-               uint4* __restrict__ y, int staged) {
+               uint4* __restrict__ y, int staged, int row_limit) {
   constexpr int N = Vec16<XT>::N;
   constexpr int KMAX = KT > 0 ? KT : 1;
   const int K = KT > 0 ? KT : K_rt;
@@ -34,6 +36,9 @@ combine_kernel(const uint4* __restrict__ rows, const int* __restrict__ slot_of,
   if (lane < K) {
     my_slot = slot_of[(size_t)t * K + lane];
     my_w = topk_w[(size_t)t * K + lane];
+    // A slot beyond the rows there are is no slot (what a dispatch that gave up half-way leaves in the entries it
+    // never wrote): it adds nothing, like a dropped assignment, and nothing outside the buffer is read.
+    if (!staged && my_slot >= row_limit) my_slot = -1;
     // push-style combine: the experts stored assignment (t, k) at row t*K+k themselves; slot_of only says whether it exists
     if (staged && my_slot >= 0) my_slot = t * K + lane;
   }
@@ -100,9 +105,10 @@ static int launch_typed(moe_plan* p, const void* rows, const int* slot_of, const
   const int runs_per_row = (vec_per_row + kCombRun - 1) / kCombRun;
   const long long warps = (long long)c.T * runs_per_row;
   const int grid = (int)((warps + kCombThreads / 32 - 1) / (kCombThreads / 32));
+  const int row_limit = (int)min((long long)p->P * kTileRows, (long long)INT_MAX);
 #define MOEHUB_COMBINE(KT)                                                                          \
   launch_pdl(combine_kernel<XT, KT>, dim3(grid), dim3(kCombThreads), 0, st, (const uint4*)rows, slot_of, topk_w, \
-             c.T, c.K, vec_per_row, runs_per_row, (uint4*)y, staged ? 1 : 0)
+             c.T, c.K, vec_per_row, runs_per_row, (uint4*)y, staged ? 1 : 0, row_limit)
   switch (c.K) {
     case 1: MOEHUB_COMBINE(1); break;
     case 2: MOEHUB_COMBINE(2); break;

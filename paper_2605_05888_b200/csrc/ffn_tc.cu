@@ -62,6 +62,7 @@ struct TcShared {
   unsigned long long tmem_full[2];
   unsigned long long tmem_empty[2];
   unsigned long long item_bar[kItemRing];
+  unsigned long long drain;  // the MMA thread's last commit when it gives up: nothing of its own is in flight after it
   int item_ring[kItemRing];
   uint32_t tmem_base;
   int abort_flag;
@@ -98,6 +99,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
       mbar_init(smem_u32(&sh->tmem_empty[a]), 4);
     }
     for (int i = 0; i < kItemRing; ++i) mbar_init(smem_u32(&sh->item_bar[i]), 1);
+    mbar_init(smem_u32(&sh->drain), 1);
     sh->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -382,6 +384,14 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
         tc_commit(smem_u32(&sh->tmem_full[acc]));  // accumulator complete
       }
       if (fail_site) sh->abort_flag = 1;
+      if (fail_site || *abort_flag) {
+        // Giving up with MMAs possibly still running: they read the stages and write tensor memory, so wait
+        // (bounded) for all of them before the CTA frees either.
+        tc_commit(smem_u32(&sh->drain));
+        const unsigned long long t0 = globaltimer();
+        while (!mbar_try(smem_u32(&sh->drain), 0u))
+          if (globaltimer() - t0 > wait_ns + 1000000ull) break;
+      }
     }
   } else {
     // ===================== epilogue =====================
@@ -442,7 +452,10 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                   long long orow = (long long)(row0 + c + i);
-                  if (prm.push_src != nullptr) orow = __ldcg(prm.push_src + row0 + c + i);  // the row's own token position
+                  if (prm.push_src != nullptr) {  // the row's own token position; anything else (a stale word after a
+                    orow = __ldcg(prm.push_src + row0 + c + i);  // dispatch that gave up) is no position
+                    if (orow >= total_rows) orow = -1;
+                  }
                   if (orow >= 0) out[(size_t)orow * H + h] = __float2bfloat16_rn(__uint_as_float(v[i]));
                 }
               }
@@ -477,7 +490,7 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
         // information after its final GEMM and stores the result straight to the token's position.
         if (prm.push_src != nullptr) {
           const int src = __ldcg(prm.push_src + row);
-          if (src < 0) row_live = false;  // an empty slot: nothing to return
+          if (src < 0 || src >= total_rows) row_live = false;  // an empty slot (or no position at all): nothing to return
           else row = (size_t)src;
         }
         __nv_bfloat16* dst = out + row * H + (size_t)it.nb * 256;

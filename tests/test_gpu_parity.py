@@ -471,6 +471,10 @@ def test_overlapped_consumer_wait_runs_out_and_reports_it():
     args = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
     plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, overlap=1, wait_limit_ns=1000)
     y = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+    # The dispatch gives up half-way too (its own waits have the same limit) and leaves entries of slot_of and of
+    # the source information unwritten: whatever they hold must not be used as a row number by the later stages.
+    plan.layer_tensor(6).fill_(2 ** 31 - 1)
+    plan.layer_tensor(5).fill_(2 ** 31 - 1)
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
     plan.moe_layer(*args, y)
@@ -713,6 +717,29 @@ def test_empty_batch_is_a_legal_call(mode, dtype):
     torch.cuda.synchronize()
     assert plan.moe_last_status() == (0, 0)
     assert out_rows.eq(5.0).all()                                          # no tile, no expert work
+
+
+@pytest.mark.parametrize("dtype", [BF16, FP32])
+def test_combine_treats_a_slot_beyond_the_pool_as_absent(dtype):
+    """slot_of entries at or beyond the pool's rows (what an abandoned dispatch can leave behind) add nothing
+    and are never used as an address: y is the weighted sum over the valid slots only."""
+    w = inputs.Workload("bad_slots", T=64, H=256, E=8, R=2, K=4, F=128, dtype=dtype)
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED)
+    rows = plan.P * 128
+    g = torch.Generator(device="cuda").manual_seed(5)
+    pool = torch.randn((rows, w.H), device="cuda", generator=g).to(Hh.el_dtype(w))
+    slot = torch.randint(0, rows, (w.T, w.K), device="cuda", generator=g, dtype=torch.int32)
+    slot[::3, 1] = rows               # first row past the pool
+    slot[1::3, 2] = 2 ** 31 - 1       # as far out as an int goes
+    slot[2::3, 0] = -1                # a dropped assignment
+    tw = torch.rand((w.T, w.K), device="cuda", generator=g)
+    y = torch.empty((w.T, w.H), dtype=Hh.el_dtype(w), device="cuda")
+    plan.moe_combine(pool, slot, tw, y)
+    torch.cuda.synchronize()
+    valid = (slot >= 0) & (slot < rows)
+    want = (pool.double()[slot.clamp(0, rows - 1).long()] * (tw.double() * valid).unsqueeze(-1)).sum(1)
+    tol = 2.0 ** -7 if dtype == BF16 else 1e-5
+    assert torch.allclose(y.double(), want, rtol=tol, atol=tol)
 
 
 def test_pipelined_host_steps_match_single_steps():
