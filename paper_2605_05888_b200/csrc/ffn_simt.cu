@@ -17,12 +17,12 @@ template <typename XT, bool SWIGLU>
 __global__ void __launch_bounds__(kSimtThreads)
 ffn_simt_kernel(const XT* __restrict__ A, int lda, const int* __restrict__ tile_expert,
                 const XT* __restrict__ B1, const XT* __restrict__ B2, size_t expert_stride, int tp,
-                size_t shard_offset, int ldb, int N, int Kd, XT* __restrict__ C, int ldc) {
+                size_t shard_offset, int ldb, int N, int Kd, XT* __restrict__ C, int ldc, int E) {
   const int p = blockIdx.y;
   pdl_wait();
   pdl_trigger();
   const int e = tile_expert[p];
-  if (e < 0) return;
+  if (e < 0 || e >= E) return;  // no owner, or no expert at all (a caller's own table): nothing of the weights is read
   const int n0 = blockIdx.x * kSimtBN;
   const size_t row0 = (size_t)p * kTileRows;
   // e is a virtual expert: shard e % tp of expert e / tp (tp = 1: the expert itself)
@@ -100,11 +100,11 @@ static int launch_typed(moe_plan* p, const void* recv, const int* tile_expert, c
   mark(p, 3, st);
   dim3 g1((c.F + kSimtBN - 1) / kSimtBN, (unsigned)p->P);
   launch_pdl(ffn_simt_kernel<XT, true>, g1, dim3(kSimtThreads), 0, st, (const XT*)recv, c.H, tile_expert,
-             (const XT*)wg, (const XT*)wu, stride, tp, (size_t)c.F * c.H, c.H, c.F, c.H, (XT*)p->s.inter, c.F);
+             (const XT*)wg, (const XT*)wu, stride, tp, (size_t)c.F * c.H, c.H, c.F, c.H, (XT*)p->s.inter, c.F, c.E);
   mark(p, 4, st);
   dim3 g2((c.H + kSimtBN - 1) / kSimtBN, (unsigned)p->P);
   launch_pdl(ffn_simt_kernel<XT, false>, g2, dim3(kSimtThreads), 0, st, (const XT*)p->s.inter, c.F, tile_expert,
-             (const XT*)wd, (const XT*)nullptr, stride, tp, (size_t)c.F, c.F * tp, c.H, c.F, (XT*)out_rows, c.H);
+             (const XT*)wd, (const XT*)nullptr, stride, tp, (size_t)c.F, c.F * tp, c.H, c.F, (XT*)out_rows, c.H, c.E);
   p->launches += 2;
   return (int)cudaGetLastError();
 }
