@@ -16,7 +16,7 @@
 // another CTA anywhere in the dispatch.  Only the order of rows inside a region is decided at run time,
 // by one aggregated atomicAdd per touched expert per token block.
 //
-// Rows move with bulk asynchronous copies (cp.async.bulk, no tensor map, no multicast): one thread per
+// Rows move with plain bulk asynchronous copies (global to shared and back, no tensor map): one thread per
 // CTA loads a row (or a 16 KB chunk of it) into a ring of shared-memory buffers and stores it from there
 // to each of its K slots; the copies do not depend on resident warps or registers, loads run a few units
 // ahead of the stores, and up to 8 x K row stores are in flight per CTA.  A second warp raises the
