@@ -784,3 +784,27 @@ def test_layer_output_is_bit_identical_across_runs_and_dispatch_schemes():
             orders.append(plan.layer_tensor(6).cpu().numpy().tobytes())
     assert len(set(outs)) == 1
     assert len(set(orders)) > 1     # the placements did differ (scan vs atomic at the least)
+
+
+def test_overlapped_launch_many_runs_same_bytes():
+    """Forty runs of the overlapped launch on a layer with hot and cold experts (several tiles per hot expert, the
+    narrow form for the cold ones, two expert launches): every run must give the bytes of the stream-ordered layer,
+    with the receive pool refilled with 1e30 before each run - a consumer that started a tile too early, or a
+    counter left over from the run before, would change them."""
+    w = inputs.Workload("overlap_soak", T=3000, H=1024, E=48, R=4, K=4, F=512, dtype=BF16, zipf_s=1.0, seed=9)
+    x, wr, bias, wg, wu, wd = Hh.oracle_inputs(w)
+    dev = [Hh.to_dev(a) for a in (x, wr, bias, wg, wu, wd)]
+    base = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, ffn_split=1)
+    y0 = torch.empty((w.T, w.H), dtype=torch.bfloat16, device="cuda")
+    base.moe_layer(*dev, y0)
+    torch.cuda.synchronize()
+    assert base.moe_last_status() == (0, 0)
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_ORDERED, overlap=1, ffn_split=1)
+    y = torch.empty_like(y0)
+    for i in range(40):
+        plan.layer_tensor(2).fill_(1.0e30)
+        y.fill_(3.0)
+        plan.moe_layer(*dev, y)
+        torch.cuda.synchronize()
+        assert plan.moe_last_status() == (0, 0), i
+        assert torch.equal(y, y0), i
