@@ -120,7 +120,10 @@ typedef struct {
                                    floor(T*K*S/128) + E*S tiles, and the combine step adds the
                                    K*S partial rows.  Needs F % S == 0, E*S <= 256, K*S <= 32;
                                    0 or 1 = none                                               */
-  int32_t reserved_;            /* must be 0                                                  */
+  int32_t route_filter;         /* router with more than 64 experts on bf16 data: 0 = tensor-core filter
+                                   (approximate logits by tcgen05 MMAs, then the exact fp32 chain only
+                                   for the experts that can still be among the K largest: the picks
+                                   are the exact ones, bit for bit); -1 = every chain computed        */
   int64_t capacity_rows;        /* mode 1: rows per expert region, multiple of 128, 0 = T
                                    rounded up (overflow-free); modes 0/2: ignored            */
   uint64_t spin_limit;          /* bound (iterations) on the dispatch kernels' waits, 0 = 1<<22 */

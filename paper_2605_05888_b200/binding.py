@@ -34,7 +34,7 @@ class MoeConfig(ctypes.Structure):
                 ("identity_experts", ctypes.c_int32), ("ffn_kernel", ctypes.c_int32), ("ffn_split", ctypes.c_int32),
                 ("ffn_hot_min_tiles", ctypes.c_int32), ("ffn_thin_tiles", ctypes.c_int32),
                 ("overlap", ctypes.c_int32), ("combine_mode", ctypes.c_int32),
-                ("tp_shards", ctypes.c_int32), ("reserved_", ctypes.c_int32),
+                ("tp_shards", ctypes.c_int32), ("route_filter", ctypes.c_int32),
                 ("capacity_rows", ctypes.c_int64), ("spin_limit", ctypes.c_uint64), ("wait_limit_ns", ctypes.c_uint64)]
 
 
@@ -119,9 +119,9 @@ def _stream(stream) -> int:
 
 def make_config(T, H, E, R, K, F, dtype, renormalize=0, dispatch_mode=DISPATCH_ATOMIC_PAGED, identity_experts=0,
                 ffn_kernel=0, capacity_rows=0, spin_limit=0, ffn_split=0, wait_limit_ns=0,
-                ffn_hot_min_tiles=0, ffn_thin_tiles=0, overlap=0, combine_mode=0, tp_shards=0) -> MoeConfig:
+                ffn_hot_min_tiles=0, ffn_thin_tiles=0, overlap=0, combine_mode=0, tp_shards=0, route_filter=0) -> MoeConfig:
     return MoeConfig(T, H, E, R, K, F, dtype, int(renormalize), dispatch_mode, int(identity_experts), ffn_kernel, int(ffn_split),
-                     int(ffn_hot_min_tiles), int(ffn_thin_tiles), int(overlap), int(combine_mode), int(tp_shards), 0, capacity_rows, spin_limit, wait_limit_ns)
+                     int(ffn_hot_min_tiles), int(ffn_thin_tiles), int(overlap), int(combine_mode), int(tp_shards), int(route_filter), capacity_rows, spin_limit, wait_limit_ns)
 
 
 def moe_pool_tiles(cfg: MoeConfig) -> int:

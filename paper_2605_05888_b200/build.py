@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 SO = os.path.join(HERE, "libmoehub.so")
-SOURCES = ["api.cu", "route.cu", "dispatch.cu", "dispatch_ep.cu", "combine.cu", "ffn_simt.cu", "ffn_tc.cu", "ffn_tc2.cu"]
+SOURCES = ["api.cu", "route.cu", "route_filter.cu", "dispatch.cu", "dispatch_ep.cu", "combine.cu", "ffn_simt.cu", "ffn_tc.cu", "ffn_tc2.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

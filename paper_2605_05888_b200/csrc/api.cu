@@ -45,6 +45,7 @@ int check_config(const moe_config_t* user, Geometry* g) {
   if (!c->identity_experts && c->F <= 0) return MOE_ERR_ARG;
   if (c->E > 256 || c->K > 32) return MOE_ERR_UNSUPPORTED;
   if (c->combine_mode < 0 || c->combine_mode > 1) return MOE_ERR_ARG;
+  if (c->route_filter < -1 || c->route_filter > 0) return MOE_ERR_ARG;
   if (c->combine_mode == 1 && (c->dtype != MOE_DTYPE_BF16 || c->ffn_kernel != 0 || c->identity_experts))
     return MOE_ERR_UNSUPPORTED;
   const int eb = c->dtype == MOE_DTYPE_BF16 ? 2 : 4;
@@ -119,6 +120,9 @@ size_t carve(const moe_config_t& c, const Geometry& g, char* base, Scratch* s, s
   t.gemm1_done = (int*)take(sizeof(int) * (size_t)((g.P > 0 ? g.P : 1) + 4));  // + the expert kernel's item and exit counters
   const size_t pool_rows = (size_t)g.P * kTileRows;
   if (!c.identity_experts) t.inter = take(pool_rows * c.F * g.eb);
+  const bool filter = c.dtype == MOE_DTYPE_BF16 && c.E / g.tp > 64 && c.route_filter >= 0;  // c.E counts every TP shard
+  t.route_logits = filter ? (float*)take(sizeof(float) * (size_t)(c.T > 0 ? c.T : 1) * 256) : nullptr;
+  t.route_wnorm2 = filter ? (float*)take(sizeof(float) * 256) : nullptr;
   t.topk_idx = (int*)take(sizeof(int) * (size_t)c.T * c.K);
   t.topk_w = (float*)take(sizeof(float) * (size_t)c.T * c.K);
   t.recv = take(pool_rows * c.H * g.eb);

@@ -39,6 +39,8 @@ struct Scratch {          // device pointers carved out of the caller's workspac
   unsigned long long* item_ns;   // [4 * P * (NB1 + NB2)] work-item timeline of the tensor-core expert kernel (measurement)
   int* gemm1_done;        // [P+4]  per-tile status counter: GEMM1 blocks finished (x4 epilogue warps); [P..P+1] item counters, [P+2..P+3] exit counters of the expert kernel's launches
   void* inter;            // [P*128, F] SwiGLU intermediate
+  float* route_logits;    // [T, 256] approximate router logits of the tensor-core filter (wide router, bf16)
+  float* route_wnorm2;    // [256]    squared norms of the router's weight rows, recomputed by every call
   // moe_layer's internal buffers
   int* topk_idx;
   float* topk_w;
@@ -150,6 +152,10 @@ inline cudaError_t ensure_dynamic_smem(Kern kern, size_t bytes, int device, Smem
 // prep: the per-call resets and the row counts of an ordered dispatch that follows (nullptr: none).
 int launch_route(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx,
                  float* topk_w, const PrepArgs* prep, cudaStream_t st);
+// the tensor-core filter in front of the exact chains (many experts, bf16): see route_filter.cu
+bool route_filter_applies(const moe_plan* p);
+int launch_route_filter(moe_plan* p, const void* x, const void* wr, const float* bias, int* topk_idx, float* topk_w,
+                        const PrepArgs& prep, cudaStream_t st);
 // prepared: the kernel before this call has already done what make_prep() describes.
 int launch_dispatch(moe_plan* p, const void* x, const int* topk_idx, void* recv, int* expert_count,
                     int* tile_expert, int* src_info, int* slot_of, int* tile_count, int* rows_done,

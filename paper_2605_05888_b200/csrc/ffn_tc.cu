@@ -564,35 +564,6 @@ ffn_tc_kernel(const __grid_constant__ CUtensorMap map_a1, const __grid_constant_
 }
 
 // ---- host side ------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-static int get_encoder(moe_plan* p, EncodeTiledFn* fn) {
-  if (!p->encode_tiled) {
-    void* sym = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess || !sym ||
-        q != cudaDriverEntryPointSuccess)
-      return MOE_ERR_CUDA;
-    p->encode_tiled = sym;
-  }
-  *fn = (EncodeTiledFn)p->encode_tiled;
-  return MOE_OK;
-}
-
-// bf16 matrix [rows, cols] (row-major, cols contiguous), box [box_rows, 64 cols], 128-byte swizzle.
-static int make_map_2d(EncodeTiledFn enc, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
-                       uint32_t box_rows) {
-  cuuint64_t dims[2] = {cols, rows};
-  cuuint64_t strides[1] = {cols * 2};
-  cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
-  cuuint32_t estr[2] = {1, 1};
-  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  return r == CUDA_SUCCESS ? MOE_OK : MOE_ERR_CUDA;
-}
 // bf16 tensor [E, rows, cols], box [1, box_rows, 64].
 static int make_map_3d(EncodeTiledFn enc, CUtensorMap* m, const void* base, uint64_t E, uint64_t rows, uint64_t cols,
                        uint32_t box_rows) {

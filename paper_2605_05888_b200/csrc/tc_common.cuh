@@ -376,4 +376,35 @@ struct ClockProbe {
 int launch_ffn_tc2_kernel(const CUtensorMap& a1, const CUtensorMap& bg, const CUtensorMap& bu, const CUtensorMap& a2,
                           const CUtensorMap& bd, const FfnParams& prm, int grid, cudaStream_t st);
 
+// ---- tensor maps (host side) ---------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline int get_encoder(moe_plan* p, EncodeTiledFn* fn) {
+  if (!p->encode_tiled) {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &q) != cudaSuccess || !sym ||
+        q != cudaDriverEntryPointSuccess)
+      return MOE_ERR_CUDA;
+    p->encode_tiled = sym;
+  }
+  *fn = (EncodeTiledFn)p->encode_tiled;
+  return MOE_OK;
+}
+
+// bf16 matrix [rows, cols] (row-major, cols contiguous), box [box_rows, 64 cols], 128-byte swizzle.
+inline int make_map_2d(EncodeTiledFn enc, CUtensorMap* m, const void* base, uint64_t rows, uint64_t cols,
+                       uint32_t box_rows) {
+  cuuint64_t dims[2] = {cols, rows};
+  cuuint64_t strides[1] = {cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MOE_OK : MOE_ERR_CUDA;
+}
+
 }  // namespace moehub

@@ -449,7 +449,8 @@ def test_overlapped_dispatch_and_experts_match_oracle(w, split):
         plan.moe_layer(*args, y)
         torch.cuda.synchronize()
         assert plan.moe_last_status() == (0, 0)
-        assert plan.moe_last_launch_count() == 2 + (2 if split == 1 else 1)   # router, expert launch(es) carrying the dispatch, combine
+        router = 2 if (w.dtype == BF16 and w.E > 64) else 1                     # many experts on bf16: filter + refine
+        assert plan.moe_last_launch_count() == router + 1 + (2 if split == 1 else 1)   # router, expert launch(es) carrying the dispatch, combine
         Hh.check_route(plan.layer_tensor(0), plan.layer_tensor(1), ref["topk_idx"], ref["topk_w"])
         Hh.check_dispatch(w, plan.P, x, ref["topk_idx"], ref, plan.layer_tensor(2), plan.layer_tensor(3),
                           plan.layer_tensor(4), plan.layer_tensor(5), plan.layer_tensor(6))
@@ -808,3 +809,53 @@ def test_overlapped_launch_many_runs_same_bytes():
         torch.cuda.synchronize()
         assert plan.moe_last_status() == (0, 0), i
         assert torch.equal(y, y0), i
+
+
+def _route_only(w, x, wr, bias, **kw):
+    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED, **kw)
+    idx = torch.empty((w.T, w.K), dtype=torch.int32, device="cuda")
+    tw = torch.empty((w.T, w.K), dtype=torch.float32, device="cuda")
+    plan.moe_route(Hh.to_dev(x), Hh.to_dev(wr), Hh.to_dev(bias), idx, tw)
+    torch.cuda.synchronize()
+    return plan, idx, tw
+
+
+@pytest.mark.parametrize("case", ["zero_rows", "equal_experts", "near_ties"])
+def test_router_filter_degenerate_rows(case):
+    """The tensor-core filter of the wide router where its candidate sets are as large as they get: tokens that are
+    all zero (every logit equal: all 256 experts are candidates, the picks are experts 0..K-1), experts with identical
+    weight rows (exact ties decided by index), and logits a few ulps apart."""
+    w = inputs.Workload("filter_" + case, T=150, H=512, E=256, R=8, K=8, F=8, dtype=BF16, identity_experts=True, seed=4)
+    x, wr, bias, *_ = Hh.oracle_inputs(w, with_experts=False)
+    x, wr = x.copy(), wr.copy()
+    if case == "zero_rows":
+        x[::3] = 0
+    elif case == "equal_experts":
+        wr[1::2] = wr[0::2]                 # experts 2i and 2i+1 are the same row: every logit comes twice
+    else:
+        wr[:] = wr[0]                        # all experts alike ...
+        wr[:, 0] = inputs.fp32_to_bf16_bits(np.linspace(-1e-2, 1e-2, w.E).astype(np.float32))   # ... but for one column
+    _, idx, tw = _route_only(w, x, wr, None)
+    ridx, rw, _ = oracle.route(x, wr, None, w.K, w.dtype)
+    Hh.check_route(idx, tw, ridx, rw)
+    # and the plain chains-for-everybody router gives the same
+    _, idx2, tw2 = _route_only(w, x, wr, None, route_filter=-1)
+    assert torch.equal(idx, idx2)
+
+
+def test_router_filter_with_a_tiny_wait_limit_reports_or_routes():
+    """Every wait of the two filter kernels is bounded.  With a limit of a nanosecond a wait either still finds its
+    copy landed (a poll takes longer than that) or runs out: then the kernels give up by themselves and the status says
+    so.  Never a hang, never a wrong pick without a status; a plan with the normal limit routes correctly afterwards."""
+    w = inputs.Workload("filter_timeout", T=2048, H=2048, E=256, R=8, K=8, F=8, dtype=BF16, identity_experts=True)
+    x, wr, bias, *_ = Hh.oracle_inputs(w, with_experts=False)
+    ridx, rw, _ = oracle.route(x, wr, bias, w.K, w.dtype)
+    plan, idx, tw = _route_only(w, x, wr, bias, wait_limit_ns=1)
+    code, detail = plan.moe_last_status()
+    if code == 0:
+        Hh.check_route(idx, tw, ridx, rw)
+    else:
+        assert code == -6 and detail in (3, 4, 5), (code, detail)
+    plan2, idx2, tw2 = _route_only(w, x, wr, bias)
+    assert plan2.moe_last_status() == (0, 0)
+    Hh.check_route(idx2, tw2, ridx, rw)
