@@ -148,7 +148,9 @@ int moe_plan_destroy(moe_plan_t* plan);
 
 /* Step 1 (Section II-A, routing): logits l[t,e] = sum_h x[t,h]*Wr[e,h] (+bias[e]) as one
  * ascending fp32 FMA chain, softmax over the E experts, the K largest logits (lowest index
- * wins ties), in descending order.
+ * wins ties), in descending order.  (With more than 64 experts on bf16 data the chain is evaluated only for
+ * the experts that a tensor-core pass and an error bound derived from the data leave in question; the picks are
+ * those of the chains of all experts, bit for bit - see route_filter in moe_config_t.)
  * d_x [T,H], d_wr [E,H] (dtype); d_bias [E] fp32 or NULL;
  * out: d_topk_idx [T,K] int32, d_topk_w [T,K] fp32.
  * An empty batch (T = 0) is legal in every call of this header: the per-token pointers may then be NULL,

@@ -10,6 +10,11 @@
 // stage the operands and the others only compute.  Afterwards the logits
 // go through shared memory to one warp per token, which keeps them in registers (E/32 per lane)
 // and runs K rounds of a shuffle arg-max (ties: lowest expert index), then the softmax weights.
+//
+// With more than 64 experts on bf16 data the default is a different pair of kernels (route_filter.cu): tensor
+// cores compute approximate logits, and the exact chain runs only for the experts that can still be among the
+// K largest - the same picks, a fraction of the chains.  The kernels here remain the path for fp32 data, for
+// up to 64 experts, and for route_filter = -1.
 #include <float.h>
 
 #include "route_common.cuh"
