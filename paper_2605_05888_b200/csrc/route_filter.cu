@@ -68,7 +68,7 @@ route_tc_logits_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
-                 "r"(256u) : "memory");
+                 "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   pdl_wait();
@@ -121,7 +121,10 @@ route_tc_logits_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         const uint32_t a_addr = smem_u32(stage_base + stage * kStageBytes);
         const uint64_t adesc = smem_desc_sw128(a_addr), bdesc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
-        for (int k = 0; k < kBK / 16; ++k) tc_mma(tmem_base, adesc + 2 * k, bdesc + 2 * k, kIdesc, (kb | k) != 0 ? 1u : 0u);
+        // two accumulators, even and odd steps: half as many additions in a row for each logit (they are summed
+        // in the epilogue), which halves what the accumulation's rounding adds up to
+        for (int k = 0; k < kBK / 16; ++k)
+          tc_mma(tmem_base + (uint32_t)(kb & 1) * kRfEP, adesc + 2 * k, bdesc + 2 * k, kIdesc, ((kb >> 1) | k) != 0 ? 1u : 0u);
         tc_commit(smem_u32(&sh->empty[stage]));
         if (++stage == kStages) { stage = 0; phase_bit ^= 1u; }
       }
@@ -160,13 +163,16 @@ route_tc_logits_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       float* dst = logits + (size_t)t * kRfEP;
 #pragma unroll 1
       for (int c = 0; c < kRfEP; c += 16) {
-        uint32_t v[16];
+        uint32_t v[16], v2[16];
         tc_ld16(t_row + c, v);
+        tc_ld16(t_row + kRfEP + c, v2);
         tc_wait_ld();
         if (t < T) {
+          float f[16];
 #pragma unroll
-          for (int q = 0; q < 16; q += 4)
-            *reinterpret_cast<uint4*>(dst + c + q) = make_uint4(v[q], v[q + 1], v[q + 2], v[q + 3]);
+          for (int q = 0; q < 16; ++q) f[q] = KB > 1 ? __uint_as_float(v[q]) + __uint_as_float(v2[q]) : __uint_as_float(v[q]);
+#pragma unroll
+          for (int q = 0; q < 16; q += 4) *reinterpret_cast<float4*>(dst + c + q) = make_float4(f[q], f[q + 1], f[q + 2], f[q + 3]);
         }
       }
     }
@@ -177,7 +183,7 @@ route_tc_logits_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   __syncthreads();
   tc_fence_after();
   if (warp == 1)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(256u) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
 }
 
 
