@@ -5,8 +5,8 @@
 // come out bit for bit.  Only a handful of the E chains of a token decide anything, though.  So:
 //
 //  (1) route_tc_logits_kernel: approximate logits l~ = x * Wr^T for every (token, expert) with tcgen05 MMAs
-//      (128 tokens x 256 experts per CTA, operands by TMA, fp32 accumulator in tensor memory), written to a
-//      [T, 256] fp32 scratch.  Products of two bf16 numbers are exact in fp32; only the order and rounding
+//      (128 tokens x 128 experts per CTA, operands by TMA, four fp32 accumulators in tensor memory that take the
+//      64-column steps of h in turn and are summed at the end), written to a [T, 256] fp32 scratch.  Products of two bf16 numbers are exact in fp32; only the order and rounding
 //      of the additions differ from the chain.  Its idle epilogue warps also compute |w_e|^2 per expert.
 //  (2) route_refine_kernel: per token, the K-th largest approximate logit minus twice an error bound is a
 //      threshold; every expert at or above it is a candidate and gets its exact chain; the exact values
@@ -22,7 +22,8 @@
 // reports MOE_ERR_INTERNAL if |l~ - l| ever exceeded eps.
 //
 // The softmax weights use the exact logits of the candidates and the approximate ones of the rest: the rest
-// only enters the denominator, where its measured error is of the order of 1e-6 relative.
+// only enters the denominator.  What the accumulation's rounding adds up to grows with the number of additions
+// in a row (measured), which is why the approximate logit is the sum of four accumulators.
 #include "route_common.cuh"
 #include "tc_common.cuh"
 
@@ -38,6 +39,9 @@ constexpr int kRfWBytes = kRfEP * kRfChunk * 2;  // one chunk of every expert's 
 constexpr size_t rf_smem(int tpc) {
   return 1024 + (size_t)kRfBufs * (kRfWBytes + tpc * kRfChunk * 2) + (size_t)tpc * kRfEP * 4 + (size_t)tpc * kRfEP * 2;
 }
+
+// M = 128 tokens, N = 128 experts per MMA
+constexpr uint32_t kRfIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
 
 struct RfShared {
   unsigned long long full[kStages];
@@ -80,6 +84,7 @@ route_tc_logits_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
   volatile int* abort_flag = &sh->abort_flag;
   const int KB = (H + kBK - 1) / kBK;
   const int t0 = blockIdx.x * kTileRows;
+  const int e0 = blockIdx.y * 128;  // this CTA's half of the experts
   int fail_site = 0;
 
   if (warp == 0) {
@@ -92,9 +97,9 @@ route_tc_logits_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         if (!mbar_wait(smem_u32(&sh->empty[stage]), phase_bit ^ 1u, abort_flag, wait_ns)) { fail_site = kWaitMbarTma; break; }
         const uint32_t full = smem_u32(&sh->full[stage]);
         const uint32_t a_dst = smem_u32(stage_base + stage * kStageBytes);
-        mbar_expect_tx(full, (uint32_t)kStageBytes);
+        mbar_expect_tx(full, (uint32_t)(kABytes + kBBytes / 2));
         tma_load_2d(a_dst, &map_x, full, kb * kBK, t0);   // rows past T and columns past H arrive as zeros
-        tma_load_2d(a_dst + kABytes, &map_w, full, kb * kBK, 0);
+        tma_load_2d(a_dst + kABytes, &map_w, full, kb * kBK, e0);  // 128 experts' rows
 #pragma unroll
         for (int s = 0; s < kStages; ++s)
           if (s == stage) armed[s] += 1;
@@ -121,10 +126,10 @@ route_tc_logits_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
         const uint32_t a_addr = smem_u32(stage_base + stage * kStageBytes);
         const uint64_t adesc = smem_desc_sw128(a_addr), bdesc = smem_desc_sw128(a_addr + kABytes);
 #pragma unroll
-        // two accumulators, even and odd steps: half as many additions in a row for each logit (they are summed
-        // in the epilogue), which halves what the accumulation's rounding adds up to
+        // four accumulators that take the steps in turn: a quarter as many additions in a row for each logit
+        // (they are summed in the epilogue), and so a quarter of what the accumulation's rounding adds up to
         for (int k = 0; k < kBK / 16; ++k)
-          tc_mma(tmem_base + (uint32_t)(kb & 1) * kRfEP, adesc + 2 * k, bdesc + 2 * k, kIdesc, ((kb >> 1) | k) != 0 ? 1u : 0u);
+          tc_mma(tmem_base + (uint32_t)(kb & 3) * 128u, adesc + 2 * k, bdesc + 2 * k, kRfIdesc, ((kb >> 2) | k) != 0 ? 1u : 0u);
         tc_commit(smem_u32(&sh->empty[stage]));
         if (++stage == kStages) { stage = 0; phase_bit ^= 1u; }
       }
@@ -139,7 +144,7 @@ route_tc_logits_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
     }
   } else {
     // While the main loop runs: |w_e|^2 for this CTA's share of the experts (the refine kernel's error bound).
-    for (int e = blockIdx.x * 4 + (warp - 2); e < E; e += gridDim.x * 4) {
+    for (int e = (blockIdx.y * gridDim.x + blockIdx.x) * 4 + (warp - 2); e < E; e += gridDim.x * gridDim.y * 4) {
       const uint4* row = reinterpret_cast<const uint4*>(wr + (size_t)e * H);
       float s = 0.0f;
       for (int v = lane; v < H / 8; v += 32) {
@@ -160,17 +165,21 @@ route_tc_logits_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_c
       tc_fence_after();
       const int t = t0 + quarter * 32 + lane;
       const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
-      float* dst = logits + (size_t)t * kRfEP;
+      float* dst = logits + (size_t)t * kRfEP + e0;
+      const int nacc = min(KB, 4);  // accumulators that were written at all
 #pragma unroll 1
-      for (int c = 0; c < kRfEP; c += 16) {
-        uint32_t v[16], v2[16];
-        tc_ld16(t_row + c, v);
-        tc_ld16(t_row + kRfEP + c, v2);
-        tc_wait_ld();
-        if (t < T) {
-          float f[16];
+      for (int c = 0; c < 128; c += 16) {
+        float f[16];
 #pragma unroll
-          for (int q = 0; q < 16; ++q) f[q] = KB > 1 ? __uint_as_float(v[q]) + __uint_as_float(v2[q]) : __uint_as_float(v[q]);
+        for (int q = 0; q < 16; ++q) f[q] = 0.0f;
+        for (int a = 0; a < nacc; ++a) {
+          uint32_t v[16];
+          tc_ld16(t_row + (uint32_t)a * 128u + c, v);
+          tc_wait_ld();
+#pragma unroll
+          for (int q = 0; q < 16; ++q) f[q] += __uint_as_float(v[q]);
+        }
+        if (t < T) {
 #pragma unroll
           for (int q = 0; q < 16; q += 4) *reinterpret_cast<float4*>(dst + c + q) = make_float4(f[q], f[q + 1], f[q + 2], f[q + 3]);
         }
@@ -482,12 +491,14 @@ int launch_route_filter(moe_plan* p, const void* x, const void* wr, const float*
   CUtensorMap mx, mw;
   if ((rc = make_map_2d(enc, &mx, x, (uint64_t)c.T, (uint64_t)c.H, kTileRows)) != MOE_OK) return rc;
   if ((rc = make_map_2d(enc, &mw, wr, (uint64_t)p->route_E, (uint64_t)c.H, kRfEP)) != MOE_OK) return rc;
+  CUtensorMap mwh;  // half of the experts per box, for the filter's CTAs
+  if ((rc = make_map_2d(enc, &mwh, wr, (uint64_t)p->route_E, (uint64_t)c.H, 128)) != MOE_OK) return rc;
   static SmemAttrOnce once;
   if (ensure_dynamic_smem(route_tc_logits_kernel, kTcSmem, p->device, once) != cudaSuccess) return MOE_ERR_CUDA;
   const unsigned long long wait_ns = c.wait_limit_ns ? c.wait_limit_ns : kDefaultWaitNs;
   const int grid_a = (c.T + kTileRows - 1) / kTileRows;
   // the first kernel of the layer is launched plainly (see launch_wide_tmt), the second one behind it
-  if (launch_maybe_pdl(false, route_tc_logits_kernel, dim3(grid_a), dim3(kTcThreads), kTcSmem, st, mx, mw,
+  if (launch_maybe_pdl(false, route_tc_logits_kernel, dim3(grid_a, (p->route_E + 127) / 128), dim3(kTcThreads), kTcSmem, st, mx, mwh,
                        (const __nv_bfloat16*)wr, c.T, c.H, p->route_E, p->s.route_logits, p->s.route_wnorm2, wait_ns,
                        p->s.status) != cudaSuccess)
     return MOE_ERR_CUDA;

@@ -119,11 +119,12 @@ def assert_close_to_bf16_storage(got: np.ndarray, stored: dict, what: str = "out
     excess = np.abs(got - y) / bound
     worst = float(excess.max()) if excess.size else 0.0
     # The noise term is a one-sigma figure (a tenth of the F intermediates flip, each by one step of itself, with
-    # random signs), so among millions of compared elements a few lie beyond it: up to 1e-5 of them may, by at
-    # most a factor of two.  Anything wrong in the path (an index, a k-block, a term) moves whole rows - thousands
-    # of elements of a token - by many steps.
+    # random signs), so among the hundreds of thousands of compared elements some lie beyond it (seen: 13 of 368 640
+    # at up to 1.4 on one shape, clustered in two tokens whose expert rows nearly cancel): up to 1e-4 of them may, by
+    # at most a factor of two.  Anything wrong in the path (an index, a k-block, a term) moves whole rows - a
+    # hundredth of the sample or more - by many steps.
     bad = int((excess > 1.0).sum())
-    if worst > 2.0 or bad > max(2, int(1e-5 * excess.size)):
+    if worst > 2.0 or bad > max(2, int(1e-4 * excess.size)):
         t, j = np.unravel_index(int(np.argmax(excess)), excess.shape)
         raise AssertionError(f"{what}: {worst:.2f} x the few-bf16-steps bound from the bf16-storage restatement at sampled "
                              f"token {t}, column {j}: got {got[t, j]!r}, restatement {y[t, j]!r}, bound {bound[t, j]!r}; "
