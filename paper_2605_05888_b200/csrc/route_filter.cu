@@ -228,6 +228,7 @@ route_refine_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
   __shared__ int s_ncand[TPC];
   __shared__ float s_eps[TPC];
   __shared__ unsigned long long s_full[kRfBufs];
+  __shared__ unsigned long long s_empty[kRfBufs];  // a buffer may be refilled once every warp has left it
   __shared__ int s_abort;
   extern __shared__ uint8_t rf_dyn[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(rf_dyn) + 1023) & ~(uintptr_t)1023);
@@ -242,7 +243,10 @@ route_refine_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
   const bool live = tl < tvalid;
   const unsigned hmask = 0xffffu << (16 * half);
   if (threadIdx.x == 0) {
-    for (int b = 0; b < kRfBufs; ++b) mbar_init(smem_u32(&s_full[b]), 1);
+    for (int b = 0; b < kRfBufs; ++b) {
+      mbar_init(smem_u32(&s_full[b]), 1);
+      mbar_init(smem_u32(&s_empty[b]), NT / 32);
+    }
     s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -314,8 +318,17 @@ route_refine_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
   const int nchunk = (H + kRfChunk - 1) / kRfChunk;
   int issued = 0, consumed = 0;  // chunks over all passes: buffer = count % kRfBufs, phase = count / kRfBufs
   bool failed = false;
-  auto issue = [&](int ch) {  // thread 0 only
+  // The copies are issued by one thread: the first lane of the last warp, which has chains to run only when the
+  // CTA's list is full.  The warps are not held together by a barrier per step: each waits for the step's buffer,
+  // runs its chains over it and reports that it has left it; the issuing thread refills a buffer when all have.
+  const bool producer = threadIdx.x == NT - 32;
+  auto issue = [&](int ch) {  // the producer only
     const int b = issued % kRfBufs;
+    if (!mbar_wait(smem_u32(&s_empty[b]), ((uint32_t)(issued / kRfBufs) & 1u) ^ 1u, abort_flag, wait_ns)) {
+      failed = true;
+      s_abort = 1;
+      return;
+    }
     const uint32_t bar = smem_u32(&s_full[b]);
     mbar_expect_tx(bar, (uint32_t)(kRfWBytes + kXBytes));
     tma_load_2d(smem_u32(w_stage + (size_t)b * kRfWBytes), &map_w, bar, ch * kRfChunk, 0);   // rows past E, columns past H: zeros
@@ -388,11 +401,11 @@ route_refine_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
         xo[q] = (uint32_t)tk * 128u + (((uint32_t)q ^ (uint32_t)(tk & 7)) << 4);
       }
       const uint32_t w_base = smem_u32(w_stage), x_base = smem_u32(x_stage);
-      if (threadIdx.x == 0 && !failed)  // (after a wait that ran out nothing more is issued: a buffer may still be in flight)
-        for (int ch = 0; ch < kRfBufs - 1 && ch < nchunk; ++ch) issue(ch);
+      if (producer)  // (after a wait that ran out nothing more is issued: a buffer may still be in flight)
+        for (int ch = 0; ch < kRfBufs - 1 && ch < nchunk && !failed; ++ch) issue(ch);
       float acc = 0.0f;
       for (int ch = 0; ch < nchunk; ++ch) {
-        if (threadIdx.x == 0 && !failed && ch + kRfBufs - 1 < nchunk) issue(ch + kRfBufs - 1);  // its buffer was read last in step ch - 1
+        if (producer && !failed && ch + kRfBufs - 1 < nchunk) issue(ch + kRfBufs - 1);
         const int b = consumed % kRfBufs;
         // one lane per warp polls the barrier (a thousand pollers would keep the shared-memory pipe busy)
         if (lane == 0 && !failed && !mbar_wait(smem_u32(&s_full[b]), (uint32_t)(consumed / kRfBufs) & 1u, abort_flag, wait_ns)) {
@@ -417,7 +430,8 @@ route_refine_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
             acc = __fmaf_rn(bf16_hi(xa.w), bf16_hi(wa.w), acc);
           }
         }
-        __syncthreads();  // every chain is done with the buffer before it is refilled
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&s_empty[b]));  // this warp has left the buffer
       }
       if (e >= 0 && !failed) {
         const float exact = bias != nullptr ? acc + bias[e] : acc;
@@ -460,7 +474,7 @@ route_refine_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
   if (s_abort) {
     // A copy that was waited for too long is still on its way: every issued copy has to land before the CTA's
     // shared memory goes away (bounded again; the copies depend on nobody).
-    if (threadIdx.x == 0) {
+    if (producer) {
       for (int g = 0; g < issued; ++g) {
         if (g + kRfBufs < issued) continue;  // an older fill of the same buffer: the later one's phase covers it
         const unsigned long long ts = globaltimer();
