@@ -368,9 +368,10 @@ def run_cuda(args, w: inputs.Workload) -> None:
     mj1 = sampler.energy_mj()
     ms_total = e0.elapsed_time(e1)
     clocks = sampler.stop()
-    if mj0 is not None and mj1 is not None and mj1 > mj0:
-        # NVML's energy counter over the timed region (it advances in steps of some tens of milliseconds, so
-        # short regions read coarsely): joules per layer and the mean board power they imply.
+    if mj0 is not None and mj1 is not None and mj1 > mj0 and ms_total >= 800.0:
+        # NVML's energy counter over the timed region: joules per layer and the mean board power they imply.  The
+        # counter advances in steps of some tens of milliseconds and lags, so only regions of about a second or
+        # more are reported (--steps 150 or so on the default workload).
         clocks["energy_j_per_step"] = round((mj1 - mj0) / 1e3 / args.steps, 3)
         clocks["mean_power_w"] = round((mj1 - mj0) / ms_total, 1)
     # SM clock the tensor-core expert kernel really ran at (cycles / time measured inside the kernel): THE clock
