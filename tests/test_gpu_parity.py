@@ -578,6 +578,7 @@ def test_push_combine_is_refused_where_it_is_not_built():
 TP_CASES = [(inputs.Workload("tp_bf16", T=333, H=264, E=12, R=3, K=3, F=400, dtype=BF16), 2),
             (inputs.Workload("tp_bf16_4", T=700, H=320, E=4, R=2, K=2, F=1024, dtype=BF16, zipf_s=1.0), 4),
             (inputs.Workload("tp_many", T=300, H=256, E=64, R=8, K=8, F=256, dtype=BF16, zipf_s=1.0), 4),
+            (inputs.Workload("tp_filtered_router", T=260, H=512, E=128, R=8, K=4, F=256, dtype=BF16, zipf_s=1.0), 2),  # 128 experts: the router's filter path
             (inputs.Workload("tp_fp32", T=130, H=128, E=8, R=2, K=2, F=192, dtype=FP32), 3)]
 
 
