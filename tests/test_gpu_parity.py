@@ -166,9 +166,10 @@ def test_router_tie_patterns_exhaustive():
             Hh.check_route(idx, tw, ridx, rw)
 
 
+@pytest.mark.parametrize("E", [60, 160])   # the narrow router; the tensor-core filter of the wide one
 @pytest.mark.parametrize("renorm", [0, 1])
-def test_router_renormalize_and_bias(renorm):
-    w = inputs.Workload("renorm", T=200, H=512, E=60, R=4, K=4, F=8, dtype=BF16, zipf_s=1.0, seed=3)
+def test_router_renormalize_and_bias(renorm, E):
+    w = inputs.Workload("renorm", T=200, H=512, E=E, R=4, K=4, F=8, dtype=BF16, zipf_s=1.0, seed=3)
     x, wr, bias, *_ = Hh.oracle_inputs(w, with_experts=False)
     cfg = B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype, renormalize=renorm)
     plan = B.Plan(cfg)
@@ -201,13 +202,14 @@ def test_router_every_kernel_shape(shape):
     w = inputs.Workload("router_shape", T=T, H=H, E=E, R=1, K=K, F=8, dtype=dtype, zipf_s=zipf, seed=11,
                         identity_experts=True)
     x, wr, bias, *_ = Hh.oracle_inputs(w, with_experts=False)
-    plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED)
-    idx = torch.empty((T, K), dtype=torch.int32, device="cuda")
-    tw = torch.empty((T, K), dtype=torch.float32, device="cuda")
-    plan.moe_route(Hh.to_dev(x), Hh.to_dev(wr), Hh.to_dev(bias), idx, tw)
-    torch.cuda.synchronize()
     ridx, rw, _ = oracle.route(x, wr, bias, K, dtype)
-    Hh.check_route(idx, tw, ridx, rw)
+    for route_filter in ((0, -1) if (dtype == BF16 and E > 64) else (0,)):   # -1: the all-chains kernel for many experts
+        plan = Hh.make_plan(w, B.DISPATCH_ATOMIC_PAGED, route_filter=route_filter)
+        idx = torch.empty((T, K), dtype=torch.int32, device="cuda")
+        tw = torch.empty((T, K), dtype=torch.float32, device="cuda")
+        plan.moe_route(Hh.to_dev(x), Hh.to_dev(wr), Hh.to_dev(bias), idx, tw)
+        torch.cuda.synchronize()
+        Hh.check_route(idx, tw, ridx, rw)
 
 
 # ------------------------------------------------------------------ dispatch edge cases
