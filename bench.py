@@ -331,7 +331,7 @@ def run_cuda(args, w: inputs.Workload) -> None:
             "ordered": B.DISPATCH_ATOMIC_ORDERED}[dispatch]
     plan = B.Plan(B.make_config(w.T, w.H, w.E, w.R, w.K, w.F, w.dtype, dispatch_mode=mode,
                                 identity_experts=int(w.identity_experts), ffn_split=int(args.ffn_split),
-                                ffn_kernel=args.ffn_kernel, ffn_hot_min_tiles=args.ffn_hot_min_tiles, ffn_thin_tiles=args.ffn_thin_tiles,
+                                ffn_kernel=args.ffn_kernel, ffn_hot_min_tiles=args.ffn_hot_min_tiles, ffn_thin_tiles=args.ffn_thin_tiles, route_filter=args.route_filter,
                                 overlap=args.overlap, combine_mode=args.combine_mode, tp_shards=args.tp_shards))
     y = torch.empty((w.T, w.H), dtype=el, device="cuda")
     stream = torch.cuda.current_stream()
@@ -609,6 +609,7 @@ def main() -> None:
     ap.add_argument("--ffn-hot-min-tiles", type=int, default=0,
                     help="two-launch expert GEMMs: experts with at least this many tiles are walked as tensor-bound "
                          "work, interleaved with the weight-streaming-bound rest (0: library default, -1: off)")
+    ap.add_argument("--route-filter", type=int, default=0, choices=[0, -1], help="-1: the router computes every expert's chain (no tensor-core filter)")
     ap.add_argument("--ffn-thin-tiles", type=int, default=0, help="-1: no transposed narrow form for small single tiles")
     ap.add_argument("--tp-shards", type=int, default=0,
                     help="expert + tensor parallelism: every expert cut into this many shards with a receive region each")
